@@ -1,0 +1,153 @@
+"""CPU oracle (fp64, plain C) for paged GQA decode attention and KV append.
+
+TEST INFRASTRUCTURE ONLY: importable from ``tests/``, from the smoke check and
+from the benchmark's CPU-baseline leg. The CUDA library never imports it and it
+never imports the CUDA library.
+
+The arithmetic lives in ``pd_oracle.c`` (see its header for the definition and
+the pins); this module compiles it with gcc, loads it through ctypes and
+marshals NumPy arrays. bf16 tensors travel as ``uint16`` bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "pd_oracle.c")
+_LIB = os.path.join(_HERE, "libpd_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile ``pd_oracle.c`` into ``libpd_oracle.so`` (gcc, no fast-math)."""
+    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    if force or stale:
+        tmp = f"{_LIB}.{os.getpid()}.tmp"
+        subprocess.run(
+            ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-pthread", _SRC, "-o", tmp, "-lm"],
+            check=True,
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        p = ctypes.c_void_p
+        i = ctypes.c_int
+        lib.pd_oracle_decode_attn.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, i, ctypes.c_float, p, p, i]
+        lib.pd_oracle_decode_attn.restype = i
+        lib.pd_oracle_lse_merge.argtypes = [p, p, i, i, p, p]
+        lib.pd_oracle_lse_merge.restype = i
+        lib.pd_oracle_kv_append.argtypes = [p, p, p, p, p, p, i, i, i, i, i, ctypes.c_int64, i]
+        lib.pd_oracle_kv_append.restype = i
+        _lib = lib
+    return _lib
+
+
+def bf16_bits(t) -> np.ndarray:
+    """Bit patterns (uint16, C-contiguous) of a bf16 torch tensor on any device."""
+    import torch
+
+    assert t.dtype == torch.bfloat16
+    return t.detach().contiguous().cpu().view(torch.int16).numpy().view(np.uint16)
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round-to-nearest-even fp32 -> bf16 bit patterns (finite inputs)."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    rounded = (u + 0x7FFF + ((u >> 16) & 1)) >> 16
+    return rounded.astype(np.uint16)
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Exact widening of bf16 bit patterns to fp64."""
+    u = np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << 16
+    return u.view(np.float32).astype(np.float64)
+
+
+def _c(a: np.ndarray, dtype) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def decode_attn(q, k_pages, v_pages, page_table, ctx_lens, sm_scale, *, t_begin=None, t_end=None,
+                nthreads: int | None = None):
+    """softmax(sm_scale * q K^T) V per (sequence, query head) over a paged cache.
+
+    q: uint16 [B, Hq, d]; k_pages/v_pages: uint16 [NP, Hkv, P, d];
+    page_table: int32 [B, MP]; ctx_lens: int32 [B]. Optional ``t_begin`` /
+    ``t_end`` (int32 [B]) restrict every sequence to a token range (used to form
+    split partials). Returns (out fp64 [B, Hq, d], lse fp64 [B, Hq]).
+    """
+    lib = _load()
+    q = _c(q, np.uint16)
+    k_pages = _c(k_pages, np.uint16)
+    v_pages = _c(v_pages, np.uint16)
+    page_table = _c(page_table, np.int32)
+    ctx_lens = _c(ctx_lens, np.int32)
+    B, Hq, d = q.shape
+    NP, Hkv, P, d2 = k_pages.shape
+    assert d2 == d and v_pages.shape == k_pages.shape
+    assert page_table.ndim == 2 and page_table.shape[0] >= B and ctx_lens.shape[0] >= B
+    MP = page_table.shape[1]
+    # every page the definition will touch must exist
+    for b in range(B):
+        lo = 0 if t_begin is None else int(t_begin[b])
+        hi = int(ctx_lens[b]) if t_end is None else int(t_end[b])
+        if hi > lo:
+            assert hi <= MP * P
+            used = page_table[b, lo // P:(hi + P - 1) // P]
+            assert used.min() >= 0 and used.max() < NP, "page id out of range"
+    tb = None if t_begin is None else _c(t_begin, np.int32)
+    te = None if t_end is None else _c(t_end, np.int32)
+    out = np.empty((B, Hq, d), dtype=np.float64)
+    lse = np.empty((B, Hq), dtype=np.float64)
+    if nthreads is None:
+        nthreads = os.cpu_count() or 1
+    rc = lib.pd_oracle_decode_attn(
+        q.ctypes.data, k_pages.ctypes.data, v_pages.ctypes.data, page_table.ctypes.data,
+        ctx_lens.ctypes.data, None if tb is None else tb.ctypes.data,
+        None if te is None else te.ctypes.data, B, Hq, Hkv, d, P, MP,
+        ctypes.c_float(np.float32(sm_scale)), out.ctypes.data, lse.ctypes.data, int(nthreads))
+    if rc != 0:
+        raise RuntimeError(f"pd_oracle_decode_attn failed ({rc})")
+    return out, lse
+
+
+def lse_merge(o_parts, lse_parts):
+    """Merge partial results of one row. o_parts fp64 [n, d], lse_parts fp64 [n]."""
+    lib = _load()
+    o_parts = _c(o_parts, np.float64)
+    lse_parts = _c(lse_parts, np.float64)
+    n, d = o_parts.shape
+    out = np.empty(d, dtype=np.float64)
+    lse = np.empty(1, dtype=np.float64)
+    rc = lib.pd_oracle_lse_merge(o_parts.ctypes.data, lse_parts.ctypes.data, n, d, out.ctypes.data,
+                                 lse.ctypes.data)
+    if rc != 0:
+        raise RuntimeError(f"pd_oracle_lse_merge failed ({rc})")
+    return out, float(lse[0])
+
+
+def kv_append(k_new, v_new, k_pages, v_pages, page_table, ctx_lens, *, advance: bool = True) -> int:
+    """In-place one-token append on host mirrors of the pools (uint16) and ctx_lens (int32)."""
+    lib = _load()
+    for a, dt in ((k_pages, np.uint16), (v_pages, np.uint16), (ctx_lens, np.int32)):
+        assert isinstance(a, np.ndarray) and a.dtype == dt and a.flags.c_contiguous and a.flags.writeable
+    k_new = _c(k_new, np.uint16)
+    v_new = _c(v_new, np.uint16)
+    page_table = _c(page_table, np.int32)
+    B, Hkv, d = k_new.shape
+    NP, Hkv2, P, d2 = k_pages.shape
+    assert (Hkv2, d2) == (Hkv, d) and v_pages.shape == k_pages.shape and v_new.shape == k_new.shape
+    return lib.pd_oracle_kv_append(
+        k_new.ctypes.data, v_new.ctypes.data, k_pages.ctypes.data, v_pages.ctypes.data,
+        page_table.ctypes.data, ctx_lens.ctypes.data, B, Hkv, d, P, page_table.shape[1], NP,
+        1 if advance else 0)

@@ -1,0 +1,229 @@
+/*
+ * CPU oracle for paged grouped-query decode attention and the 1-token KV append.
+ *
+ * TEST INFRASTRUCTURE ONLY. This file is the slow, plain statement of what the
+ * path computes. It shares no code with the CUDA library, is never linked into
+ * it and must never be called from a product path.
+ *
+ * What it states. The paper's decode cost model has a per-sequence term b whose
+ * source is the extra KV-cache HBM reads of every concurrently decoding
+ * sequence (Eq. 1, text below it), and every generated token joins the context
+ * of its trajectory (Sec. 2.1, p_{i+1} = p_i + r_i + o_i). The paper prints no
+ * attention formula; the computation behind the b term is scaled dot-product
+ * attention of one new query token over the cached tokens, with each KV head
+ * shared by a contiguous group of query heads:
+ *
+ *   kvh = h / g,            g = num_q_heads / num_kv_heads
+ *   K_t = k_pages[page_table[b][t / P]][kvh][t % P][:]     t = 0 .. L_b - 1
+ *   s_t = sm_scale * <q[b][h], K_t>
+ *   out[b][h] = sum_t softmax(s)_t * V_t,    lse[b][h] = log sum_t exp(s_t)
+ *
+ * Everything is evaluated in fp64 in index order, two passes (max, then sums),
+ * no blocking, no online rescaling. bf16 inputs convert to fp64 exactly.
+ *
+ * Pins (tests/test_oracle_pins.py): one-token context, identical keys, two
+ * closed forms (tanh(1/2); a three-token softmax), brute force on tiny inputs,
+ * an independently written NumPy formulation, page-permutation invariance,
+ * shift invariance, poison in masked slots, overflow safety, split + LSE merge
+ * over every partition of a short context.
+ *
+ * Pool layout (a choice of this repository, the paper describes none):
+ *   k_pages, v_pages : [num_pages][num_kv_heads][page_size][head_dim] bf16
+ *   page_table       : [batch][max_pages_per_seq] int32, entry i = physical
+ *                      page of tokens [i*P, (i+1)*P); entries past
+ *                      ceil(L/P) are never read
+ *   ctx_lens         : [batch] int32
+ */
+#include <math.h>
+#include <pthread.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+static double bf16_to_f64(uint16_t bits)
+{
+    uint32_t u = ((uint32_t)bits) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+typedef struct {
+    const uint16_t *q, *k_pages, *v_pages;
+    const int32_t *page_table, *ctx_lens;
+    const int32_t *t_begin, *t_end; /* optional per-sequence token range */
+    int B, Hq, Hkv, d, P, MP;
+    double scale;
+    double *out, *lse;
+    int next_row; /* work counter, guarded by mu */
+    pthread_mutex_t mu;
+} attn_job;
+
+/* One (sequence, query head) row: the definition, written out. */
+static void attn_row(const attn_job *J, int b, int h, double *s_buf)
+{
+    const int d = J->d, P = J->P;
+    const int g = J->Hq / J->Hkv;
+    const int kvh = h / g;
+    int t0 = 0, t1 = J->ctx_lens[b];
+    if (J->t_begin) t0 = J->t_begin[b];
+    if (J->t_end) t1 = J->t_end[b];
+    double *o = J->out + ((size_t)b * J->Hq + h) * d;
+    for (int j = 0; j < d; ++j) o[j] = 0.0;
+    if (t1 <= t0) { /* empty context: zero output, lse = -inf */
+        J->lse[(size_t)b * J->Hq + h] = -INFINITY;
+        return;
+    }
+    const uint16_t *qrow = J->q + ((size_t)b * J->Hq + h) * d;
+    const size_t page_stride = (size_t)J->Hkv * P * d;
+    /* pass 1: logits and their maximum */
+    double m = -INFINITY;
+    for (int t = t0; t < t1; ++t) {
+        int32_t page = J->page_table[(size_t)b * J->MP + t / P];
+        const uint16_t *krow = J->k_pages + (size_t)page * page_stride + ((size_t)kvh * P + t % P) * d;
+        double dot = 0.0;
+        for (int j = 0; j < d; ++j) dot += bf16_to_f64(qrow[j]) * bf16_to_f64(krow[j]);
+        double s = J->scale * dot;
+        s_buf[t - t0] = s;
+        if (s > m) m = s;
+    }
+    /* pass 2: normaliser and weighted sum of V */
+    double Z = 0.0;
+    for (int t = t0; t < t1; ++t) {
+        double p = exp(s_buf[t - t0] - m);
+        Z += p;
+        int32_t page = J->page_table[(size_t)b * J->MP + t / P];
+        const uint16_t *vrow = J->v_pages + (size_t)page * page_stride + ((size_t)kvh * P + t % P) * d;
+        for (int j = 0; j < d; ++j) o[j] += p * bf16_to_f64(vrow[j]);
+    }
+    for (int j = 0; j < d; ++j) o[j] /= Z;
+    J->lse[(size_t)b * J->Hq + h] = m + log(Z);
+}
+
+static void *attn_worker(void *arg)
+{
+    attn_job *J = (attn_job *)arg;
+    int maxlen = 1;
+    for (int b = 0; b < J->B; ++b) {
+        int t0 = J->t_begin ? J->t_begin[b] : 0;
+        int t1 = J->t_end ? J->t_end[b] : J->ctx_lens[b];
+        if (t1 - t0 > maxlen) maxlen = t1 - t0;
+    }
+    double *s_buf = (double *)malloc(sizeof(double) * (size_t)maxlen);
+    if (!s_buf) return (void *)1;
+    const int rows = J->B * J->Hq;
+    for (;;) {
+        pthread_mutex_lock(&J->mu);
+        int r = J->next_row++;
+        pthread_mutex_unlock(&J->mu);
+        if (r >= rows) break;
+        attn_row(J, r / J->Hq, r % J->Hq, s_buf);
+    }
+    free(s_buf);
+    return NULL;
+}
+
+/*
+ * Attention over tokens [t_begin[b], t_end[b]) of every sequence (NULL range
+ * pointers mean [0, ctx_lens[b])). out: [B][Hq][d] fp64, lse: [B][Hq] fp64.
+ * Returns 0, or -1 on bad arguments / allocation failure.
+ */
+int pd_oracle_decode_attn(const uint16_t *q, const uint16_t *k_pages, const uint16_t *v_pages,
+                          const int32_t *page_table, const int32_t *ctx_lens,
+                          const int32_t *t_begin, const int32_t *t_end,
+                          int B, int Hq, int Hkv, int d, int P, int MP, float sm_scale,
+                          double *out, double *lse, int nthreads)
+{
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || d <= 0 || P <= 0 || MP <= 0) return -1;
+    if (nthreads < 1) nthreads = 1;
+    if (nthreads > 256) nthreads = 256;
+    attn_job J;
+    J.q = q; J.k_pages = k_pages; J.v_pages = v_pages;
+    J.page_table = page_table; J.ctx_lens = ctx_lens;
+    J.t_begin = t_begin; J.t_end = t_end;
+    J.B = B; J.Hq = Hq; J.Hkv = Hkv; J.d = d; J.P = P; J.MP = MP;
+    J.scale = (double)sm_scale; /* the fp32 value the caller passes, widened */
+    J.out = out; J.lse = lse; J.next_row = 0;
+    pthread_mutex_init(&J.mu, NULL);
+    int rc = 0;
+    if (nthreads == 1) {
+        if (attn_worker(&J) != NULL) rc = -1;
+    } else {
+        pthread_t th[256];
+        int started = 0;
+        for (int i = 0; i < nthreads; ++i) {
+            if (pthread_create(&th[i], NULL, attn_worker, &J) != 0) break;
+            ++started;
+        }
+        if (started == 0) rc = -1;
+        for (int i = 0; i < started; ++i) {
+            void *ret = NULL;
+            pthread_join(th[i], &ret);
+            if (ret != NULL) rc = -1;
+        }
+    }
+    pthread_mutex_destroy(&J.mu);
+    return rc;
+}
+
+/*
+ * Merge of n partial results of ONE row, each the attention over a disjoint
+ * part of the context: o_parts [n][d] (each already normalised over its part),
+ * lse_parts [n]. With w_i = exp(lse_i - max lse):
+ *   out = sum_i w_i o_i / sum_i w_i,   lse = max lse + log sum_i w_i
+ * Parts with lse = -inf (empty) carry no weight.
+ */
+int pd_oracle_lse_merge(const double *o_parts, const double *lse_parts, int n, int d,
+                        double *out, double *lse)
+{
+    if (n < 0 || d <= 0) return -1;
+    double M = -INFINITY;
+    for (int i = 0; i < n; ++i)
+        if (lse_parts[i] > M) M = lse_parts[i];
+    for (int j = 0; j < d; ++j) out[j] = 0.0;
+    if (M == -INFINITY) {
+        *lse = -INFINITY;
+        return 0;
+    }
+    double W = 0.0;
+    for (int i = 0; i < n; ++i) {
+        if (lse_parts[i] == -INFINITY) continue;
+        double w = exp(lse_parts[i] - M);
+        W += w;
+        for (int j = 0; j < d; ++j) out[j] += w * o_parts[(size_t)i * d + j];
+    }
+    for (int j = 0; j < d; ++j) out[j] /= W;
+    *lse = M + log(W);
+    return 0;
+}
+
+/*
+ * One-token append (Sec. 2.1: each generated token extends its trajectory's
+ * context): for every sequence b, pos = ctx_lens[b], the d bf16 values of each
+ * KV head of k_new[b] / v_new[b] ([B][Hkv][d]) are copied into slot pos % P of
+ * page page_table[b][pos / P]; then ctx_lens[b] += 1 when advance != 0.
+ * Pure byte copy. Returns 0, or -(b+1) for the first sequence whose position
+ * or page id is out of range (nothing is written for that sequence).
+ */
+int pd_oracle_kv_append(const uint16_t *k_new, const uint16_t *v_new,
+                        uint16_t *k_pages, uint16_t *v_pages,
+                        const int32_t *page_table, int32_t *ctx_lens,
+                        int B, int Hkv, int d, int P, int MP, int64_t num_pages, int advance)
+{
+    int rc = 0;
+    const size_t page_stride = (size_t)Hkv * P * d;
+    for (int b = 0; b < B; ++b) {
+        int pos = ctx_lens[b];
+        if (pos < 0 || pos / P >= MP) { if (!rc) rc = -(b + 1); continue; }
+        int32_t page = page_table[(size_t)b * MP + pos / P];
+        if (page < 0 || (int64_t)page >= num_pages) { if (!rc) rc = -(b + 1); continue; }
+        for (int kvh = 0; kvh < Hkv; ++kvh) {
+            size_t dst = (size_t)page * page_stride + ((size_t)kvh * P + pos % P) * d;
+            size_t src = ((size_t)b * Hkv + kvh) * d;
+            memcpy(k_pages + dst, k_new + src, sizeof(uint16_t) * (size_t)d);
+            memcpy(v_pages + dst, v_new + src, sizeof(uint16_t) * (size_t)d);
+        }
+        if (advance) ctx_lens[b] = pos + 1;
+    }
+    return rc;
+}
