@@ -1,0 +1,395 @@
+"""Benchmark of the paged decode-attention hot path on B200.
+
+One step = one pass of the whole path over one batch: KV append of one token
+per sequence, then split-KV attention and the LSE merge over the grown contexts.
+The headline value is achieved KV-cache read bandwidth (GB/s): the bytes of K
+and V every query must read, divided by the time of the whole step. Inputs are
+synthetic, shaped like the paper's rollout workloads (see ``workloads``).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl cuda|reference]
+
+Prints ONE JSON line on rank 0. ``--impl reference`` times the CPU oracle (test
+infrastructure, run as it stands) on the host cores instead of the CUDA path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "decode-attn achieved HBM GB/s (% of B200 peak) and seq-steps/s per layer"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per launch of the split kernel from the committed ncu capture, as a
+# ratio to the algorithmic KV bytes of that launch (profiles/); None = no capture yet.
+NCU_TRAFFIC_RATIO = None
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    REASONS = {
+        0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x10: "sync_boost",
+        0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+        0x100: "display_clock_setting",
+    }
+
+    def __init__(self, device_index: int, period_s: float = 0.002):
+        super().__init__(daemon=True)
+        self.period = period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            import torch
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception as e:  # NVML missing: report that instead of clocks
+            self.err = repr(e)
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+                bits = int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["nvml unavailable"]}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def aggregate_over_ranks(local_ms: float, local_units: float, world_size: int, backend_device=None):
+    """Whole-job figures: time = max over ranks, units = sum over ranks (no data-path collective)."""
+    if world_size == 1:
+        return local_ms, local_units
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([local_ms], dtype=torch.float64, device=backend_device)
+    u = torch.tensor([local_units], dtype=torch.float64, device=backend_device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def workload_config(w, lens, cfg_id):
+    return {
+        "workload": f"configs[{cfg_id}] {w.name}", "batch": int(w.batch), "num_q_heads": w.num_q_heads,
+        "num_kv_heads": w.num_kv_heads, "head_dim": w.head_dim, "page_size": w.page_size,
+        "ctx_tokens_total": int(np.sum(lens)), "ctx_len_min": int(np.min(lens)), "ctx_len_max": int(np.max(lens)),
+    }
+
+
+# ------------------------------------------------------------------------------------------ CUDA arm
+
+def run_cuda(args):
+    import torch
+
+    import paper_2609_35158_b200 as pd
+    import workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    cfg_id = args.config
+    w = wl.WORKLOADS[cfg_id]
+    K, W = args.steps, args.warmup
+    # weak scaling: every rank holds its own batch of the same shape (sequences are independent)
+    seed = cfg_id + 1000 * rank
+    lens0 = wl.context_lengths(cfg_id, seed=seed)
+    B = w.batch
+    total_steps = 2 * (W + K) + 8  # device-resident loop, then the host-buffer loop
+    dynamic_alloc = cfg_id == 4   # pages handed out by the host free list inside the loop
+    cache = wl.build_paged_cache(lens0, w.num_kv_heads, w.head_dim, seed=seed, device=dev,
+                                 reserve_tokens=total_steps, preassign_reserve=not dynamic_alloc)
+    alloc = wl.PageAllocator(cache)
+    ctx = pd.pd_create(w.num_q_heads, w.num_kv_heads, w.head_dim, w.page_size, B, cache.page_table.shape[1],
+                       cache.num_pages, local_rank)
+    R = 4  # rotating activations so no step re-reads the previous step's q / k_new / v_new from L2
+    qs = [wl.random_bf16((B, w.num_q_heads, w.head_dim), seed * 100 + 10 + i, dev) for i in range(R)]
+    kns = [wl.random_bf16((B, w.num_kv_heads, w.head_dim), seed * 100 + 20 + i, dev) for i in range(R)]
+    vns = [wl.random_bf16((B, w.num_kv_heads, w.head_dim), seed * 100 + 30 + i, dev) for i in range(R)]
+    out = torch.empty((B, w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+    lens = lens0.astype(np.int64).copy()
+    bpt = w.kv_bytes_per_token
+
+    def allocate_pages():
+        if not dynamic_alloc:
+            return
+        need, logical, phys = alloc.assign(lens)
+        if len(need):
+            cache.page_table[torch.from_numpy(need).to(dev, non_blocking=True),
+                             torch.from_numpy(logical).to(dev, non_blocking=True)] = \
+                torch.from_numpy(phys).to(dev, non_blocking=True)
+
+    def device_step(i):
+        nonlocal lens
+        allocate_pages()
+        pd.pd_kv_append(ctx, kns[i % R], vns[i % R], cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens)
+        pd.pd_decode_attn(ctx, qs[i % R], cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, out,
+                          sm_scale=w.sm_scale)
+        lens = lens + 1
+        return int(lens.sum()) * bpt  # KV bytes this step's attention must read
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident loop: the headline value
+    for i in range(W):
+        device_step(i)
+    torch.cuda.synchronize()
+    code = pd.pd_device_status(ctx)
+    assert code[0] == 0, f"device fault during warm-up: {code}"
+    befores = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    afters = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    launches0 = pd.pd_launch_count(ctx)
+    barrier()
+    sampler.start()
+    t0.record()
+    kv_bytes = 0
+    for i in range(K):
+        pd.pd_set_profile_events(ctx, befores[i], afters[i])
+        kv_bytes += device_step(W + i)
+    t1.record()
+    barrier()
+    clocks = sampler.stop()
+    pd.pd_set_profile_events(ctx, None, None)
+    launches = pd.pd_launch_count(ctx) - launches0
+    local_ms = t0.elapsed_time(t1)
+    split_ms = float(np.mean([b.elapsed_time(a) for b, a in zip(befores, afters)]))
+    plan = pd.pd_last_plan(ctx)
+    assert pd.pd_device_status(ctx)[0] == 0
+    total_ms, total_bytes = aggregate_over_ranks(local_ms, float(kv_bytes), world, dev)
+    value_gbs = total_bytes / (total_ms * 1e-3) / 1e9
+    bytes_per_step_local = kv_bytes / K
+
+    # ---- host-buffer loop: same step through pd_decode_step_host, copies inside the timed region
+    hq = [t.cpu().pin_memory() for t in qs]
+    hk = [t.cpu().pin_memory() for t in kns]
+    hv = [t.cpu().pin_memory() for t in vns]
+    hout = torch.empty((B, w.num_q_heads, w.head_dim), dtype=torch.bfloat16).pin_memory()
+
+    def host_step(i):
+        nonlocal lens
+        allocate_pages()
+        pd.pd_decode_step_host(ctx, hq[i % R], hk[i % R], hv[i % R], cache.k_pages, cache.v_pages, cache.page_table,
+                               cache.ctx_lens, hout, sm_scale=w.sm_scale)
+        lens = lens + 1
+        return int(lens.sum()) * bpt
+
+    for i in range(W):
+        host_step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    e2e_bytes = 0
+    for i in range(K):
+        e2e_bytes += host_step(W + i)
+    e1.record()
+    barrier()
+    e2e_ms, e2e_total = aggregate_over_ranks(e0.elapsed_time(e1), float(e2e_bytes), world, dev)
+    e2e_gbs = e2e_total / (e2e_ms * 1e-3) / 1e9
+    h2d = (hq[0].numel() + hk[0].numel() + hv[0].numel()) * 2
+    d2h = hout.numel() * 2
+    assert pd.pd_device_status(ctx)[0] == 0
+
+    # ---- CPU baseline: the oracle as it stands, on this machine's host cores (rank 0, N = 1 only)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = time_oracle_once(w, cache, qs[0], lens)
+
+    peak, peak_kind = measured_hbm_peak()
+    achieved = bytes_per_step_local / (split_ms * 1e-3) / 1e9
+    result = {
+        "metric": METRIC, "value": round(value_gbs, 2), "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": round(total_ms / K, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {**workload_config(w, lens, cfg_id),
+                   "l2": f"KV read per step {bytes_per_step_local / 1e9:.2f} GB per GPU >> 126 MB L2; activations rotate over {R} buffers",
+                   "parallelism": "1 GPU" if world == 1 else f"{world} independent replicas, sequences sharded by batch, no collective",
+                   "plan": plan},
+        "pct_of_measured_hbm_peak": round(100 * value_gbs / world / peak, 2),
+        "pct_of_nominal_8tbs": round(100 * value_gbs / world / NOMINAL_HBM_GBS, 2),
+        "seq_steps_per_s": round(B * world * K / (total_ms * 1e-3), 1),
+        "clocks": clocks,
+        "e2e": {"value": round(e2e_gbs, 2), "unit": "GB/s", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "ms_per_step": round(e2e_ms / K, 5),
+                "note": "pd_decode_step_host: q/k_new/v_new from pinned host memory, out back to host, every step; the KV cache is device-resident state"},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "decode_attn_split_kernel", "achieved": round(achieved, 2), "peak": peak,
+                     "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}",
+                     "traffic": None if NCU_TRAFFIC_RATIO is None else int(NCU_TRAFFIC_RATIO * bytes_per_step_local),
+                     "algorithmic_bytes_per_launch": int(bytes_per_step_local), "avg_launch_ms": round(split_ms, 5)},
+        "cpu_baseline": cpu_baseline,
+    }
+    pd.pd_destroy(ctx)
+    if rank == 0:
+        print(json.dumps(result), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.destroy_process_group()
+
+
+def time_oracle_once(w, cache, q, lens, max_seconds_hint: float = 30.0):
+    """Times the oracle on (a prefix of) the batch held in ``cache``; returns the cpu_baseline object."""
+    import torch
+
+    import oracle
+
+    cores = os.cpu_count() or 1
+    B = len(lens)
+    # bounded sample: the oracle handles roughly 1.5e6 (token x query head) per core-second
+    n = B
+    while n > 1 and float(np.sum(lens[:n])) * w.num_q_heads / (1.5e6 * cores) > max_seconds_hint:
+        n //= 2
+    # bring only the pages those sequences own to the host, renumbered (the result does not depend on page ids)
+    P = cache.k_pages.shape[2]
+    table = cache.page_table.detach().cpu().numpy()
+    sub_lens = np.asarray(lens, dtype=np.int32)[:n]
+    rows = [table[b, :(int(lens[b]) + P - 1) // P] for b in range(n)]
+    new_table = np.full((n, table.shape[1]), -1, dtype=np.int32)
+    cur = 0
+    for i, r in enumerate(rows):
+        new_table[i, :len(r)] = np.arange(cur, cur + len(r))
+        cur += len(r)
+    phys = torch.from_numpy(np.concatenate(rows).astype(np.int64)).to(cache.k_pages.device)
+    kp = oracle.bf16_bits(cache.k_pages.index_select(0, phys))
+    vp = oracle.bf16_bits(cache.v_pages.index_select(0, phys))
+    qb = oracle.bf16_bits(q[:n])
+    t = time.perf_counter()
+    oracle.decode_attn(qb, kp, vp, new_table, sub_lens, w.sm_scale, nthreads=cores)
+    dt = time.perf_counter() - t
+    nbytes = float(np.sum(sub_lens)) * w.kv_bytes_per_token
+    return {"value": round(nbytes / dt / 1e9, 4), "unit": "GB/s", "cores": cores, "kind": "oracle",
+            "sample": f"attention of the first {n} of {B} sequences ({int(np.sum(sub_lens))} cached tokens, "
+                      f"{nbytes / 1e9:.3f} GB of KV), one step, {dt:.2f} s wall on {cores} threads",
+            "seconds": round(dt, 3)}
+
+
+# ------------------------------------------------------------------------------------------ reference arm
+
+def run_reference(args):
+    """The CPU oracle timed on the host cores: each step = attention over a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    import workloads as wl
+
+    cfg_id = args.config
+    w = wl.WORKLOADS[cfg_id]
+    K, W = args.steps, args.warmup
+    cores = os.cpu_count() or 1
+    lens_all = wl.context_lengths(cfg_id)
+    # bounded sample: whole run (K + W steps) within about two minutes. The oracle handles
+    # roughly 2e6 (token x query head) per core-second; stay well below that.
+    budget_tokens = 120.0 * 1.5e6 * cores / w.num_q_heads / max(1, K + W)
+    n = 1
+    while n < len(lens_all) and float(np.sum(lens_all[:n + 1])) <= budget_tokens:
+        n += 1
+    lens = lens_all[:n].copy()
+    if float(np.sum(lens)) > budget_tokens:  # a single long sequence: shorten it
+        lens[0] = max(16, int(budget_tokens))
+    cache = wl.build_paged_cache(lens, w.num_kv_heads, w.head_dim, seed=cfg_id, device="cpu")
+    q = oracle.bf16_bits(wl.random_bf16((n, w.num_q_heads, w.head_dim), 100 + cfg_id, "cpu"))
+    kp, vp = oracle.bf16_bits(cache.k_pages), oracle.bf16_bits(cache.v_pages)
+    nbytes = float(np.sum(lens)) * w.kv_bytes_per_token
+
+    def step():
+        oracle.decode_attn(q, kp, vp, cache.page_table_host, lens, w.sm_scale, nthreads=cores)
+
+    for _ in range(W):
+        step()
+    t = time.perf_counter()
+    for _ in range(K):
+        step()
+    dt = time.perf_counter() - t
+    value = nbytes * K / dt / 1e9
+    sample = (f"attention of the first {n} of {len(lens_all)} sequences ({int(np.sum(lens))} cached tokens, "
+              f"{nbytes / 1e9:.4f} GB of KV per step)")
+    result = {
+        "impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": "GB/s",
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": K, "warmup": W,
+        "ms_per_step": round(dt / K * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {**workload_config(w, lens, cfg_id), "sample": sample},
+        "cpu_baseline": {"value": round(value, 4), "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(value, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(result), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4])
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "cuda":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

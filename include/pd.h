@@ -1,0 +1,174 @@
+/*
+ * pd.h - C ABI of the paged decode-attention library (CUDA, sm_100a).
+ *
+ * The library covers the per-sequence term of the paper's decode cost model:
+ * in Eq. 1 a decode iteration costs A + b*B/N, where b is the marginal cost of
+ * one more concurrent sequence and comes mainly from that sequence's KV-cache
+ * HBM reads; Eq. 2 lowers the concurrency to B/(1+theta) while sequences wait
+ * on the environment. The two operations behind that term are exported here:
+ * the attention of one new query token per sequence over its cached context,
+ * and the append of that token's K/V to the cache (Sec. 2.1: every generated
+ * token joins its trajectory's context).
+ *
+ * Data layout (a choice of this library; the paper describes none):
+ *   q, out         [batch][num_q_heads][head_dim]                      bf16
+ *   k_new, v_new   [batch][num_kv_heads][head_dim]                     bf16
+ *   k_pages,
+ *   v_pages        [num_pages][num_kv_heads][page_size][head_dim]      bf16
+ *   page_table     [batch][max_pages_per_seq] int32; entry i is the physical
+ *                  page of tokens [i*page_size, (i+1)*page_size); entries at or
+ *                  past ceil(ctx_lens[b]/page_size) are never read
+ *   ctx_lens       [batch] int32, tokens visible to the query
+ *   lse            [batch][num_q_heads] fp32, natural log of sum exp(scaled logits)
+ * Query head h reads KV head h / (num_q_heads / num_kv_heads).
+ *
+ * Unless a function says otherwise every pointer is a DEVICE pointer to memory
+ * the caller owns, 16-byte aligned, on the device given at pd_create; `stream`
+ * is a cudaStream_t passed as void* (NULL = the default stream). Calls enqueue
+ * work and return without synchronising. Return value: PD_OK or a negative
+ * PD_ERR_* code; nothing throws, aborts or prints. The library owns only the
+ * workspace pd_create allocates.
+ */
+#ifndef PD_H
+#define PD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PD_OK 0
+#define PD_ERR_INVALID_ARG (-1)  /* null/misaligned pointer, size out of the configured range */
+#define PD_ERR_UNSUPPORTED (-2)  /* geometry this build has no kernel for                     */
+#define PD_ERR_CUDA (-3)         /* a CUDA runtime/driver call failed (allocation, launch)    */
+#define PD_ERR_WORKSPACE (-4)    /* request exceeds the workspace sized at pd_create          */
+#define PD_ERR_DEVICE_FAULT (-5) /* a kernel met an out-of-range page id or position          */
+#define PD_ERR_TIMEOUT (-6)      /* a kernel gave up a bounded wait on an asynchronous copy   */
+
+/* pd_config.flags */
+#define PD_FLAG_NONE 0u
+/* pd_kv_append call_flags */
+#define PD_APPEND_NO_ADVANCE 1u /* leave ctx_lens unchanged */
+
+typedef struct pd_ctx pd_ctx; /* opaque */
+
+typedef struct pd_config {
+    int32_t num_q_heads;       /* multiple of num_kv_heads; group size in {1,2,4,8}           */
+    int32_t num_kv_heads;
+    int32_t head_dim;          /* 64 or 128                                                   */
+    int32_t page_size;         /* 16                                                          */
+    int32_t max_batch;         /* 1 .. 4096; sizes the workspace and the host-step staging    */
+    int32_t max_pages_per_seq; /* row length of page_table                                    */
+    int64_t num_pages;         /* pages in each pool                                          */
+    int32_t device;            /* CUDA ordinal                                                */
+    uint32_t flags;
+} pd_config;
+
+/*
+ * Creates a context on cfg->device: checks the geometry, allocates the workspace
+ * for split partials (device) and the staging buffers pd_decode_step_host uses.
+ * *out is NULL on failure. Not thread-safe per context; use one context per
+ * host thread or serialise calls.
+ */
+int pd_create(const pd_config *cfg, pd_ctx **out);
+
+/* Synchronises the device, frees the workspace. NULL is accepted. */
+int pd_destroy(pd_ctx *ctx);
+
+/*
+ * KV append (Sec. 2.1, growth of the context by one token per decode step).
+ * For every b < batch: pos = ctx_lens[b]; the head_dim bf16 values of each KV
+ * head of k_new[b] and v_new[b] are copied, bit for bit, to slot pos % page_size
+ * of page page_table[b][pos / page_size] in k_pages / v_pages; then ctx_lens[b]
+ * becomes pos + 1 (unless PD_APPEND_NO_ADVANCE). A sequence whose position is
+ * past the table or whose page id is outside [0, num_pages) is skipped, its
+ * length is not advanced, and the fault is latched for pd_device_status.
+ * The page for pos must already be in the table (page allocation is the
+ * caller's job).
+ */
+int pd_kv_append(pd_ctx *ctx, const void *k_new, const void *v_new, void *k_pages, void *v_pages,
+                 const int32_t *page_table, int32_t *ctx_lens, int32_t batch, uint32_t call_flags,
+                 void *stream);
+
+/*
+ * Decode attention (the KV-read term b of Eq. 1): for every b < batch and query
+ * head h, out[b][h] = softmax(sm_scale * q[b][h] . K^T) V over the ctx_lens[b]
+ * cached tokens of KV head h / group, and, if lse is not NULL,
+ * lse[b][h] = log sum_t exp(sm_scale * q[b][h] . K_t). ctx_lens[b] == 0 gives
+ * out = 0 and lse = -inf. Slots past ctx_lens[b] and unused pages may hold
+ * anything (NaN included) and do not influence the result.
+ *
+ * The flattened list of (sequence, KV head, page) units is cut into equal
+ * ranges, one per worker warp, so that few long sequences (low decode
+ * concurrency, Eq. 2) still occupy every SM; a range that holds only part of a
+ * (sequence, KV head) context produces an fp32 partial (unnormalised output,
+ * running max, running sum) in the workspace and a second kernel merges the
+ * partials of each row by log-sum-exp. split_pages = 0 picks the range length
+ * from the total page count and the SM count on the device; split_pages > 0
+ * forces that many pages per range (raised silently if the workspace could not
+ * hold the resulting partials). Results are bit-reproducible run to run for a
+ * fixed split_pages and device.
+ *
+ * sm_scale must be finite and positive. q/out rows are head_dim bf16.
+ */
+int pd_decode_attn(pd_ctx *ctx, const void *q, const void *k_pages, const void *v_pages,
+                   const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse,
+                   int32_t batch, float sm_scale, int32_t split_pages, void *stream);
+
+/*
+ * One whole decode step for callers that hold the step's activations on the
+ * HOST: copies q_host, k_new_host, v_new_host (host pointers, pinned or
+ * pageable, same shapes as q/k_new/v_new) to device staging, runs pd_kv_append
+ * (advancing ctx_lens) then pd_decode_attn over the grown contexts, copies the
+ * result to out_host (host, [batch][num_q_heads][head_dim] bf16) and waits for
+ * the stream, so out_host is valid on return. The cache itself (k_pages,
+ * v_pages, page_table, ctx_lens) stays on the device.
+ */
+int pd_decode_step_host(pd_ctx *ctx, const void *q_host, const void *k_new_host, const void *v_new_host,
+                        void *k_pages, void *v_pages, const int32_t *page_table, int32_t *ctx_lens,
+                        void *out_host, int32_t batch, float sm_scale, int32_t split_pages, void *stream);
+
+/*
+ * Waits for `stream`, then reports and clears the first fault a kernel of this
+ * context latched since the last call: *code is PD_OK, PD_ERR_DEVICE_FAULT or
+ * PD_ERR_TIMEOUT; *seq the sequence index (or -1); *detail the offending page
+ * id / position. Any of the three output pointers may be NULL. Returns *code.
+ */
+int pd_device_status(pd_ctx *ctx, void *stream, int32_t *code, int32_t *seq, int32_t *detail);
+
+/*
+ * Timing hook for benchmarks: after this call every pd_decode_attn of this
+ * context records `before` on its stream just ahead of the split kernel and
+ * `after` right behind it (both cudaEvent_t passed as void*, owned by the
+ * caller, who must keep them alive until the work has run). Passing two NULLs
+ * switches the hook off. The events bracket the split kernel only, not the merge.
+ */
+int pd_set_profile_events(pd_ctx *ctx, void *before, void *after);
+
+/* Bytes of device workspace the context holds. */
+int pd_workspace_bytes(const pd_ctx *ctx, size_t *bytes);
+
+/* Number of kernels this context has launched since pd_create. */
+int pd_launch_count(const pd_ctx *ctx, int64_t *launches);
+
+/*
+ * Plan of the most recent pd_decode_attn call, read back from the device after
+ * waiting for `stream`: total (sequence, KV head, page) units, pages per range,
+ * number of ranges, number of worker warps launched. For tests and reporting.
+ */
+int pd_last_plan(pd_ctx *ctx, void *stream, int64_t *total_units, int32_t *pages_per_range,
+                 int32_t *num_ranges, int32_t *num_workers);
+
+const char *pd_status_string(int status);
+
+/* Text of the most recent failure recorded by this context (CUDA error string
+ * included where one exists); owned by the context, valid until the next call. */
+const char *pd_last_error(const pd_ctx *ctx);
+int pd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PD_H */

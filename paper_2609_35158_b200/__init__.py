@@ -1,0 +1,183 @@
+"""Python binding of ``libpd.so``: paged GQA decode attention + KV append on B200.
+
+Argument marshalling only. Every function has the name and the argument order
+of its C counterpart in ``include/pd.h``; tensors are torch tensors whose
+``data_ptr()`` is handed to the library, streams default to torch's current
+stream. Nothing here computes: if the CUDA library cannot be loaded the import
+fails, there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+PD_OK = 0
+PD_ERR_INVALID_ARG = -1
+PD_ERR_UNSUPPORTED = -2
+PD_ERR_CUDA = -3
+PD_ERR_WORKSPACE = -4
+PD_ERR_DEVICE_FAULT = -5
+PD_ERR_TIMEOUT = -6
+PD_APPEND_NO_ADVANCE = 1
+
+# every symbol include/pd.h declares
+EXPORTS = (
+    "pd_create", "pd_destroy", "pd_kv_append", "pd_decode_attn", "pd_decode_step_host", "pd_device_status",
+    "pd_set_profile_events", "pd_workspace_bytes", "pd_launch_count", "pd_last_plan", "pd_status_string", "pd_last_error", "pd_version",
+)
+
+
+class pd_config(ctypes.Structure):
+    _fields_ = [
+        ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+        ("page_size", ctypes.c_int32), ("max_batch", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32),
+        ("num_pages", ctypes.c_int64), ("device", ctypes.c_int32), ("flags", ctypes.c_uint32),
+    ]
+
+
+class PdError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        self.code = code
+        msg = f"{where}: {pd_status_string(code)} ({code})"
+        super().__init__(msg + (f" - {detail}" if detail else ""))
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path):
+        raise ImportError(
+            f"{path} is missing: build it with `python -m paper_2609_35158_b200.build` "
+            "(nvcc, sm_100a). This package has no fallback path.")
+    lib = ctypes.CDLL(path)
+    vp, i32, u32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_int64, ctypes.c_float
+    lib.pd_create.argtypes = [ctypes.POINTER(pd_config), ctypes.POINTER(vp)]
+    lib.pd_destroy.argtypes = [vp]
+    lib.pd_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, u32, vp]
+    lib.pd_decode_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, vp]
+    lib.pd_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, vp]
+    lib.pd_device_status.argtypes = [vp, vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    lib.pd_set_profile_events.argtypes = [vp, vp, vp]
+    lib.pd_workspace_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
+    lib.pd_launch_count.argtypes = [vp, ctypes.POINTER(i64)]
+    lib.pd_last_plan.argtypes = [vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                 ctypes.POINTER(i32)]
+    lib.pd_status_string.argtypes = [ctypes.c_int]
+    lib.pd_status_string.restype = ctypes.c_char_p
+    lib.pd_last_error.argtypes = [vp]
+    lib.pd_last_error.restype = ctypes.c_char_p
+    lib.pd_version.argtypes = []
+    for name in EXPORTS:
+        if name not in ("pd_status_string", "pd_last_error"):
+            getattr(lib, name).restype = ctypes.c_int
+    return lib
+
+
+_lib = _load()
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _check(rc: int, where: str, ctx=None):
+    if rc != PD_OK:
+        raise PdError(rc, where, pd_last_error(ctx) if ctx else "")
+
+
+def pd_version() -> int:
+    return _lib.pd_version()
+
+
+def pd_status_string(code: int) -> str:
+    return _lib.pd_status_string(code).decode()
+
+
+def pd_last_error(ctx) -> str:
+    return _lib.pd_last_error(ctx).decode()
+
+
+def pd_create(num_q_heads, num_kv_heads, head_dim, page_size, max_batch, max_pages_per_seq, num_pages,
+              device=0, flags=0):
+    """Returns an opaque context handle (ctypes void pointer)."""
+    cfg = pd_config(num_q_heads, num_kv_heads, head_dim, page_size, max_batch, max_pages_per_seq, num_pages,
+                    device, flags)
+    ctx = ctypes.c_void_p()
+    _check(_lib.pd_create(ctypes.byref(cfg), ctypes.byref(ctx)), "pd_create")
+    return ctx
+
+
+def pd_destroy(ctx) -> None:
+    _lib.pd_destroy(ctx)
+
+
+def pd_kv_append(ctx, k_new, v_new, k_pages, v_pages, page_table, ctx_lens, batch=None, call_flags=0, stream=None):
+    batch = k_new.shape[0] if batch is None else batch
+    _check(_lib.pd_kv_append(ctx, _ptr(k_new), _ptr(v_new), _ptr(k_pages), _ptr(v_pages), _ptr(page_table),
+                             _ptr(ctx_lens), batch, call_flags, _stream(stream)), "pd_kv_append", ctx)
+
+
+def pd_decode_attn(ctx, q, k_pages, v_pages, page_table, ctx_lens, out, lse=None, batch=None, sm_scale=1.0,
+                   split_pages=0, stream=None):
+    batch = q.shape[0] if batch is None else batch
+    _check(_lib.pd_decode_attn(ctx, _ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(page_table), _ptr(ctx_lens),
+                               _ptr(out), _ptr(lse), batch, sm_scale, split_pages, _stream(stream)),
+           "pd_decode_attn", ctx)
+
+
+def pd_decode_step_host(ctx, q_host, k_new_host, v_new_host, k_pages, v_pages, page_table, ctx_lens, out_host,
+                        batch=None, sm_scale=1.0, split_pages=0, stream=None):
+    """q_host, k_new_host, v_new_host, out_host are CPU tensors (pinned for full copy speed)."""
+    for t in (q_host, k_new_host, v_new_host, out_host):
+        assert not t.is_cuda and t.is_contiguous()
+    batch = q_host.shape[0] if batch is None else batch
+    _check(_lib.pd_decode_step_host(ctx, _ptr(q_host), _ptr(k_new_host), _ptr(v_new_host), _ptr(k_pages),
+                                    _ptr(v_pages), _ptr(page_table), _ptr(ctx_lens), _ptr(out_host), batch,
+                                    sm_scale, split_pages, _stream(stream)), "pd_decode_step_host", ctx)
+
+
+def pd_device_status(ctx, stream=None):
+    """(code, seq, detail) of the first latched device fault; clears it."""
+    code, seq, detail = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    _lib.pd_device_status(ctx, _stream(stream), ctypes.byref(code), ctypes.byref(seq), ctypes.byref(detail))
+    return code.value, seq.value, detail.value
+
+
+def pd_set_profile_events(ctx, before=None, after=None) -> None:
+    """``before`` / ``after``: ``torch.cuda.Event(enable_timing=True)`` objects (or None, None)."""
+    def handle(ev):
+        if ev is None:
+            return None
+        if ev.cuda_event == 0:  # torch creates the CUDA event lazily, on first record
+            ev.record()
+        return ev.cuda_event
+    _check(_lib.pd_set_profile_events(ctx, handle(before), handle(after)), "pd_set_profile_events", ctx)
+
+
+def pd_workspace_bytes(ctx) -> int:
+    n = ctypes.c_size_t()
+    _check(_lib.pd_workspace_bytes(ctx, ctypes.byref(n)), "pd_workspace_bytes", ctx)
+    return n.value
+
+
+def pd_launch_count(ctx) -> int:
+    n = ctypes.c_int64()
+    _check(_lib.pd_launch_count(ctx, ctypes.byref(n)), "pd_launch_count", ctx)
+    return n.value
+
+
+def pd_last_plan(ctx, stream=None) -> dict:
+    total, per, ranges, workers = ctypes.c_int64(), ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    _check(_lib.pd_last_plan(ctx, _stream(stream), ctypes.byref(total), ctypes.byref(per), ctypes.byref(ranges),
+                             ctypes.byref(workers)), "pd_last_plan", ctx)
+    return {"total_units": total.value, "pages_per_range": per.value, "num_ranges": ranges.value,
+            "num_workers": workers.value}

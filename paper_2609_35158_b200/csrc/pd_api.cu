@@ -1,0 +1,390 @@
+// C ABI of the paged decode-attention library: context, argument checks,
+// tensor-map encoding and kernel launches. See include/pd.h for the contract.
+#include "../../include/pd.h"
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "pd_kernels.cuh"
+
+namespace {
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+struct pd_ctx {
+    pd_config cfg{};
+    int group = 0;
+    int num_sms = 0;
+    int num_ctas = 0;
+    pd::AttnVariant variant{};
+    size_t smem_bytes = 0;
+    int max_ranges = 0;
+    int min_pages_auto = 1;
+    size_t slots = 0;
+    // device workspace (one allocation)
+    void *workspace = nullptr;
+    size_t workspace_bytes = 0;
+    float *part_o = nullptr;
+    float2 *part_ml = nullptr;
+    int32_t *cum_pages = nullptr;
+    int32_t *plan = nullptr;
+    int32_t *status = nullptr;
+    // staging for pd_decode_step_host
+    __nv_bfloat16 *stage_q = nullptr, *stage_k = nullptr, *stage_v = nullptr, *stage_out = nullptr;
+    // tensor maps, cached per pool pointer
+    EncodeTiledFn encode = nullptr;
+    const void *map_k_ptr = nullptr, *map_v_ptr = nullptr;
+    alignas(64) CUtensorMap tm_k{};
+    alignas(64) CUtensorMap tm_v{};
+    cudaEvent_t ev_before = nullptr, ev_after = nullptr;  // optional timing hook around the split kernel
+    int64_t launches = 0;
+    char last_error[256] = {0};
+};
+
+namespace {
+
+int fail(pd_ctx *ctx, int code, const char *what, cudaError_t err = cudaSuccess) {
+    if (ctx != nullptr) {
+        if (err != cudaSuccess) std::snprintf(ctx->last_error, sizeof ctx->last_error, "%s: %s", what, cudaGetErrorString(err));
+        else std::snprintf(ctx->last_error, sizeof ctx->last_error, "%s", what);
+    }
+    return code;
+}
+
+bool aligned16(const void *p) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int env_int(const char *name, int fallback) {
+    const char *v = std::getenv(name);
+    return (v != nullptr && *v != '\0') ? std::atoi(v) : fallback;
+}
+
+// 2-D view of a pool: rows = (page, KV head, slot), columns = head_dim bf16.
+// Box = 16 rows x 64 columns (128 B) with the 128-byte swizzle.
+int encode_pool_map(pd_ctx *ctx, const void *pool, CUtensorMap *out) {
+    const pd_config &c = ctx->cfg;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c.head_dim),
+                                static_cast<cuuint64_t>(c.num_pages) * c.num_kv_heads * c.page_size};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c.head_dim) * 2};
+    const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(c.page_size)};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    const CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box,
+                                   elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        std::snprintf(ctx->last_error, sizeof ctx->last_error, "cuTensorMapEncodeTiled failed (%d)", static_cast<int>(r));
+        return PD_ERR_CUDA;
+    }
+    return PD_OK;
+}
+
+int check_batch(pd_ctx *ctx, int32_t batch) {
+    if (ctx == nullptr) return PD_ERR_INVALID_ARG;
+    if (batch < 0 || batch > ctx->cfg.max_batch) return fail(ctx, PD_ERR_INVALID_ARG, "batch outside [0, max_batch]");
+    return PD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int pd_version(void) { return 100; }
+
+const char *pd_status_string(int status) {
+    switch (status) {
+        case PD_OK: return "ok";
+        case PD_ERR_INVALID_ARG: return "invalid argument";
+        case PD_ERR_UNSUPPORTED: return "unsupported geometry";
+        case PD_ERR_CUDA: return "CUDA call failed";
+        case PD_ERR_WORKSPACE: return "workspace too small";
+        case PD_ERR_DEVICE_FAULT: return "kernel met an out-of-range page id or length";
+        case PD_ERR_TIMEOUT: return "kernel gave up a bounded wait";
+        default: return "unknown status";
+    }
+}
+
+const char *pd_last_error(const pd_ctx *ctx) { return ctx != nullptr ? ctx->last_error : "null context"; }
+
+int pd_create(const pd_config *cfg, pd_ctx **out) {
+    if (out == nullptr) return PD_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg == nullptr) return PD_ERR_INVALID_ARG;
+    if (cfg->num_q_heads <= 0 || cfg->num_kv_heads <= 0 || cfg->num_q_heads % cfg->num_kv_heads != 0 ||
+        cfg->max_batch < 1 || cfg->max_batch > pd::kMaxBatch || cfg->max_pages_per_seq < 1 || cfg->num_pages < 1 ||
+        cfg->device < 0)
+        return PD_ERR_INVALID_ARG;
+    const int group = cfg->num_q_heads / cfg->num_kv_heads;
+    if (cfg->page_size != pd::kPageSize || (cfg->head_dim != 64 && cfg->head_dim != 128) ||
+        (group != 1 && group != 2 && group != 4 && group != 8))
+        return PD_ERR_UNSUPPORTED;
+    // TMA row coordinates and page ids are 32-bit
+    if (cfg->num_pages * cfg->num_kv_heads * cfg->page_size >= (int64_t(1) << 31)) return PD_ERR_UNSUPPORTED;
+    if (static_cast<int64_t>(cfg->max_pages_per_seq) * cfg->page_size >= (int64_t(1) << 31)) return PD_ERR_UNSUPPORTED;
+
+    DeviceGuard guard(cfg->device);
+    if (!guard.ok) return PD_ERR_CUDA;
+    cudaDeviceProp prop{};
+    if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return PD_ERR_CUDA;
+    if (prop.major != 10) return PD_ERR_UNSUPPORTED;  // built for sm_100a only
+
+    pd_ctx *ctx = new (std::nothrow) pd_ctx();
+    if (ctx == nullptr) return PD_ERR_CUDA;
+    ctx->cfg = *cfg;
+    ctx->group = group;
+    ctx->num_sms = prop.multiProcessorCount;
+
+    // kernel shape: one CTA per SM, each warp an independent worker with its own stage ring
+    pd::AttnVariant v{};
+    v.head_dim = cfg->head_dim;
+    v.warps = env_int("PD_TUNE_WARPS", 8);
+    v.stages = env_int("PD_TUNE_STAGES", cfg->head_dim == 128 ? 3 : 6);
+    v.hilo = env_int("PD_TUNE_HILO", 1);
+    ctx->variant = v;
+    ctx->num_ctas = ctx->num_sms * env_int("PD_TUNE_CTAS_PER_SM", 1);
+    ctx->min_pages_auto = env_int("PD_TUNE_MIN_PAGES", 4);
+    cudaError_t err = pd::prepare_decode_attn(v, &ctx->smem_bytes);
+    if (err != cudaSuccess) {
+        delete ctx;
+        return err == cudaErrorInvalidValue ? PD_ERR_UNSUPPORTED : PD_ERR_CUDA;
+    }
+
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult q{};
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || fn == nullptr ||
+        q != cudaDriverEntryPointSuccess) {
+        delete ctx;
+        return PD_ERR_CUDA;
+    }
+    ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+
+    // workspace: partial slots = ranges + one per (sequence, KV head)
+    const int n_workers = ctx->num_ctas * v.warps;
+    ctx->max_ranges = 4 * n_workers;
+    ctx->slots = static_cast<size_t>(ctx->max_ranges) + static_cast<size_t>(cfg->max_batch) * cfg->num_kv_heads;
+    auto round256 = [](size_t n) { return (n + 255) & ~size_t(255); };
+    const size_t b_part_o = round256(ctx->slots * group * cfg->head_dim * sizeof(float));
+    const size_t b_part_ml = round256(ctx->slots * group * sizeof(float2));
+    const size_t b_cum = round256((static_cast<size_t>(cfg->max_batch) + 1) * sizeof(int32_t));
+    const size_t b_plan = round256(pd::kPlanWords * sizeof(int32_t));
+    const size_t b_status = round256(pd::kStatusWords * sizeof(int32_t));
+    const size_t b_q = round256(static_cast<size_t>(cfg->max_batch) * cfg->num_q_heads * cfg->head_dim * 2);
+    const size_t b_kv = round256(static_cast<size_t>(cfg->max_batch) * cfg->num_kv_heads * cfg->head_dim * 2);
+    ctx->workspace_bytes = b_part_o + b_part_ml + b_cum + b_plan + b_status + 2 * b_q + 2 * b_kv;
+    err = cudaMalloc(&ctx->workspace, ctx->workspace_bytes);
+    if (err != cudaSuccess) {
+        delete ctx;
+        return PD_ERR_CUDA;
+    }
+    char *w = static_cast<char *>(ctx->workspace);
+    ctx->part_o = reinterpret_cast<float *>(w); w += b_part_o;
+    ctx->part_ml = reinterpret_cast<float2 *>(w); w += b_part_ml;
+    ctx->cum_pages = reinterpret_cast<int32_t *>(w); w += b_cum;
+    ctx->plan = reinterpret_cast<int32_t *>(w); w += b_plan;
+    ctx->status = reinterpret_cast<int32_t *>(w); w += b_status;
+    ctx->stage_q = reinterpret_cast<__nv_bfloat16 *>(w); w += b_q;
+    ctx->stage_out = reinterpret_cast<__nv_bfloat16 *>(w); w += b_q;
+    ctx->stage_k = reinterpret_cast<__nv_bfloat16 *>(w); w += b_kv;
+    ctx->stage_v = reinterpret_cast<__nv_bfloat16 *>(w); w += b_kv;
+    err = cudaMemset(ctx->workspace, 0, ctx->workspace_bytes);
+    if (err != cudaSuccess) {
+        cudaFree(ctx->workspace);
+        delete ctx;
+        return PD_ERR_CUDA;
+    }
+    *out = ctx;
+    return PD_OK;
+}
+
+int pd_destroy(pd_ctx *ctx) {
+    if (ctx == nullptr) return PD_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    cudaDeviceSynchronize();
+    cudaFree(ctx->workspace);
+    delete ctx;
+    return PD_OK;
+}
+
+int pd_kv_append(pd_ctx *ctx, const void *k_new, const void *v_new, void *k_pages, void *v_pages,
+                 const int32_t *page_table, int32_t *ctx_lens, int32_t batch, uint32_t call_flags, void *stream) {
+    if (int rc = check_batch(ctx, batch)) return rc;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_pages) || !aligned16(v_pages) || page_table == nullptr ||
+        ctx_lens == nullptr)
+        return fail(ctx, PD_ERR_INVALID_ARG, "pd_kv_append: null or misaligned pointer");
+    if (call_flags & ~PD_APPEND_NO_ADVANCE) return fail(ctx, PD_ERR_INVALID_ARG, "pd_kv_append: unknown call flag");
+    if (batch == 0) return PD_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
+    pd::AppendParams p{};
+    p.k_new = static_cast<const __nv_bfloat16 *>(k_new);
+    p.v_new = static_cast<const __nv_bfloat16 *>(v_new);
+    p.k_pages = static_cast<__nv_bfloat16 *>(k_pages);
+    p.v_pages = static_cast<__nv_bfloat16 *>(v_pages);
+    p.page_table = page_table;
+    p.ctx_lens = ctx_lens;
+    p.status = ctx->status;
+    p.B = batch;
+    p.Hkv = ctx->cfg.num_kv_heads;
+    p.D = ctx->cfg.head_dim;
+    p.MP = ctx->cfg.max_pages_per_seq;
+    p.num_pages = static_cast<int32_t>(ctx->cfg.num_pages);
+    p.advance = (call_flags & PD_APPEND_NO_ADVANCE) ? 0 : 1;
+    const cudaError_t err = pd::launch_kv_append(p, static_cast<cudaStream_t>(stream));
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "kv_append launch", err);
+    ctx->launches += 1;
+    return PD_OK;
+}
+
+int pd_decode_attn(pd_ctx *ctx, const void *q, const void *k_pages, const void *v_pages, const int32_t *page_table,
+                   const int32_t *ctx_lens, void *out, float *lse, int32_t batch, float sm_scale, int32_t split_pages,
+                   void *stream) {
+    if (int rc = check_batch(ctx, batch)) return rc;
+    if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(out) || page_table == nullptr ||
+        ctx_lens == nullptr)
+        return fail(ctx, PD_ERR_INVALID_ARG, "pd_decode_attn: null or misaligned pointer");
+    if (!(sm_scale > 0.f) || !(sm_scale < 3.0e38f)) return fail(ctx, PD_ERR_INVALID_ARG, "sm_scale must be finite and positive");
+    if (split_pages < 0) return fail(ctx, PD_ERR_INVALID_ARG, "split_pages must be >= 0");
+    if (batch == 0) return PD_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
+    if (ctx->map_k_ptr != k_pages) {
+        if (int rc = encode_pool_map(ctx, k_pages, &ctx->tm_k)) return rc;
+        ctx->map_k_ptr = k_pages;
+    }
+    if (ctx->map_v_ptr != v_pages) {
+        if (int rc = encode_pool_map(ctx, v_pages, &ctx->tm_v)) return rc;
+        ctx->map_v_ptr = v_pages;
+    }
+    pd::AttnParams p{};
+    p.q = static_cast<const __nv_bfloat16 *>(q);
+    p.page_table = page_table;
+    p.ctx_lens = ctx_lens;
+    p.out = static_cast<__nv_bfloat16 *>(out);
+    p.lse = lse;
+    p.part_o = ctx->part_o;
+    p.part_ml = ctx->part_ml;
+    p.cum_pages = ctx->cum_pages;
+    p.plan = ctx->plan;
+    p.status = ctx->status;
+    p.B = batch;
+    p.Hq = ctx->cfg.num_q_heads;
+    p.Hkv = ctx->cfg.num_kv_heads;
+    p.G = ctx->group;
+    p.MP = ctx->cfg.max_pages_per_seq;
+    p.num_pages = static_cast<int32_t>(ctx->cfg.num_pages);
+    p.scale_log2 = sm_scale * 1.4426950408889634f;
+    p.split_pages = split_pages;
+    p.max_ranges = ctx->max_ranges;
+    p.min_pages_auto = ctx->min_pages_auto;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (ctx->ev_before != nullptr) cudaEventRecord(ctx->ev_before, s);
+    cudaError_t err = pd::launch_decode_attn(ctx->variant, ctx->tm_k, ctx->tm_v, p, ctx->num_ctas, ctx->smem_bytes, s);
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "decode_attn_split launch", err);
+    if (ctx->ev_after != nullptr) cudaEventRecord(ctx->ev_after, s);
+    err = pd::launch_lse_merge(ctx->cfg.head_dim, p, s);
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "lse_merge launch", err);
+    ctx->launches += 2;
+    return PD_OK;
+}
+
+int pd_decode_step_host(pd_ctx *ctx, const void *q_host, const void *k_new_host, const void *v_new_host, void *k_pages,
+                        void *v_pages, const int32_t *page_table, int32_t *ctx_lens, void *out_host, int32_t batch,
+                        float sm_scale, int32_t split_pages, void *stream) {
+    if (int rc = check_batch(ctx, batch)) return rc;
+    if (q_host == nullptr || k_new_host == nullptr || v_new_host == nullptr || out_host == nullptr)
+        return fail(ctx, PD_ERR_INVALID_ARG, "pd_decode_step_host: null host pointer");
+    if (batch == 0) return PD_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t nq = static_cast<size_t>(batch) * ctx->cfg.num_q_heads * ctx->cfg.head_dim * 2;
+    const size_t nkv = static_cast<size_t>(batch) * ctx->cfg.num_kv_heads * ctx->cfg.head_dim * 2;
+    cudaError_t err = cudaMemcpyAsync(ctx->stage_q, q_host, nq, cudaMemcpyHostToDevice, s);
+    if (err == cudaSuccess) err = cudaMemcpyAsync(ctx->stage_k, k_new_host, nkv, cudaMemcpyHostToDevice, s);
+    if (err == cudaSuccess) err = cudaMemcpyAsync(ctx->stage_v, v_new_host, nkv, cudaMemcpyHostToDevice, s);
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "host-to-device copy", err);
+    if (int rc = pd_kv_append(ctx, ctx->stage_k, ctx->stage_v, k_pages, v_pages, page_table, ctx_lens, batch, 0, stream))
+        return rc;
+    if (int rc = pd_decode_attn(ctx, ctx->stage_q, k_pages, v_pages, page_table, ctx_lens, ctx->stage_out, nullptr, batch,
+                                sm_scale, split_pages, stream))
+        return rc;
+    err = cudaMemcpyAsync(out_host, ctx->stage_out, nq, cudaMemcpyDeviceToHost, s);
+    if (err == cudaSuccess) err = cudaStreamSynchronize(s);
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "device-to-host copy", err);
+    return PD_OK;
+}
+
+int pd_device_status(pd_ctx *ctx, void *stream, int32_t *code, int32_t *seq, int32_t *detail) {
+    if (ctx == nullptr) return PD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t host[pd::kStatusWords] = {0, 0, 0, 0};
+    cudaError_t err = cudaMemcpyAsync(host, ctx->status, sizeof host, cudaMemcpyDeviceToHost, s);
+    if (err == cudaSuccess) err = cudaMemsetAsync(ctx->status, 0, sizeof host, s);
+    if (err == cudaSuccess) err = cudaStreamSynchronize(s);
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "status read", err);
+    int rc = PD_OK;
+    if (host[0] == pd::kDevBadPage || host[0] == pd::kDevBadLength) rc = PD_ERR_DEVICE_FAULT;
+    else if (host[0] == pd::kDevTimeout) rc = PD_ERR_TIMEOUT;
+    if (code != nullptr) *code = rc;
+    if (seq != nullptr) *seq = rc == PD_OK ? -1 : host[1];
+    if (detail != nullptr) *detail = rc == PD_OK ? 0 : host[2];
+    return rc;
+}
+
+int pd_set_profile_events(pd_ctx *ctx, void *before, void *after) {
+    if (ctx == nullptr || ((before == nullptr) != (after == nullptr))) return PD_ERR_INVALID_ARG;
+    ctx->ev_before = static_cast<cudaEvent_t>(before);
+    ctx->ev_after = static_cast<cudaEvent_t>(after);
+    return PD_OK;
+}
+
+int pd_workspace_bytes(const pd_ctx *ctx, size_t *bytes) {
+    if (ctx == nullptr || bytes == nullptr) return PD_ERR_INVALID_ARG;
+    *bytes = ctx->workspace_bytes;
+    return PD_OK;
+}
+
+int pd_launch_count(const pd_ctx *ctx, int64_t *launches) {
+    if (ctx == nullptr || launches == nullptr) return PD_ERR_INVALID_ARG;
+    *launches = ctx->launches;
+    return PD_OK;
+}
+
+int pd_last_plan(pd_ctx *ctx, void *stream, int64_t *total_units, int32_t *pages_per_range, int32_t *num_ranges,
+                 int32_t *num_workers) {
+    if (ctx == nullptr) return PD_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t host[pd::kPlanWords] = {0};
+    cudaError_t err = cudaMemcpyAsync(host, ctx->plan, sizeof host, cudaMemcpyDeviceToHost, s);
+    if (err == cudaSuccess) err = cudaStreamSynchronize(s);
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "plan read", err);
+    if (total_units != nullptr)
+        *total_units = (static_cast<int64_t>(host[1]) << 32) | static_cast<uint32_t>(host[0]);
+    if (pages_per_range != nullptr) *pages_per_range = host[2];
+    if (num_ranges != nullptr) *num_ranges = host[3];
+    if (num_workers != nullptr) *num_workers = host[4];
+    return PD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,63 @@
+// Parameter blocks and host-side launchers shared by the kernels and the C ABI.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace pd {
+
+constexpr int kPageSize = 16;       // tokens per page
+constexpr int kMaxBatch = 4096;     // prefix sums of page counts live in shared memory
+constexpr int kPlanWords = 8;       // plan[0..1] total units (lo, hi), [2] pages per range, [3] ranges, [4] workers
+constexpr int kStatusWords = 4;     // status[0] code, [1] sequence, [2] detail
+
+// Device-side fault codes latched in status[0] (first one wins).
+constexpr int kDevOk = 0;
+constexpr int kDevBadPage = 1;      // page id outside [0, num_pages)
+constexpr int kDevBadLength = 2;    // ctx_len negative or past the page table
+constexpr int kDevTimeout = 3;      // bounded wait on an asynchronous copy ran out
+
+struct AttnParams {
+    const __nv_bfloat16 *q;     // [B][Hq][D]
+    const int32_t *page_table;  // [B][MP]
+    const int32_t *ctx_lens;    // [B]
+    __nv_bfloat16 *out;         // [B][Hq][D]
+    float *lse;                 // [B][Hq] or null
+    float *part_o;              // [slots][G][D] unnormalised partial outputs
+    float2 *part_ml;            // [slots][G]    (running max in log2 units, running sum)
+    int32_t *cum_pages;         // [B+1] exclusive prefix sum of pages per sequence (written by CTA 0)
+    int32_t *plan;              // [kPlanWords]
+    int32_t *status;            // [kStatusWords]
+    int32_t B, Hq, Hkv, G, MP;
+    int32_t num_pages;
+    float scale_log2;           // sm_scale * log2(e)
+    int32_t split_pages;        // 0 = automatic
+    int32_t max_ranges;         // partial slots available beyond one per (sequence, KV head)
+    int32_t min_pages_auto;     // lower bound on pages per range in automatic mode
+};
+
+struct AppendParams {
+    const __nv_bfloat16 *k_new, *v_new;  // [B][Hkv][D]
+    __nv_bfloat16 *k_pages, *v_pages;    // [NP][Hkv][16][D]
+    const int32_t *page_table;
+    int32_t *ctx_lens;
+    int32_t *status;
+    int32_t B, Hkv, D, MP;
+    int32_t num_pages;
+    int32_t advance;
+};
+
+// Shape of one compiled variant of the split kernel.
+struct AttnVariant {
+    int head_dim, warps, stages, hilo;
+};
+
+// Launchers (defined next to their kernels). They return the CUDA error of the launch.
+cudaError_t launch_kv_append(const AppendParams &p, cudaStream_t stream);
+cudaError_t prepare_decode_attn(const AttnVariant &v, size_t *smem_bytes);  // opt-in shared memory, once
+cudaError_t launch_decode_attn(const AttnVariant &v, const CUtensorMap &tm_k, const CUtensorMap &tm_v,
+                               const AttnParams &p, int num_ctas, size_t smem_bytes, cudaStream_t stream);
+cudaError_t launch_lse_merge(int head_dim, const AttnParams &p, cudaStream_t stream);
+
+}  // namespace pd

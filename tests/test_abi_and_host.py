@@ -1,0 +1,115 @@
+"""CPU-side checks: the C-ABI library builds, loads and exports what include/pd.h declares;
+host-side logic of the benchmark's multi-rank aggregation runs under gloo with two ranks."""
+import ctypes
+import os
+import re
+import subprocess
+import sys
+
+import numpy as np
+import pytest
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def header_functions():
+    text = open(os.path.join(ROOT, "include", "pd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(pd_[a-z_]+)\s*\(", text)))
+
+
+def test_library_builds_and_exports_every_declared_symbol():
+    from paper_2609_35158_b200 import build as pd_build
+
+    lib_path = pd_build.build_library()
+    lib = ctypes.CDLL(lib_path)
+    declared = header_functions()
+    assert {"pd_create", "pd_destroy", "pd_kv_append", "pd_decode_attn", "pd_decode_step_host"} <= set(declared)
+    for name in declared:
+        assert hasattr(lib, name), f"{name} declared in pd.h but not exported"
+    import paper_2609_35158_b200 as pd
+
+    assert sorted(pd.EXPORTS) == declared
+    for name in declared:
+        assert callable(getattr(pd, name)), f"binding lacks {name}"
+    assert pd.pd_version() >= 100
+    assert pd.pd_status_string(pd.PD_ERR_UNSUPPORTED) == "unsupported geometry"
+
+
+def test_create_rejects_bad_geometry_before_touching_the_device():
+    import paper_2609_35158_b200 as pd
+
+    for args, code in (((8, 3, 64, 16, 4, 4, 16), pd.PD_ERR_INVALID_ARG),
+                       ((8, 2, 96, 16, 4, 4, 16), pd.PD_ERR_UNSUPPORTED),
+                       ((8, 2, 64, 8, 4, 4, 16), pd.PD_ERR_UNSUPPORTED),
+                       ((32, 2, 64, 16, 4, 4, 16), pd.PD_ERR_UNSUPPORTED),
+                       ((8, 2, 64, 16, 0, 4, 16), pd.PD_ERR_INVALID_ARG),
+                       ((8, 2, 64, 16, 5000, 4, 16), pd.PD_ERR_INVALID_ARG),
+                       ((8, 2, 64, 16, 4, 4, 1 << 40), pd.PD_ERR_UNSUPPORTED)):
+        with pytest.raises(pd.PdError) as e:
+            pd.pd_create(*args)
+        assert e.value.code == code
+    if not torch.cuda.is_available():  # no device: a clean error code, not a crash
+        with pytest.raises(pd.PdError) as e:
+            pd.pd_create(8, 2, 64, 16, 4, 4, 16)
+        assert e.value.code == pd.PD_ERR_CUDA
+
+
+def test_product_path_does_not_import_the_oracle():
+    for rel in ("paper_2609_35158_b200/__init__.py", "paper_2609_35158_b200/build.py"):
+        src = open(os.path.join(ROOT, rel)).read()
+        assert "oracle" not in src
+    for f in os.listdir(os.path.join(ROOT, "paper_2609_35158_b200", "csrc")):
+        assert "oracle" not in open(os.path.join(ROOT, "paper_2609_35158_b200", "csrc", f)).read()
+    assert "paper_2609_35158_b200" not in open(os.path.join(ROOT, "oracle", "__init__.py")).read()
+
+
+WORKER = r"""
+import os, sys
+sys.path.insert(0, {root!r})
+import numpy as np, torch, torch.distributed as dist
+import bench, workloads as wl
+rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+dist.init_process_group("gloo", init_method="tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+lens = wl.context_lengths(1)
+mine = wl.shard_sequences(lens, world)[rank]
+local_tokens = float(lens[mine].sum())
+ms, tokens = bench.aggregate_over_ranks(10.0 + 5.0 * rank, local_tokens, world)
+assert ms == 15.0, ms                      # max over ranks
+assert tokens == float(lens.sum()), tokens # every sequence on exactly one rank
+gathered = [None] * world
+dist.all_gather_object(gathered, mine.tolist())
+assert sorted(sum(gathered, [])) == list(range(len(lens)))
+dist.destroy_process_group()
+print("rank", rank, "ok")
+"""
+
+
+def test_two_rank_sharding_and_aggregation_under_gloo(tmp_path):
+    import socket
+
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    script = tmp_path / "worker.py"
+    script.write_text(WORKER.format(root=ROOT, port=port))
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, str(script)], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.STDOUT, text=True))
+    for p in procs:
+        out, _ = p.communicate(timeout=180)
+        assert p.returncode == 0, out
+
+
+def test_error_metric_helper():
+    from pd_testlib import error_metrics
+
+    ref = np.zeros((2, 3, 4)); ref[..., 0] = 1.0
+    got = torch.tensor(ref, dtype=torch.bfloat16)
+    assert error_metrics(got, ref) == (0.0, 0.0)
+    got[0, 0, 1] = 0.5
+    m, r = error_metrics(got, ref)
+    assert m == 0.5 and abs(r - 0.5) < 1e-12
