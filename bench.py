@@ -29,9 +29,10 @@ import numpy as np  # noqa: E402
 METRIC = "decode-attn achieved HBM GB/s (% of B200 peak) and seq-steps/s per layer"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per launch of the split kernel from the committed ncu capture, as a
-# ratio to the algorithmic KV bytes of that launch (profiles/); None = no capture yet.
-NCU_TRAFFIC_RATIO = None
+# DRAM bytes (read + write) per launch of the split kernel in the committed ncu capture
+# (profiles/decode_attn_split_config3_ncu.md: 1.577394 GB + 4.45 MB), as a ratio to the
+# algorithmic KV bytes of that launch (1.576878 GB); traffic grows in proportion to the pages read.
+NCU_TRAFFIC_RATIO = 1.0031
 
 
 def measured_hbm_peak():
@@ -312,12 +313,19 @@ def time_oracle_once(w, cache, q, lens, max_seconds_hint: float = 30.0):
     qb = oracle.bf16_bits(q[:n])
     t = time.perf_counter()
     oracle.decode_attn(qb, kp, vp, new_table, sub_lens, w.sm_scale, nthreads=cores)
-    dt = time.perf_counter() - t
+    first = time.perf_counter() - t
+    # repeat the same step until about 15 core-seconds of CPU work have been timed
+    reps = int(min(20, max(1, round(15.0 / max(first * cores, 1e-3)))))
+    t = time.perf_counter()
+    for _ in range(reps):
+        oracle.decode_attn(qb, kp, vp, new_table, sub_lens, w.sm_scale, nthreads=cores)
+    dt = (time.perf_counter() - t) / reps
     nbytes = float(np.sum(sub_lens)) * w.kv_bytes_per_token
     return {"value": round(nbytes / dt / 1e9, 4), "unit": "GB/s", "cores": cores, "kind": "oracle",
             "sample": f"attention of the first {n} of {B} sequences ({int(np.sum(sub_lens))} cached tokens, "
-                      f"{nbytes / 1e9:.3f} GB of KV), one step, {dt:.2f} s wall on {cores} threads",
-            "seconds": round(dt, 3)}
+                      f"{nbytes / 1e9:.3f} GB of KV per step), {reps} steps, {dt:.2f} s wall per step on "
+                      f"{cores} threads",
+            "seconds_per_step": round(dt, 3)}
 
 
 # ------------------------------------------------------------------------------------------ reference arm
