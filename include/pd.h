@@ -131,6 +131,43 @@ int pd_decode_step_host(pd_ctx *ctx, const void *q_host, const void *k_new_host,
                         void *out_host, int32_t batch, float sm_scale, int32_t split_pages, void *stream);
 
 /*
+ * Decode attention without any allocation (the paper has no counterpart; this
+ * is a packaging variant of pd_decode_attn for restricted hosts).
+ *
+ * For callers that cannot allocate device memory at the time they need
+ * attention: an engine that has already given the whole device to its own
+ * KV-cache pool, a plugin that lives inside another framework's memory budget,
+ * a process whose allocator is frozen after warm-up. pd_create calls cudaMalloc
+ * and is therefore closed to them; this function needs no context. It computes
+ * exactly what pd_decode_attn computes with split_pages = 0, with the kernels'
+ * scratch (fp32 partials, page prefix sums, plan and status words) held in a
+ * fixed 16 MiB array inside the library image. Every device that loads the
+ * library carries that array until the process exits. The function calls no
+ * cudaMalloc, cudaFree or allocating library routine.
+ *
+ * Geometry comes from *cfg (num_q_heads, num_kv_heads, head_dim, page_size,
+ * max_pages_per_seq, num_pages, device; max_batch and flags are ignored); the
+ * tensors are the caller's, as for pd_decode_attn. Limit: the partials must fit
+ * the fixed array, i.e. roughly (SM count * 8 + batch * num_kv_heads) *
+ * group * (head_dim * 4 + 8) bytes <= 16 MiB - on a 148-SM device about
+ * batch <= 350 at 32/8 heads, head_dim 128. Larger batches return
+ * PD_ERR_WORKSPACE and launch nothing.
+ *
+ * The first call on each device resolves the array's device address and sets
+ * the kernel's shared-memory attribute; make that first call outside any CUDA
+ * stream capture. All calls on a device share the one array, which keeps the
+ * previous call's contents (the function clears the status latch itself, the
+ * only word that must start at zero): two calls whose kernels may overlap on
+ * the GPU - different streams, or concurrent host threads - race on it. Issue
+ * them on one stream or order them with events. Out-of-range page ids are
+ * clamped to page 0 as in pd_decode_attn but are not reported, since there is
+ * no context to query.
+ */
+int pd_decode_attn_static(const pd_config *cfg, const void *q, const void *k_pages, const void *v_pages,
+                          const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse,
+                          int32_t batch, float sm_scale, void *stream);
+
+/*
  * Waits for `stream`, then reports and clears the first fault a kernel of this
  * context latched since the last call: *code is PD_OK, PD_ERR_DEVICE_FAULT or
  * PD_ERR_TIMEOUT; *seq the sequence index (or -1); *detail the offending page

@@ -26,7 +26,8 @@ PD_APPEND_NO_ADVANCE = 1
 
 # every symbol include/pd.h declares
 EXPORTS = (
-    "pd_create", "pd_destroy", "pd_kv_append", "pd_decode_attn", "pd_decode_step_host", "pd_device_status",
+    "pd_create", "pd_destroy", "pd_kv_append", "pd_decode_attn", "pd_decode_attn_static", "pd_decode_step_host",
+    "pd_device_status",
     "pd_set_profile_events", "pd_workspace_bytes", "pd_launch_count", "pd_last_plan", "pd_status_string", "pd_last_error", "pd_version",
 )
 
@@ -58,6 +59,7 @@ def _load() -> ctypes.CDLL:
     lib.pd_destroy.argtypes = [vp]
     lib.pd_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, u32, vp]
     lib.pd_decode_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, vp]
+    lib.pd_decode_attn_static.argtypes = [ctypes.POINTER(pd_config), vp, vp, vp, vp, vp, vp, vp, i32, f32, vp]
     lib.pd_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, vp]
     lib.pd_device_status.argtypes = [vp, vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
     lib.pd_set_profile_events.argtypes = [vp, vp, vp]
@@ -132,6 +134,16 @@ def pd_decode_attn(ctx, q, k_pages, v_pages, page_table, ctx_lens, out, lse=None
     _check(_lib.pd_decode_attn(ctx, _ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(page_table), _ptr(ctx_lens),
                                _ptr(out), _ptr(lse), batch, sm_scale, split_pages, _stream(stream)),
            "pd_decode_attn", ctx)
+
+
+def pd_decode_attn_static(cfg: pd_config, q, k_pages, v_pages, page_table, ctx_lens, out, lse=None, batch=None,
+                          sm_scale=1.0, stream=None):
+    """Attention for callers that may not allocate: no context, scratch lives in a fixed array
+    inside the library. ``cfg`` is a ``pd_config`` describing the geometry and the device."""
+    batch = q.shape[0] if batch is None else batch
+    _check(_lib.pd_decode_attn_static(ctypes.byref(cfg), _ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(page_table),
+                                      _ptr(ctx_lens), _ptr(out), _ptr(lse), batch, sm_scale, _stream(stream)),
+           "pd_decode_attn_static")
 
 
 def pd_decode_step_host(ctx, q_host, k_new_host, v_new_host, k_pages, v_pages, page_table, ctx_lens, out_host,
