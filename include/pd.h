@@ -100,16 +100,17 @@ int pd_kv_append(pd_ctx *ctx, const void *k_new, const void *v_new, void *k_page
  * out = 0 and lse = -inf. Slots past ctx_lens[b] and unused pages may hold
  * anything (NaN included) and do not influence the result.
  *
- * The flattened list of (sequence, KV head, page) units is cut into equal
- * ranges, one per worker warp, so that few long sequences (low decode
- * concurrency, Eq. 2) still occupy every SM; a range that holds only part of a
- * (sequence, KV head) context produces an fp32 partial (unnormalised output,
- * running max, running sum) in the workspace and a second kernel merges the
- * partials of each row by log-sum-exp. split_pages = 0 picks the range length
- * from the total page count and the SM count on the device; split_pages > 0
- * forces that many pages per range (raised silently if the workspace could not
- * hold the resulting partials). Results are bit-reproducible run to run for a
- * fixed split_pages and device.
+ * The flattened list of (sequence, KV head, page) units is cut into ranges that
+ * worker warps claim in order, long ranges first and short ones last, so that
+ * few long sequences (low decode concurrency, Eq. 2) still occupy every SM and
+ * all SMs finish together; a range that holds only part of a (sequence, KV
+ * head) context produces an fp32 partial (unnormalised output, running max,
+ * running sum) in the workspace and a second kernel merges the partials of each
+ * row by log-sum-exp. split_pages = 0 derives the ranges from the total page
+ * count and the SM count of the device; split_pages > 0 forces ranges of that
+ * many pages (raised silently if the workspace could not hold the resulting
+ * partials). Range boundaries never depend on timing, so results are
+ * bit-reproducible run to run for a fixed split_pages and device.
  *
  * sm_scale must be finite and positive. q/out rows are head_dim bf16.
  */
@@ -184,6 +185,17 @@ int pd_device_status(pd_ctx *ctx, void *stream, int32_t *code, int32_t *seq, int
  */
 int pd_set_profile_events(pd_ctx *ctx, void *before, void *after);
 
+/*
+ * Per-worker timestamps of the most recent pd_decode_attn, for profiling the
+ * start-up and tail of the split kernel. Available only when the environment
+ * variable PD_TRACE_WORKERS=1 was set at pd_create (otherwise
+ * PD_ERR_UNSUPPORTED). Waits for `stream`, then copies up to max_workers
+ * records of four uint64 nanosecond values (%globaltimer: kernel entry, first
+ * tile landed, last tile landed, exit) to host_out (HOST pointer) and stores
+ * the number of records in *num_workers.
+ */
+int pd_read_worker_trace(pd_ctx *ctx, void *stream, uint64_t *host_out, int32_t max_workers, int32_t *num_workers);
+
 /* Bytes of device workspace the context holds. */
 int pd_workspace_bytes(const pd_ctx *ctx, size_t *bytes);
 
@@ -192,8 +204,9 @@ int pd_launch_count(const pd_ctx *ctx, int64_t *launches);
 
 /*
  * Plan of the most recent pd_decode_attn call, read back from the device after
- * waiting for `stream`: total (sequence, KV head, page) units, pages per range,
- * number of ranges, number of worker warps launched. For tests and reporting.
+ * waiting for `stream`: total (sequence, KV head, page) units, pages per range
+ * of the first (longest) level of ranges, number of ranges over all levels,
+ * number of worker warps launched. For tests and reporting.
  */
 int pd_last_plan(pd_ctx *ctx, void *stream, int64_t *total_units, int32_t *pages_per_range,
                  int32_t *num_ranges, int32_t *num_workers);

@@ -27,7 +27,7 @@ PD_APPEND_NO_ADVANCE = 1
 # every symbol include/pd.h declares
 EXPORTS = (
     "pd_create", "pd_destroy", "pd_kv_append", "pd_decode_attn", "pd_decode_attn_static", "pd_decode_step_host",
-    "pd_device_status",
+    "pd_device_status", "pd_read_worker_trace",
     "pd_set_profile_events", "pd_workspace_bytes", "pd_launch_count", "pd_last_plan", "pd_status_string", "pd_last_error", "pd_version",
 )
 
@@ -63,6 +63,7 @@ def _load() -> ctypes.CDLL:
     lib.pd_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, vp]
     lib.pd_device_status.argtypes = [vp, vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
     lib.pd_set_profile_events.argtypes = [vp, vp, vp]
+    lib.pd_read_worker_trace.argtypes = [vp, vp, vp, i32, ctypes.POINTER(i32)]
     lib.pd_workspace_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
     lib.pd_launch_count.argtypes = [vp, ctypes.POINTER(i64)]
     lib.pd_last_plan.argtypes = [vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i32), ctypes.POINTER(i32),
@@ -173,6 +174,17 @@ def pd_set_profile_events(ctx, before=None, after=None) -> None:
             ev.record()
         return ev.cuda_event
     _check(_lib.pd_set_profile_events(ctx, handle(before), handle(after)), "pd_set_profile_events", ctx)
+
+
+def pd_read_worker_trace(ctx, max_workers=4096, stream=None):
+    """uint64 array [workers, 4] of ns timestamps (needs PD_TRACE_WORKERS=1 at pd_create)."""
+    import numpy as np
+
+    buf = np.zeros((max_workers, 4), dtype=np.uint64)
+    n = ctypes.c_int32()
+    _check(_lib.pd_read_worker_trace(ctx, _stream(stream), buf.ctypes.data, max_workers, ctypes.byref(n)),
+           "pd_read_worker_trace", ctx)
+    return buf[:n.value]
 
 
 def pd_workspace_bytes(ctx) -> int:

@@ -39,6 +39,8 @@ struct pd_ctx {
     size_t smem_bytes = 0;
     int max_ranges = 0;
     int min_pages_auto = 1;
+    int halving_levels = 0;
+    int tail_pages = 16;
     size_t slots = 0;
     // device workspace (one allocation)
     void *workspace = nullptr;
@@ -48,6 +50,8 @@ struct pd_ctx {
     int32_t *cum_pages = nullptr;
     int32_t *plan = nullptr;
     int32_t *status = nullptr;
+    unsigned long long *trace = nullptr;  // per-worker timestamps, only with PD_TRACE_WORKERS=1
+    int trace_workers = 0;
     // staging for pd_decode_step_host
     __nv_bfloat16 *stage_q = nullptr, *stage_k = nullptr, *stage_v = nullptr, *stage_out = nullptr;
     // tensor maps, cached per pool pointer
@@ -160,6 +164,12 @@ int pd_create(const pd_config *cfg, pd_ctx **out) {
     ctx->variant = v;
     ctx->num_ctas = ctx->num_sms * env_int("PD_TUNE_CTAS_PER_SM", 1);
     ctx->min_pages_auto = env_int("PD_TUNE_MIN_PAGES", 4);
+    ctx->halving_levels = env_int("PD_TUNE_LEVELS", 6);
+    ctx->tail_pages = env_int("PD_TUNE_TAIL", 16);
+    if (ctx->halving_levels < 0 || ctx->halving_levels > pd::kMaxLevels - 2 || ctx->tail_pages < 1) {
+        delete ctx;
+        return PD_ERR_INVALID_ARG;
+    }
     cudaError_t err = pd::prepare_decode_attn(v, &ctx->smem_bytes);
     if (err != cudaSuccess) {
         delete ctx;
@@ -177,7 +187,7 @@ int pd_create(const pd_config *cfg, pd_ctx **out) {
 
     // workspace: partial slots = ranges + one per (sequence, KV head)
     const int n_workers = ctx->num_ctas * v.warps;
-    ctx->max_ranges = 4 * n_workers;
+    ctx->max_ranges = 16 * n_workers;
     ctx->slots = static_cast<size_t>(ctx->max_ranges) + static_cast<size_t>(cfg->max_batch) * cfg->num_kv_heads;
     auto round256 = [](size_t n) { return (n + 255) & ~size_t(255); };
     const size_t b_part_o = round256(ctx->slots * group * cfg->head_dim * sizeof(float));
@@ -187,7 +197,8 @@ int pd_create(const pd_config *cfg, pd_ctx **out) {
     const size_t b_status = round256(pd::kStatusWords * sizeof(int32_t));
     const size_t b_q = round256(static_cast<size_t>(cfg->max_batch) * cfg->num_q_heads * cfg->head_dim * 2);
     const size_t b_kv = round256(static_cast<size_t>(cfg->max_batch) * cfg->num_kv_heads * cfg->head_dim * 2);
-    ctx->workspace_bytes = b_part_o + b_part_ml + b_cum + b_plan + b_status + 2 * b_q + 2 * b_kv;
+    const size_t b_trace = env_int("PD_TRACE_WORKERS", 0) ? round256(static_cast<size_t>(n_workers) * 4 * 8) : 0;
+    ctx->workspace_bytes = b_part_o + b_part_ml + b_cum + b_plan + b_status + 2 * b_q + 2 * b_kv + b_trace;
     err = cudaMalloc(&ctx->workspace, ctx->workspace_bytes);
     if (err != cudaSuccess) {
         delete ctx;
@@ -203,6 +214,10 @@ int pd_create(const pd_config *cfg, pd_ctx **out) {
     ctx->stage_out = reinterpret_cast<__nv_bfloat16 *>(w); w += b_q;
     ctx->stage_k = reinterpret_cast<__nv_bfloat16 *>(w); w += b_kv;
     ctx->stage_v = reinterpret_cast<__nv_bfloat16 *>(w); w += b_kv;
+    if (b_trace != 0) {
+        ctx->trace = reinterpret_cast<unsigned long long *>(w);
+        ctx->trace_workers = n_workers;
+    }
     err = cudaMemset(ctx->workspace, 0, ctx->workspace_bytes);
     if (err != cudaSuccess) {
         cudaFree(ctx->workspace);
@@ -293,6 +308,9 @@ int pd_decode_attn(pd_ctx *ctx, const void *q, const void *k_pages, const void *
     p.split_pages = split_pages;
     p.max_ranges = ctx->max_ranges;
     p.min_pages_auto = ctx->min_pages_auto;
+    p.halving_levels = ctx->halving_levels;
+    p.tail_pages = ctx->tail_pages;
+    p.trace = ctx->trace;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (ctx->ev_before != nullptr) cudaEventRecord(ctx->ev_before, s);
     cudaError_t err = pd::launch_decode_attn(ctx->variant, ctx->tm_k, ctx->tm_v, p, ctx->num_ctas, ctx->smem_bytes, s);
@@ -357,6 +375,21 @@ int pd_set_profile_events(pd_ctx *ctx, void *before, void *after) {
     return PD_OK;
 }
 
+int pd_read_worker_trace(pd_ctx *ctx, void *stream, uint64_t *host_out, int32_t max_workers, int32_t *num_workers) {
+    if (ctx == nullptr || host_out == nullptr || num_workers == nullptr || max_workers < 0) return PD_ERR_INVALID_ARG;
+    *num_workers = 0;
+    if (ctx->trace == nullptr) return fail(ctx, PD_ERR_UNSUPPORTED, "tracing is off (set PD_TRACE_WORKERS=1 before pd_create)");
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
+    const int n = ctx->trace_workers < max_workers ? ctx->trace_workers : max_workers;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t err = cudaMemcpyAsync(host_out, ctx->trace, static_cast<size_t>(n) * 4 * 8, cudaMemcpyDeviceToHost, s);
+    if (err == cudaSuccess) err = cudaStreamSynchronize(s);
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "trace read", err);
+    *num_workers = n;
+    return PD_OK;
+}
+
 int pd_workspace_bytes(const pd_ctx *ctx, size_t *bytes) {
     if (ctx == nullptr || bytes == nullptr) return PD_ERR_INVALID_ARG;
     *bytes = ctx->workspace_bytes;
@@ -381,7 +414,7 @@ int pd_last_plan(pd_ctx *ctx, void *stream, int64_t *total_units, int32_t *pages
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "plan read", err);
     if (total_units != nullptr)
         *total_units = (static_cast<int64_t>(host[1]) << 32) | static_cast<uint32_t>(host[0]);
-    if (pages_per_range != nullptr) *pages_per_range = host[2];
+    if (pages_per_range != nullptr) *pages_per_range = host[pd::kPlanHeaderWords + 2];  // first (largest) level
     if (num_ranges != nullptr) *num_ranges = host[3];
     if (num_workers != nullptr) *num_workers = host[4];
     return PD_OK;

@@ -6,14 +6,23 @@
 // HBM speed; everything below serves that.
 //
 // Work decomposition. Units are (sequence, KV head, page) triples in that
-// nesting order; their flattened list is cut into ranges of `per` units. A
-// worker is ONE WARP: it owns a range, its own ring of shared-memory stages and
-// its own mbarriers, issues its own TMA loads (lane 0) and never synchronises
-// with another warp after the prologue. A range may cross (sequence, KV head)
-// boundaries; each maximal piece inside one (sequence, KV head) is a segment.
-// A segment that covers the whole context writes the final bf16 row directly;
-// any other segment writes an fp32 partial to slot (range index + pair index),
-// which is unique and contiguous per pair, and the merge kernel combines them.
+// nesting order. Their flattened list is cut into ranges by a plan every CTA
+// derives from the lengths alone: a few levels whose ranges are half of the
+// remaining fair share per worker, then a tail level of short ranges. A worker
+// is ONE WARP with its own ring of shared-memory stages and its own mbarriers;
+// it issues its own TMA loads (lane 0) and never synchronises with another warp
+// after the prologue. Its first range is its own index; further ranges are
+// claimed in index order from one atomic counter, so SMs that get more
+// bandwidth take more of the later, shorter ranges and all workers finish
+// together. The loads of the next range are issued while the current one is
+// still being consumed. Range boundaries do not depend on who claims what, so
+// results are bit-reproducible.
+//
+// A range may cross (sequence, KV head) boundaries; each maximal piece inside
+// one pair is a segment. A segment that covers the whole context writes the
+// final bf16 row directly; any other segment writes an fp32 partial to slot
+// (range index + pair index), unique and contiguous per pair, and the merge
+// kernel combines them.
 //
 // Data movement. A (page, KV head) tile is 16 tokens x D bf16, contiguous in
 // HBM. It is fetched by tiled TMA as D/64 boxes of 16 rows x 128 B with the
@@ -32,6 +41,7 @@ namespace pd {
 namespace {
 
 constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kClaimAhead = 2;  // pages left to issue in a range when the next range is claimed
 
 struct Cursor {
     int b, kvh, page, np;  // np = pages of sequence b
@@ -41,6 +51,19 @@ struct Cursor {
 // the following 32 prefetched.
 struct PageIdCache {
     int b, blk, val, nval;
+};
+
+// One level of the plan: `count` ranges of `size` units starting at unit `start`;
+// `first` is the index of its first range. lv[n_levels] is a sentinel
+// (start = total, first = number of ranges).
+struct PlanLevel {
+    long long start;
+    int size, first;
+};
+struct Plan {
+    long long total;
+    int n_levels, n_ranges;
+    PlanLevel lv[kMaxLevels + 1];
 };
 
 __device__ __forceinline__ void latch_status(int32_t *status, int code, int seq, int detail) {
@@ -85,7 +108,55 @@ __device__ void scan_pages(const AttnParams &p, int32_t *cum, int32_t *warp_sums
     __syncthreads();
 }
 
-__device__ __forceinline__ Cursor locate(const int32_t *cum, int B, int Hkv, int64_t x) {
+// The plan is a pure function of (total, workers, parameters): every CTA and the
+// merge kernel's reader derive the same one.
+__device__ void make_plan(Plan &pl, long long total, int n_workers, const AttnParams &p) {
+    pl.total = total;
+    int nl = 0, first = 0;
+    long long pos = 0;
+    if (p.split_pages > 0) {
+        long long size = p.split_pages;
+        if ((total + size - 1) / size > p.max_ranges) size = (total + p.max_ranges - 1) / p.max_ranges;
+        pl.lv[0].start = 0; pl.lv[0].size = static_cast<int>(size); pl.lv[0].first = 0;
+        first = static_cast<int>((total + size - 1) / size);
+        nl = 1;
+    } else {
+        long long fair = (total + n_workers - 1) / n_workers;
+        const int tail = static_cast<int>(max(static_cast<long long>(p.min_pages_auto),
+                                              min(static_cast<long long>(p.tail_pages), fair)));
+        for (int l = 0; l < p.halving_levels && nl < kMaxLevels - 1; ++l) {
+            const long long rem = total - pos;
+            const long long size = (rem + 2ll * n_workers - 1) / (2ll * n_workers);
+            if (size < 2ll * tail || first + 2 * n_workers > p.max_ranges) break;
+            pl.lv[nl].start = pos; pl.lv[nl].size = static_cast<int>(size); pl.lv[nl].first = first;
+            pos += size * n_workers;
+            first += n_workers;
+            ++nl;
+        }
+        const long long rem = total - pos;
+        if (rem > 0 || nl == 0) {
+            long long size = p.halving_levels > 0 ? tail : max(fair, static_cast<long long>(p.min_pages_auto));
+            const long long room = max(1, p.max_ranges - first);
+            if ((rem + size - 1) / size > room) size = (rem + room - 1) / room;
+            if (size < 1) size = 1;
+            pl.lv[nl].start = pos; pl.lv[nl].size = static_cast<int>(size); pl.lv[nl].first = first;
+            first += static_cast<int>((rem + size - 1) / size);
+            ++nl;
+        }
+    }
+    pl.lv[nl].start = total; pl.lv[nl].size = 1; pl.lv[nl].first = first;
+    pl.n_levels = nl;
+    pl.n_ranges = first;
+}
+
+__device__ __forceinline__ void range_bounds(const Plan &pl, int rid, long long &start, int &len) {
+    int l = 0;
+    while (l + 1 < pl.n_levels && rid >= pl.lv[l + 1].first) ++l;
+    start = pl.lv[l].start + static_cast<long long>(rid - pl.lv[l].first) * pl.lv[l].size;
+    len = static_cast<int>(min(static_cast<long long>(pl.lv[l].size), pl.lv[l + 1].start - start));
+}
+
+__device__ __forceinline__ Cursor locate(const int32_t *cum, int B, int Hkv, long long x) {
     const int y = static_cast<int>(x / Hkv);  // largest b with cum[b] <= y owns unit x
     int lo = 0, hi = B - 1;
     while (lo < hi) {
@@ -95,15 +166,14 @@ __device__ __forceinline__ Cursor locate(const int32_t *cum, int B, int Hkv, int
     Cursor c;
     c.b = lo;
     c.np = cum[lo + 1] - cum[lo];
-    const int rem = static_cast<int>(x - static_cast<int64_t>(Hkv) * cum[lo]);
+    const int rem = static_cast<int>(x - static_cast<long long>(Hkv) * cum[lo]);
     c.kvh = rem / c.np;
     c.page = rem - c.kvh * c.np;
     return c;
 }
 
-__device__ __forceinline__ void advance(Cursor &c, const int32_t *cum, int B, int Hkv, int pages) {
-    c.page += pages;
-    if (c.page >= c.np) {
+__device__ __forceinline__ void advance(Cursor &c, const int32_t *cum, int B, int Hkv) {
+    if (++c.page >= c.np) {
         c.page = 0;
         if (++c.kvh == Hkv) {
             c.kvh = 0;
@@ -150,10 +220,14 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     const uint32_t ring0 = (raw + 1023u) & ~1023u;  // swizzled boxes need 1024-byte alignment
     uint8_t *aligned = smem_raw + (ring0 - raw);
     uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + WARPS * STAGES * STAGE_BYTES);
-    int32_t *warp_sums = reinterpret_cast<int32_t *>(bars + WARPS * STAGES * 2);
+    Plan *plan_s = reinterpret_cast<Plan *>(bars + WARPS * STAGES * 2);
+    int32_t *stage_range = reinterpret_cast<int32_t *>(plan_s + 1);  // [WARPS][STAGES] range id of the page in a stage
+    int32_t *warp_sums = stage_range + WARPS * STAGES;
     int32_t *cum = warp_sums + 32;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned long long t_entry = p.trace != nullptr ? global_timer_ns() : 0ull;
+    unsigned long long t_first = 0ull, t_last = 0ull;
 
     // ---- prologue (whole CTA): barriers, page prefix sums, the plan
     if (lane == 0) {
@@ -166,32 +240,33 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     }
     scan_pages<THREADS>(p, cum, warp_sums);
 
-    const int64_t total = static_cast<int64_t>(p.Hkv) * cum[p.B];
     const int n_workers = gridDim.x * WARPS;
-    int64_t per;
-    if (p.split_pages > 0) {
-        per = p.split_pages;
-        if ((total + per - 1) / per > p.max_ranges) per = (total + p.max_ranges - 1) / p.max_ranges;
-    } else {
-        per = (total + n_workers - 1) / n_workers;
-        if (per < p.min_pages_auto) per = p.min_pages_auto;
-    }
-    if (per < 1) per = 1;
-    const int64_t n_ranges = (total + per - 1) / per;
+    if (tid == 0) make_plan(*plan_s, static_cast<long long>(p.Hkv) * cum[p.B], n_workers, p);
+    __syncthreads();
+    const Plan &pl = *plan_s;
     if (blockIdx.x == 0) {
         for (int i = tid; i <= p.B; i += THREADS) p.cum_pages[i] = cum[i];
         if (tid == 0) {
-            p.plan[0] = static_cast<int32_t>(total & 0xffffffffll);
-            p.plan[1] = static_cast<int32_t>(total >> 32);
-            p.plan[2] = static_cast<int32_t>(per);
-            p.plan[3] = static_cast<int32_t>(n_ranges);
+            p.plan[0] = static_cast<int32_t>(pl.total & 0xffffffffll);
+            p.plan[1] = static_cast<int32_t>(pl.total >> 32);
+            p.plan[2] = pl.n_levels;
+            p.plan[3] = pl.n_ranges;
             p.plan[4] = n_workers;
+        }
+        if (tid <= pl.n_levels) {
+            int32_t *rec = p.plan + kPlanHeaderWords + 4 * tid;
+            rec[0] = static_cast<int32_t>(pl.lv[tid].start & 0xffffffffll);
+            rec[1] = static_cast<int32_t>(pl.lv[tid].start >> 32);
+            rec[2] = pl.lv[tid].size;
+            rec[3] = pl.lv[tid].first;
         }
     }
 
     // ---- per-warp state
+    const int worker = blockIdx.x * WARPS + warp;
     const uint32_t ring = ring0 + warp * STAGES * STAGE_BYTES;
     const uint32_t bar0 = smem_u32(bars + warp * STAGES * 2);
+    int32_t *my_stage_range = stage_range + warp * STAGES;
     const uint64_t policy = l2_policy_evict_first();
     const int quad_row = lane >> 2;  // query head inside the group handled by this lane
     const int quad_col = (lane & 3) * 2;
@@ -205,174 +280,213 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
 
     PageIdCache pt;
     pt.b = -1; pt.blk = -1; pt.val = -1; pt.nval = -1;
-    uint32_t stage = 0, parity = 0;  // ring position of the next page to consume
-    bool alive = true;
 
-    for (int64_t range = blockIdx.x * WARPS + warp; range < n_ranges && alive; range += n_workers) {
-        const int64_t x0 = range * per;
-        const int n_total = static_cast<int>(min(total - x0, per));
-        Cursor cons = locate(cum, p.B, p.Hkv, x0);
-        Cursor prod = cons;
-        int issued = 0;
+    // producer side: the range being issued, the cursor inside it, the claim made ahead of need
+    Cursor prod;
+    prod.b = 0; prod.kvh = 0; prod.page = 0; prod.np = 1;
+    int p_rid = -1, p_left = 0;
+    bool p_first = true, p_done = false, have_next = false;
+    int next_raw = 0;
+    uint32_t p_stage = 0;
+    int inflight = 0;
 
-        auto issue = [&](uint32_t st) {
-            int pid = page_id(pt, p, prod.b, prod.page, lane);
-            if (pid < 0 || pid >= p.num_pages) {
-                if (lane == 0) latch_status(p.status, kDevBadPage, prod.b, pid);
-                pid = 0;
+    auto issue_next = [&]() -> bool {
+        if (p_left == 0) {
+            if (p_done) return false;
+            int rid;
+            if (p_first) {
+                rid = worker;
+                p_first = false;
+            } else {
+                if (!have_next && lane == 0) next_raw = atomicAdd(p.status + kSchedNext, 1);
+                rid = n_workers + __shfl_sync(0xffffffffu, next_raw, 0);
+                have_next = false;
             }
-            if (lane == 0) {
-                const int32_t y = (pid * p.Hkv + prod.kvh) * kPageSize;
-                const uint32_t dst = ring + st * STAGE_BYTES;
-                const uint32_t bk = bar0 + st * 16, bv = bk + 8;
-                mbar_arrive_expect_tx(bk, TILE_BYTES);
-#pragma unroll
-                for (int h = 0; h < HALVES; ++h) tma_load_2d(dst + h * HALF_BYTES, &tm_k, h * 64, y, bk, policy);
-                mbar_arrive_expect_tx(bv, TILE_BYTES);
-#pragma unroll
-                for (int h = 0; h < HALVES; ++h)
-                    tma_load_2d(dst + TILE_BYTES + h * HALF_BYTES, &tm_v, h * 64, y, bv, policy);
+            if (rid >= pl.n_ranges) {
+                p_done = true;
+                return false;
             }
-            advance(prod, cum, p.B, p.Hkv, 1);
-            ++issued;
-        };
-
-        {
-            uint32_t st = stage;
-            const int fill = min(STAGES, n_total);
-            while (issued < fill) {
-                issue(st);
-                st = (st + 1 == STAGES) ? 0 : st + 1;
-            }
+            long long start;
+            range_bounds(pl, rid, start, p_left);
+            prod = locate(cum, p.B, p.Hkv, start);
+            p_rid = rid;
         }
-
-        int consumed = 0;
-        while (consumed < n_total && alive) {
-            // ---- segment: pages [page0, page0 + seg) of (b, kvh)
-            const int b = cons.b, kvh = cons.kvh, page0 = cons.page;
-            const int seg = min(n_total - consumed, cons.np - page0);
-            const int L = clamp_len(__ldg(p.ctx_lens + b), p.MP);
-
-            // Q fragments: row quad_row of the group, zero rows beyond the group
-            uint32_t qa[KSTEPS][2];
-            {
-                const __nv_bfloat16 *qrow = p.q + (static_cast<size_t>(b) * p.Hq + kvh * G + quad_row) * D;
+        int pid = page_id(pt, p, prod.b, prod.page, lane);
+        if (pid < 0 || pid >= p.num_pages) {
+            if (lane == 0) latch_status(p.status, kDevBadPage, prod.b, pid);
+            pid = 0;
+        }
+        if (lane == 0) {
+            my_stage_range[p_stage] = p_rid;
+            const int32_t y = (pid * p.Hkv + prod.kvh) * kPageSize;
+            const uint32_t dst = ring + p_stage * STAGE_BYTES;
+            const uint32_t bk = bar0 + p_stage * 16, bv = bk + 8;
+            mbar_arrive_expect_tx(bk, TILE_BYTES);
 #pragma unroll
-                for (int kk = 0; kk < KSTEPS; ++kk) {
-                    if (quad_row < G) {
-                        qa[kk][0] = __ldg(reinterpret_cast<const uint32_t *>(qrow + kk * 16 + quad_col));
-                        qa[kk][1] = __ldg(reinterpret_cast<const uint32_t *>(qrow + kk * 16 + 8 + quad_col));
-                    } else {
-                        qa[kk][0] = 0u;
-                        qa[kk][1] = 0u;
-                    }
+            for (int h = 0; h < HALVES; ++h) tma_load_2d(dst + h * HALF_BYTES, &tm_k, h * 64, y, bk, policy);
+            mbar_arrive_expect_tx(bv, TILE_BYTES);
+#pragma unroll
+            for (int h = 0; h < HALVES; ++h)
+                tma_load_2d(dst + TILE_BYTES + h * HALF_BYTES, &tm_v, h * 64, y, bv, policy);
+        }
+        advance(prod, cum, p.B, p.Hkv);
+        --p_left;
+        if (p_left <= kClaimAhead && !have_next && !p_first) {  // claim the next range before it is needed
+            if (lane == 0) next_raw = atomicAdd(p.status + kSchedNext, 1);
+            have_next = true;
+        }
+        if (++p_stage == STAGES) p_stage = 0;
+        ++inflight;
+        __syncwarp();
+        return true;
+    };
+
+    while (inflight < STAGES && issue_next()) {}
+
+    // consumer side
+    Cursor cons;
+    cons.b = 0; cons.kvh = 0; cons.page = 0; cons.np = 1;
+    int c_rid = -1, c_left = 0;
+    uint32_t stage = 0, parity = 0;  // ring position of the next page to consume
+    bool alive = true, seg_open = false;
+    int seg_page0 = 0, L = 0;
+    uint32_t qa[KSTEPS][2];
+    float O[NTILES][4];
+    float m_run = -INFINITY, l_run = 0.f;
+
+    while (inflight > 0) {
+        if (c_left == 0) {  // first page of a range
+            c_rid = my_stage_range[stage];
+            long long start;
+            range_bounds(pl, c_rid, start, c_left);
+            cons = locate(cum, p.B, p.Hkv, start);
+        }
+        if (!seg_open) {  // first page of a segment: its queries, a fresh running state
+            seg_open = true;
+            seg_page0 = cons.page;
+            L = clamp_len(__ldg(p.ctx_lens + cons.b), p.MP);
+            const __nv_bfloat16 *qrow = p.q + (static_cast<size_t>(cons.b) * p.Hq + cons.kvh * G + quad_row) * D;
+#pragma unroll
+            for (int kk = 0; kk < KSTEPS; ++kk) {
+                if (quad_row < G) {
+                    qa[kk][0] = __ldg(reinterpret_cast<const uint32_t *>(qrow + kk * 16 + quad_col));
+                    qa[kk][1] = __ldg(reinterpret_cast<const uint32_t *>(qrow + kk * 16 + 8 + quad_col));
+                } else {
+                    qa[kk][0] = 0u;
+                    qa[kk][1] = 0u;
                 }
             }
-            float O[NTILES][4];
 #pragma unroll
             for (int j = 0; j < NTILES; ++j) { O[j][0] = 0.f; O[j][1] = 0.f; O[j][2] = 0.f; O[j][3] = 0.f; }
-            float m_run = -INFINITY, l_run = 0.f;
+            m_run = -INFINITY;
+            l_run = 0.f;
+        }
 
-            for (int i = 0; i < seg; ++i) {
-                const uint32_t kbase = ring + stage * STAGE_BYTES;
-                const uint32_t vbase = kbase + TILE_BYTES;
-                const uint32_t bk = bar0 + stage * 16, bv = bk + 8;
-                const int valid = L - (page0 + i) * kPageSize;  // tokens of this page inside the context
+        const uint32_t kbase = ring + stage * STAGE_BYTES;
+        const uint32_t vbase = kbase + TILE_BYTES;
+        const uint32_t bk = bar0 + stage * 16, bv = bk + 8;
+        const int valid = L - cons.page * kPageSize;  // tokens of this page inside the context
 
-                if (!__all_sync(0xffffffffu, mbar_wait(bk, parity))) { alive = false; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait(bk, parity))) { alive = false; break; }
+        if (p.trace != nullptr) {
+            t_last = global_timer_ns();
+            if (t_first == 0ull) t_first = t_last;
+        }
 
-                // S = Q K^T for 16 tokens: two 8-token column tiles, two accumulators each
-                float Sa[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-                float Sb[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        // S = Q K^T for 16 tokens: two 8-token column tiles, two accumulators each
+        float Sa[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        float Sb[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
-                for (int kk = 0; kk < KSTEPS; ++kk) {
-                    uint32_t b0, b1, b2, b3;
-                    ldmatrix_x4(b0, b1, b2, b3,
-                                kbase + (kk >> 2) * HALF_BYTES + k_row_off + ((((kk & 3) * 2 + k_sel) ^ r8) << 4));
-                    if (kk & 1) {
-                        mma_bf16_16816(Sb[0], qa[kk][0], 0u, qa[kk][1], 0u, b0, b1);
-                        mma_bf16_16816(Sb[1], qa[kk][0], 0u, qa[kk][1], 0u, b2, b3);
-                    } else {
-                        mma_bf16_16816(Sa[0], qa[kk][0], 0u, qa[kk][1], 0u, b0, b1);
-                        mma_bf16_16816(Sa[1], qa[kk][0], 0u, qa[kk][1], 0u, b2, b3);
-                    }
-                }
-                // this lane: row quad_row, tokens quad_col, +1, +8, +9 (log2 units)
-                float s0 = (Sa[0][0] + Sb[0][0]) * p.scale_log2, s1 = (Sa[0][1] + Sb[0][1]) * p.scale_log2;
-                float s2 = (Sa[1][0] + Sb[1][0]) * p.scale_log2, s3 = (Sa[1][1] + Sb[1][1]) * p.scale_log2;
-                if (valid < kPageSize) {  // last page of the context: mask, never multiply
-                    if (quad_col >= valid) s0 = -INFINITY;
-                    if (quad_col + 1 >= valid) s1 = -INFINITY;
-                    if (quad_col + 8 >= valid) s2 = -INFINITY;
-                    if (quad_col + 9 >= valid) s3 = -INFINITY;
-                }
-                float mx = fmaxf(fmaxf(s0, s1), fmaxf(s2, s3));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float m_new = fmaxf(m_run, mx);
-                if (__any_sync(0xffffffffu, m_new > m_run)) {  // lazy rescale of the running state
-                    const float alpha = fast_exp2(m_run - m_new);
-                    l_run *= alpha;
-#pragma unroll
-                    for (int j = 0; j < NTILES; ++j) { O[j][0] *= alpha; O[j][1] *= alpha; }
-                    m_run = m_new;
-                }
-                const float p0 = fast_exp2(s0 - m_run), p1 = fast_exp2(s1 - m_run);
-                const float p2 = fast_exp2(s2 - m_run), p3 = fast_exp2(s3 - m_run);
-                l_run += (p0 + p1) + (p2 + p3);
-                const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1), h23 = __floats2bfloat162_rn(p2, p3);
-                const uint32_t pa0 = *reinterpret_cast<const uint32_t *>(&h01);
-                const uint32_t pa2 = *reinterpret_cast<const uint32_t *>(&h23);
-                uint32_t pl0 = 0u, pl2 = 0u;
-                if (HILO) {
-                    pl0 = pack_bf16x2(p0 - __low2float(h01), p1 - __high2float(h01));
-                    pl2 = pack_bf16x2(p2 - __low2float(h23), p3 - __high2float(h23));
-                }
-
-                if (!__all_sync(0xffffffffu, mbar_wait(bv, parity))) { alive = false; break; }
-                if (valid < kPageSize) {
-                    // V rows past the context may hold NaN; 0 * NaN is NaN, so clear them first
-                    for (int row = valid; row < kPageSize; ++row)
-                        if (lane < HALVES * 8)
-                            st_shared_zero16(vbase + (lane >> 3) * HALF_BYTES + row * 128 + (lane & 7) * 16);
-                    __syncwarp();
-                }
-                // O += P V : 16 tokens (k) x D columns
-#pragma unroll
-                for (int j = 0; j < NTILES / 2; ++j) {
-                    uint32_t v0, v1, v2, v3;
-                    ldmatrix_x4_trans(v0, v1, v2, v3,
-                                      vbase + (j >> 2) * HALF_BYTES + v_row_off + ((((j & 3) * 2 + v_sel) ^ r8) << 4));
-                    mma_bf16_16816(O[2 * j], pa0, 0u, pa2, 0u, v0, v1);
-                    mma_bf16_16816(O[2 * j + 1], pa0, 0u, pa2, 0u, v2, v3);
-                    if (HILO) {
-                        mma_bf16_16816(O[2 * j], pl0, 0u, pl2, 0u, v0, v1);
-                        mma_bf16_16816(O[2 * j + 1], pl0, 0u, pl2, 0u, v2, v3);
-                    }
-                }
-                __syncwarp();  // every lane has read this stage
-                if (valid < kPageSize) fence_proxy_async();  // generic-proxy stores before the next TMA write
-                if (issued < n_total) issue(stage);
-                if (++stage == STAGES) { stage = 0; parity ^= 1u; }
+        for (int kk = 0; kk < KSTEPS; ++kk) {
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4(b0, b1, b2, b3,
+                        kbase + (kk >> 2) * HALF_BYTES + k_row_off + ((((kk & 3) * 2 + k_sel) ^ r8) << 4));
+            if (kk & 1) {
+                mma_bf16_16816(Sb[0], qa[kk][0], 0u, qa[kk][1], 0u, b0, b1);
+                mma_bf16_16816(Sb[1], qa[kk][0], 0u, qa[kk][1], 0u, b2, b3);
+            } else {
+                mma_bf16_16816(Sa[0], qa[kk][0], 0u, qa[kk][1], 0u, b0, b1);
+                mma_bf16_16816(Sa[1], qa[kk][0], 0u, qa[kk][1], 0u, b2, b3);
             }
-            if (!alive) break;
+        }
+        // this lane: row quad_row, tokens quad_col, +1, +8, +9 (log2 units)
+        float s0 = (Sa[0][0] + Sb[0][0]) * p.scale_log2, s1 = (Sa[0][1] + Sb[0][1]) * p.scale_log2;
+        float s2 = (Sa[1][0] + Sb[1][0]) * p.scale_log2, s3 = (Sa[1][1] + Sb[1][1]) * p.scale_log2;
+        if (valid < kPageSize) {  // last page of the context: mask, never multiply
+            if (quad_col >= valid) s0 = -INFINITY;
+            if (quad_col + 1 >= valid) s1 = -INFINITY;
+            if (quad_col + 8 >= valid) s2 = -INFINITY;
+            if (quad_col + 9 >= valid) s3 = -INFINITY;
+        }
+        float mx = fmaxf(fmaxf(s0, s1), fmaxf(s2, s3));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(m_run, mx);
+        if (__any_sync(0xffffffffu, m_new > m_run)) {  // lazy rescale of the running state
+            const float alpha = fast_exp2(m_run - m_new);
+            l_run *= alpha;
+#pragma unroll
+            for (int j = 0; j < NTILES; ++j) { O[j][0] *= alpha; O[j][1] *= alpha; }
+            m_run = m_new;
+        }
+        const float p0 = fast_exp2(s0 - m_run), p1 = fast_exp2(s1 - m_run);
+        const float p2 = fast_exp2(s2 - m_run), p3 = fast_exp2(s3 - m_run);
+        l_run += (p0 + p1) + (p2 + p3);
+        const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1), h23 = __floats2bfloat162_rn(p2, p3);
+        const uint32_t pa0 = *reinterpret_cast<const uint32_t *>(&h01);
+        const uint32_t pa2 = *reinterpret_cast<const uint32_t *>(&h23);
+        uint32_t pl0 = 0u, pl2 = 0u;
+        if (HILO) {
+            pl0 = pack_bf16x2(p0 - __low2float(h01), p1 - __high2float(h01));
+            pl2 = pack_bf16x2(p2 - __low2float(h23), p3 - __high2float(h23));
+        }
 
-            // ---- end of segment: final row or partial
+        if (!__all_sync(0xffffffffu, mbar_wait(bv, parity))) { alive = false; break; }
+        if (valid < kPageSize) {
+            // V rows past the context may hold NaN; 0 * NaN is NaN, so clear them first
+            for (int row = valid; row < kPageSize; ++row)
+                if (lane < HALVES * 8)
+                    st_shared_zero16(vbase + (lane >> 3) * HALF_BYTES + row * 128 + (lane & 7) * 16);
+            __syncwarp();
+        }
+        // O += P V : 16 tokens (k) x D columns
+#pragma unroll
+        for (int j = 0; j < NTILES / 2; ++j) {
+            uint32_t v0, v1, v2, v3;
+            ldmatrix_x4_trans(v0, v1, v2, v3,
+                              vbase + (j >> 2) * HALF_BYTES + v_row_off + ((((j & 3) * 2 + v_sel) ^ r8) << 4));
+            mma_bf16_16816(O[2 * j], pa0, 0u, pa2, 0u, v0, v1);
+            mma_bf16_16816(O[2 * j + 1], pa0, 0u, pa2, 0u, v2, v3);
+            if (HILO) {
+                mma_bf16_16816(O[2 * j], pl0, 0u, pl2, 0u, v0, v1);
+                mma_bf16_16816(O[2 * j + 1], pl0, 0u, pl2, 0u, v2, v3);
+            }
+        }
+        __syncwarp();  // every lane has read this stage
+        if (valid < kPageSize) fence_proxy_async();  // generic-proxy stores before the next TMA write
+        --inflight;
+        issue_next();  // refills the stage just freed (p_stage == stage here)
+        if (++stage == STAGES) { stage = 0; parity ^= 1u; }
+
+        // ---- end of segment: final row or partial
+        --c_left;
+        const bool pair_end = cons.page + 1 == cons.np;
+        if (c_left == 0 || pair_end) {
             float l_tot = l_run + __shfl_xor_sync(0xffffffffu, l_run, 1);
             l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 2);
             if (quad_row < G) {
-                const int h = kvh * G + quad_row;
-                if (page0 == 0 && seg == cons.np) {
+                const int h = cons.kvh * G + quad_row;
+                if (seg_page0 == 0 && pair_end) {
                     const float inv = 1.f / l_tot;
-                    __nv_bfloat16 *orow = p.out + (static_cast<size_t>(b) * p.Hq + h) * D + quad_col;
+                    __nv_bfloat16 *orow = p.out + (static_cast<size_t>(cons.b) * p.Hq + h) * D + quad_col;
 #pragma unroll
                     for (int j = 0; j < NTILES; ++j)
                         *reinterpret_cast<__nv_bfloat162 *>(orow + j * 8) =
                             __floats2bfloat162_rn(O[j][0] * inv, O[j][1] * inv);
                     if (p.lse != nullptr && (lane & 3) == 0)
-                        p.lse[static_cast<size_t>(b) * p.Hq + h] = (m_run + log2f(l_tot)) * kLn2;
+                        p.lse[static_cast<size_t>(cons.b) * p.Hq + h] = (m_run + log2f(l_tot)) * kLn2;
                 } else {
-                    const size_t slot = static_cast<size_t>(range) + static_cast<size_t>(b) * p.Hkv + kvh;
+                    const size_t slot = static_cast<size_t>(c_rid) + static_cast<size_t>(cons.b) * p.Hkv + cons.kvh;
                     float *orow = p.part_o + (slot * G + quad_row) * D + quad_col;
 #pragma unroll
                     for (int j = 0; j < NTILES; ++j)
@@ -380,69 +494,139 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                     if ((lane & 3) == 0) p.part_ml[slot * G + quad_row] = make_float2(m_run, l_tot);
                 }
             }
-            consumed += seg;
-            advance(cons, cum, p.B, p.Hkv, seg);
+            seg_open = false;
+        }
+        advance(cons, cum, p.B, p.Hkv);
+    }
+
+    if (lane == 0) {
+        if (!alive) latch_status(p.status, kDevTimeout, -1, worker);
+        if (p.trace != nullptr) {
+            unsigned long long *t = p.trace + static_cast<size_t>(worker) * 4;
+            t[0] = t_entry; t[1] = t_first; t[2] = t_last; t[3] = global_timer_ns();
+        }
+        // the last worker to finish re-arms the claim counter for the next launch
+        if (atomicAdd(p.status + kSchedDone, 1) == n_workers - 1) {
+            p.status[kSchedNext] = 0;
+            p.status[kSchedDone] = 0;
         }
     }
-    if (!alive && lane == 0) latch_status(p.status, kDevTimeout, -1, blockIdx.x * WARPS + warp);
 }
 
-// One warp per (sequence, query head): combine that row's partials in slot order.
-template <int D>
-__global__ void __launch_bounds__(128) lse_merge_kernel(const AttnParams p) {
+// Index of the range that holds unit x, from the plan the split kernel left in global memory.
+__device__ __forceinline__ long long range_of_unit(const int32_t *plan, long long x) {
+    const int n_levels = plan[2];
+    const int32_t *rec = plan + kPlanHeaderWords;
+    int l = 0;
+    auto start_of = [&](int i) {
+        return (static_cast<long long>(rec[4 * i + 1]) << 32) | static_cast<unsigned int>(rec[4 * i]);
+    };
+    while (l + 1 < n_levels && x >= start_of(l + 1)) ++l;
+    return rec[4 * l + 3] + (x - start_of(l)) / rec[4 * l + 2];
+}
+
+// One CTA per (sequence, KV head): its warps take the pair's partials round-robin, each keeping a
+// running (max, sum, output) per query head of the group; the per-warp results are then combined
+// through shared memory in warp order. The order of operations is fixed, so reruns are bit-identical.
+template <int D, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32) lse_merge_kernel(const AttnParams p) {
     constexpr int VEC = D / 32;
-    const int lane = threadIdx.x & 31;
-    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (row >= p.B * p.Hq) return;
-    const int b = row / p.Hq, h = row - b * p.Hq;
-    const int kvh = h / p.G, r = h - kvh * p.G;
+    constexpr int GMAX = 8;
+    __shared__ float sm_o[WARPS][GMAX][D];
+    __shared__ float2 sm_ml[WARPS][GMAX];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int pair = blockIdx.x;
+    const int b = pair / p.Hkv, kvh = pair - b * p.Hkv;
+    const int G = p.G;
     const int c0 = p.cum_pages[b], np = p.cum_pages[b + 1] - c0;
-    __nv_bfloat16 *orow = p.out + static_cast<size_t>(row) * D + lane * VEC;
-    if (np == 0) {  // empty context
-#pragma unroll
-        for (int v = 0; v < VEC; ++v) orow[v] = __float2bfloat16(0.f);
-        if (p.lse != nullptr && lane == 0) p.lse[row] = -INFINITY;
+    __nv_bfloat16 *obase = p.out + (static_cast<size_t>(b) * p.Hq + kvh * G) * D;
+    if (np == 0) {  // empty context: zero rows, lse = -inf
+        for (int i = threadIdx.x; i < G * D; i += WARPS * 32) obase[i] = __float2bfloat16(0.f);
+        if (p.lse != nullptr && threadIdx.x < G) p.lse[static_cast<size_t>(b) * p.Hq + kvh * G + threadIdx.x] = -INFINITY;
         return;
     }
-    const int64_t per = p.plan[2];
-    const int64_t u0 = static_cast<int64_t>(p.Hkv) * c0 + static_cast<int64_t>(kvh) * np;
-    const int64_t first = u0 / per, last = (u0 + np - 1) / per;
+    const long long u0 = static_cast<long long>(p.Hkv) * c0 + static_cast<long long>(kvh) * np;
+    const long long first = range_of_unit(p.plan, u0), last = range_of_unit(p.plan, u0 + np - 1);
     if (first == last) return;  // written directly by the split kernel
     const int n = static_cast<int>(last - first) + 1;
-    const size_t slot0 = static_cast<size_t>(first) + static_cast<size_t>(b) * p.Hkv + kvh;
-    float M = -INFINITY;
-    for (int i = lane; i < n; i += 32) M = fmaxf(M, p.part_ml[(slot0 + i) * p.G + r].x);
+    const size_t slot0 = static_cast<size_t>(first) + pair;
+
+    float m[GMAX], l[GMAX], acc[GMAX][VEC];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    float acc[VEC];
+    for (int r = 0; r < GMAX; ++r) {
+        m[r] = -INFINITY;
+        l[r] = 0.f;
 #pragma unroll
-    for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
-    float Lsum = 0.f;
-    for (int i = 0; i < n; ++i) {
-        const float2 ml = p.part_ml[(slot0 + i) * p.G + r];
-        const float w = exp2f(ml.x - M);
-        Lsum += w * ml.y;
-        const float *src = p.part_o + ((slot0 + i) * p.G + r) * D + lane * VEC;
-        if (VEC == 4) {
-            const float4 o = *reinterpret_cast<const float4 *>(src);
-            acc[0] += w * o.x; acc[1] += w * o.y; acc[VEC - 2] += w * o.z; acc[VEC - 1] += w * o.w;
-        } else {
-            const float2 o = *reinterpret_cast<const float2 *>(src);
-            acc[0] += w * o.x; acc[1] += w * o.y;
+        for (int v = 0; v < VEC; ++v) acc[r][v] = 0.f;
+    }
+    for (int i = warp; i < n; i += WARPS) {
+        const float2 *ml_src = p.part_ml + (slot0 + i) * G;
+        const float *o_src = p.part_o + (slot0 + i) * G * D + lane * VEC;
+        float2 ml[GMAX];
+        float o[GMAX][VEC];
+#pragma unroll
+        for (int r = 0; r < GMAX; ++r) {
+            if (r < G) {
+                ml[r] = ml_src[r];
+                if (VEC == 4) {
+                    const float4 t = *reinterpret_cast<const float4 *>(o_src + r * D);
+                    o[r][0] = t.x; o[r][1] = t.y; o[r][VEC - 2] = t.z; o[r][VEC - 1] = t.w;
+                } else {
+                    const float2 t = *reinterpret_cast<const float2 *>(o_src + r * D);
+                    o[r][0] = t.x; o[r][1] = t.y;
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < GMAX; ++r) {
+            if (r < G) {
+                const float m_new = fmaxf(m[r], ml[r].x);
+                const float a = exp2f(m[r] - m_new), w = exp2f(ml[r].x - m_new);
+                l[r] = l[r] * a + w * ml[r].y;
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) acc[r][v] = acc[r][v] * a + w * o[r][v];
+                m[r] = m_new;
+            }
         }
     }
-    const float inv = 1.f / Lsum;
 #pragma unroll
-    for (int v = 0; v < VEC; v += 2)
-        *reinterpret_cast<__nv_bfloat162 *>(orow + v) = __floats2bfloat162_rn(acc[v] * inv, acc[v + 1] * inv);
-    if (p.lse != nullptr && lane == 0) p.lse[row] = (M + log2f(Lsum)) * kLn2;
+    for (int r = 0; r < GMAX; ++r) {
+        if (r < G) {
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) sm_o[warp][r][lane * VEC + v] = acc[r][v];
+            if (lane == 0) sm_ml[warp][r] = make_float2(m[r], l[r]);
+        }
+    }
+    __syncthreads();
+    for (int r = warp; r < G; r += WARPS) {
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) M = fmaxf(M, sm_ml[w][r].x);
+        float Lsum = 0.f, out[VEC];
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) out[v] = 0.f;
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) {
+            const float wt = exp2f(sm_ml[w][r].x - M);
+            Lsum += wt * sm_ml[w][r].y;
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) out[v] += wt * sm_o[w][r][lane * VEC + v];
+        }
+        const float inv = 1.f / Lsum;
+        __nv_bfloat16 *orow = obase + static_cast<size_t>(r) * D + lane * VEC;
+#pragma unroll
+        for (int v = 0; v < VEC; v += 2)
+            *reinterpret_cast<__nv_bfloat162 *>(orow + v) = __floats2bfloat162_rn(out[v] * inv, out[v + 1] * inv);
+        if (p.lse != nullptr && lane == 0)
+            p.lse[static_cast<size_t>(b) * p.Hq + kvh * G + r] = (M + log2f(Lsum)) * kLn2;
+    }
 }
 
 template <int D, int WARPS, int STAGES, bool HILO>
 size_t smem_bytes_for() {
-    // ring + 1 KB alignment slack + barriers + warp sums + prefix sums
-    return static_cast<size_t>(WARPS) * STAGES * (2 * kPageSize * D * 2) + 1024 + WARPS * STAGES * 2 * 8 + 32 * 4 +
-           (kMaxBatch + 1) * 4;
+    // ring + 1 KB alignment slack + barriers + plan + stage tags + warp sums + prefix sums
+    return static_cast<size_t>(WARPS) * STAGES * (2 * kPageSize * D * 2) + 1024 + WARPS * STAGES * 2 * 8 +
+           sizeof(Plan) + WARPS * STAGES * 4 + 32 * 4 + (kMaxBatch + 1) * 4;
 }
 
 template <typename F>
@@ -480,10 +664,15 @@ cudaError_t launch_decode_attn(const AttnVariant &v, const CUtensorMap &tm_k, co
 }
 
 cudaError_t launch_lse_merge(int head_dim, const AttnParams &p, cudaStream_t stream) {
-    const int rows = p.B * p.Hq;
-    const int blocks = (rows + 3) / 4;
-    if (head_dim == 128) lse_merge_kernel<128><<<blocks, 128, 0, stream>>>(p);
-    else lse_merge_kernel<64><<<blocks, 128, 0, stream>>>(p);
+    // few pairs (low decode concurrency) mean many partials per pair: give each pair more warps
+    const int pairs = p.B * p.Hkv;
+    if (head_dim == 128) {
+        if (pairs <= 1024) lse_merge_kernel<128, 8><<<pairs, 256, 0, stream>>>(p);
+        else lse_merge_kernel<128, 4><<<pairs, 128, 0, stream>>>(p);
+    } else {
+        if (pairs <= 1024) lse_merge_kernel<64, 8><<<pairs, 256, 0, stream>>>(p);
+        else lse_merge_kernel<64, 4><<<pairs, 128, 0, stream>>>(p);
+    }
     return cudaGetLastError();
 }
 

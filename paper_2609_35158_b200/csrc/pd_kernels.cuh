@@ -9,8 +9,14 @@ namespace pd {
 
 constexpr int kPageSize = 16;       // tokens per page
 constexpr int kMaxBatch = 4096;     // prefix sums of page counts live in shared memory
-constexpr int kPlanWords = 8;       // plan[0..1] total units (lo, hi), [2] pages per range, [3] ranges, [4] workers
-constexpr int kStatusWords = 4;     // status[0] code, [1] sequence, [2] detail
+constexpr int kMaxLevels = 12;      // levels of the range plan (geometrically shrinking ranges, then a tail level)
+// plan[0..1] total units (lo, hi), [2] levels, [3] ranges, [4] workers, then from word 8 one record of four
+// words per level (start lo, start hi, pages per range, index of its first range) plus a closing sentinel
+constexpr int kPlanHeaderWords = 8;
+constexpr int kPlanWords = kPlanHeaderWords + 4 * (kMaxLevels + 1);
+// status[0] code, [1] sequence, [2] detail, [3] unused, [4] next range to claim, [5] workers finished
+constexpr int kStatusWords = 8;
+constexpr int kSchedNext = 4, kSchedDone = 5;
 
 // Device-side fault codes latched in status[0] (first one wins).
 constexpr int kDevOk = 0;
@@ -32,9 +38,12 @@ struct AttnParams {
     int32_t B, Hq, Hkv, G, MP;
     int32_t num_pages;
     float scale_log2;           // sm_scale * log2(e)
-    int32_t split_pages;        // 0 = automatic
+    int32_t split_pages;        // 0 = automatic plan, > 0 = one level of ranges of that many pages
     int32_t max_ranges;         // partial slots available beyond one per (sequence, KV head)
     int32_t min_pages_auto;     // lower bound on pages per range in automatic mode
+    int32_t halving_levels;     // automatic plan: number of levels whose ranges halve the remaining fair share
+    int32_t tail_pages;         // automatic plan: pages per range of the last level
+    unsigned long long *trace;  // optional [workers][4] ns timestamps: kernel entry, first data, last data, exit
 };
 
 struct AppendParams {

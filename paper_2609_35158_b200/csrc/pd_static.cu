@@ -169,6 +169,8 @@ extern "C" int pd_decode_attn_static(const pd_config *cfg, const void *q, const 
     p.split_pages = 0;
     p.max_ranges = static_cast<int32_t>(workers);
     p.min_pages_auto = 4;
+    p.halving_levels = 0;  // one level of equal ranges, one per worker: the partial count stays within the fixed array
+    p.tail_pages = 16;
     if (pd::launch_decode_attn(variant, tm_k, tm_v, p, num_ctas, local.smem_bytes[vi], s) != cudaSuccess)
         return PD_ERR_CUDA;
     if (pd::launch_lse_merge(cfg->head_dim, p, s) != cudaSuccess) return PD_ERR_CUDA;

@@ -305,7 +305,7 @@ def test_full_size_configs_all_rows(config):
     with ctx_for(cache, w.num_q_heads) as ctx:
         out, lse = run_attn(ctx, cache, q, cache.ctx_lens, w.sm_scale)
         plan = ctx.pd.pd_last_plan(ctx.h)
-    assert plan["num_ranges"] <= plan["num_workers"]
+    assert plan["num_ranges"] >= plan["num_workers"]  # every worker warp has a first range of its own
     ref, ref_lse = oracle_on_cache(q, cache, lens, w.sm_scale)
     max_abs, rel = assert_parity(out, ref, f"config {config}")
     np.testing.assert_allclose(lse.cpu().numpy(), ref_lse, rtol=2e-5, atol=2e-5)

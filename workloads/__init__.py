@@ -130,7 +130,7 @@ def _big_randn_bf16(shape, g, device):
 def build_paged_cache(lens, num_kv_heads: int, head_dim: int, *, seed: int, device="cpu",
                       page_size: int = PAGE_SIZE, reserve_tokens: int = 0, preassign_reserve: bool = True,
                       slack: float = 1.0625, max_pages_per_seq: int | None = None,
-                      poison: bool = False) -> PagedCache:
+                      poison: bool = False, permute: bool = True) -> PagedCache:
     """A scattered paged cache holding ``lens[b]`` random tokens per sequence.
 
     The pool has ``ceil(slack * sum_b ceil((lens[b] + reserve_tokens) / P))`` pages.
@@ -141,7 +141,8 @@ def build_paged_cache(lens, num_kv_heads: int, head_dim: int, *, seed: int, devi
     ``ceil(L/P)`` are ignored by readers), otherwise they stay on the free list
     for a host allocator to hand out. With ``poison`` every slot that holds no
     token (tails of last pages, reserved and free pages) is bf16 NaN and every
-    unassigned table entry is -1.
+    unassigned table entry is -1. ``permute=False`` lays the pages out in logical order
+    (a contiguous cache), for experiments on the cost of scattering.
     """
     import torch
 
@@ -154,7 +155,7 @@ def build_paged_cache(lens, num_kv_heads: int, head_dim: int, *, seed: int, devi
     MP = int(max(1, pages_cap.max())) if max_pages_per_seq is None else int(max_pages_per_seq)
     assert MP >= pages_cap.max()
     rng = np.random.Generator(np.random.PCG64([int(seed), 0x9A6E5]))
-    perm = rng.permutation(NP).astype(np.int32)
+    perm = rng.permutation(NP).astype(np.int32) if permute else np.arange(NP, dtype=np.int32)
     table = np.full((B, MP), -1, dtype=np.int32)
     cur = 0
     for b in range(B):
