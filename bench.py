@@ -192,25 +192,33 @@ def run_cuda(args):
     torch.cuda.synchronize()
     code = pd.pd_device_status(ctx)
     assert code[0] == 0, f"device fault during warm-up: {code}"
-    befores = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
-    afters = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # The library's event hook brackets the split kernel of one step. Two event records cost several
+    # microseconds of stream time and switch off launch overlap for that step, so one step in sixteen is hooked.
+    hooked = [i for i in range(K) if i % 16 == min(8, K - 1)]
+    befores = {i: torch.cuda.Event(enable_timing=True) for i in hooked}
+    afters = {i: torch.cuda.Event(enable_timing=True) for i in hooked}
     sampler = ClockSampler(local_rank)
     launches0 = pd.pd_launch_count(ctx)
     barrier()
     sampler.start()
     t0.record()
     kv_bytes = 0
+    split_bytes = 0
     for i in range(K):
-        pd.pd_set_profile_events(ctx, befores[i], afters[i])
-        kv_bytes += device_step(W + i)
+        if i in befores:
+            pd.pd_set_profile_events(ctx, befores[i], afters[i])
+        step_bytes = device_step(W + i)
+        kv_bytes += step_bytes
+        if i in befores:
+            split_bytes += step_bytes
     t1.record()
     barrier()
     clocks = sampler.stop()
-    pd.pd_set_profile_events(ctx, None, None)
     launches = pd.pd_launch_count(ctx) - launches0
     local_ms = t0.elapsed_time(t1)
-    split_ms = float(np.mean([b.elapsed_time(a) for b, a in zip(befores, afters)]))
+    split_ms = float(np.mean([befores[i].elapsed_time(afters[i]) for i in hooked]))
+    split_bytes_per_launch = split_bytes / len(hooked)
     plan = pd.pd_last_plan(ctx)
     assert pd.pd_device_status(ctx)[0] == 0
     total_ms, total_bytes = aggregate_over_ranks(local_ms, float(kv_bytes), world, dev)
@@ -253,7 +261,7 @@ def run_cuda(args):
         cpu_baseline = time_oracle_once(w, cache, qs[0], lens)
 
     peak, peak_kind = measured_hbm_peak()
-    achieved = bytes_per_step_local / (split_ms * 1e-3) / 1e9
+    achieved = split_bytes_per_launch / (split_ms * 1e-3) / 1e9
     result = {
         "metric": METRIC, "value": round(value_gbs, 2), "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": round(total_ms / K, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -272,8 +280,9 @@ def run_cuda(args):
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "decode_attn_split_kernel", "achieved": round(achieved, 2), "peak": peak,
                      "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}",
-                     "traffic": None if NCU_TRAFFIC_RATIO is None else int(NCU_TRAFFIC_RATIO * bytes_per_step_local),
-                     "algorithmic_bytes_per_launch": int(bytes_per_step_local), "avg_launch_ms": round(split_ms, 5)},
+                     "traffic": None if NCU_TRAFFIC_RATIO is None else int(NCU_TRAFFIC_RATIO * split_bytes_per_launch),
+                     "algorithmic_bytes_per_launch": int(split_bytes_per_launch), "avg_launch_ms": round(split_ms, 5),
+                     "timed": f"CUDA events recorded by the library around the split kernel, {len(hooked)} of the {K} timed launches"},
         "cpu_baseline": cpu_baseline,
     }
     pd.pd_destroy(ctx)

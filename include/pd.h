@@ -157,8 +157,8 @@ int pd_decode_step_host(pd_ctx *ctx, const void *q_host, const void *k_new_host,
  * The first call on each device resolves the array's device address and sets
  * the kernel's shared-memory attribute; make that first call outside any CUDA
  * stream capture. All calls on a device share the one array, which keeps the
- * previous call's contents (the function clears the status latch itself, the
- * only word that must start at zero): two calls whose kernels may overlap on
+ * previous call's contents (the function itself clears the few words that must
+ * start at zero: the status latch and the range-claim counters): two calls whose kernels may overlap on
  * the GPU - different streams, or concurrent host threads - race on it. Issue
  * them on one stream or order them with events. Out-of-range page ids are
  * clamped to page 0 as in pd_decode_attn but are not reported, since there is
@@ -177,11 +177,14 @@ int pd_decode_attn_static(const pd_config *cfg, const void *q, const void *k_pag
 int pd_device_status(pd_ctx *ctx, void *stream, int32_t *code, int32_t *seq, int32_t *detail);
 
 /*
- * Timing hook for benchmarks: after this call every pd_decode_attn of this
- * context records `before` on its stream just ahead of the split kernel and
- * `after` right behind it (both cudaEvent_t passed as void*, owned by the
- * caller, who must keep them alive until the work has run). Passing two NULLs
- * switches the hook off. The events bracket the split kernel only, not the merge.
+ * Timing hook for benchmarks: the NEXT pd_decode_attn of this context records
+ * `before` on its stream just ahead of the split kernel and `after` right behind
+ * it (both cudaEvent_t passed as void*, owned by the caller, who must keep them
+ * alive until the work has run), then the hook clears itself. That call launches
+ * its kernels without programmatic overlap, so the events bracket the split
+ * kernel alone, not the merge. Two event records cost several microseconds of
+ * stream time: hook a sample of the steps, not all of them. Passing two NULLs
+ * cancels a pending hook.
  */
 int pd_set_profile_events(pd_ctx *ctx, void *before, void *after);
 

@@ -41,6 +41,7 @@ struct pd_ctx {
     int min_pages_auto = 1;
     int halving_levels = 0;
     int tail_pages = 16;
+    int pdl = 1;
     size_t slots = 0;
     // device workspace (one allocation)
     void *workspace = nullptr;
@@ -166,6 +167,7 @@ int pd_create(const pd_config *cfg, pd_ctx **out) {
     ctx->min_pages_auto = env_int("PD_TUNE_MIN_PAGES", 4);
     ctx->halving_levels = env_int("PD_TUNE_LEVELS", 6);
     ctx->tail_pages = env_int("PD_TUNE_TAIL", 16);
+    ctx->pdl = env_int("PD_TUNE_PDL", 1);
     if (ctx->halving_levels < 0 || ctx->halving_levels > pd::kMaxLevels - 2 || ctx->tail_pages < 1) {
         delete ctx;
         return PD_ERR_INVALID_ARG;
@@ -261,6 +263,7 @@ int pd_kv_append(pd_ctx *ctx, const void *k_new, const void *v_new, void *k_page
     p.MP = ctx->cfg.max_pages_per_seq;
     p.num_pages = static_cast<int32_t>(ctx->cfg.num_pages);
     p.advance = (call_flags & PD_APPEND_NO_ADVANCE) ? 0 : 1;
+    p.pdl = ctx->pdl;
     const cudaError_t err = pd::launch_kv_append(p, static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "kv_append launch", err);
     ctx->launches += 1;
@@ -310,12 +313,18 @@ int pd_decode_attn(pd_ctx *ctx, const void *q, const void *k_pages, const void *
     p.min_pages_auto = ctx->min_pages_auto;
     p.halving_levels = ctx->halving_levels;
     p.tail_pages = ctx->tail_pages;
+    const bool hooked = ctx->ev_before != nullptr;
+    p.pdl = hooked ? 0 : ctx->pdl;  // timing events must bracket the split kernel alone: no overlap with neighbours
     p.trace = ctx->trace;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (ctx->ev_before != nullptr) cudaEventRecord(ctx->ev_before, s);
+    if (hooked) cudaEventRecord(ctx->ev_before, s);
     cudaError_t err = pd::launch_decode_attn(ctx->variant, ctx->tm_k, ctx->tm_v, p, ctx->num_ctas, ctx->smem_bytes, s);
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "decode_attn_split launch", err);
-    if (ctx->ev_after != nullptr) cudaEventRecord(ctx->ev_after, s);
+    if (hooked) {
+        cudaEventRecord(ctx->ev_after, s);
+        ctx->ev_before = nullptr;  // one-shot
+        ctx->ev_after = nullptr;
+    }
     err = pd::launch_lse_merge(ctx->cfg.head_dim, p, s);
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "lse_merge launch", err);
     ctx->launches += 2;

@@ -230,6 +230,7 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     unsigned long long t_first = 0ull, t_last = 0ull;
 
     // ---- prologue (whole CTA): barriers, page prefix sums, the plan
+    launch_dependents();  // the merge kernel may take its place on the SMs; it waits for this grid to finish
     if (lane == 0) {
         for (int s = 0; s < STAGES * 2; ++s) mbar_init(smem_u32(bars + (warp * STAGES * 2 + s)), 1);
         mbar_init_fence();
@@ -238,6 +239,7 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         prefetch_tensormap(&tm_k);
         prefetch_tensormap(&tm_v);
     }
+    grid_dependency_wait();  // everything above is independent of the previous kernel's writes
     scan_pages<THREADS>(p, cum, warp_sums);
 
     const int n_workers = gridDim.x * WARPS;
@@ -525,100 +527,103 @@ __device__ __forceinline__ long long range_of_unit(const int32_t *plan, long lon
     return rec[4 * l + 3] + (x - start_of(l)) / rec[4 * l + 2];
 }
 
-// One CTA per (sequence, KV head): its warps take the pair's partials round-robin, each keeping a
-// running (max, sum, output) per query head of the group; the per-warp results are then combined
-// through shared memory in warp order. The order of operations is fixed, so reruns are bit-identical.
+// One CTA per (sequence, query head): its warps take the row's partials round-robin, eight loads in
+// flight each, keeping a running (max, sum, output); the per-warp results are then combined through
+// shared memory in warp order. The order of operations is fixed, so reruns are bit-identical.
 template <int D, int WARPS>
 __global__ void __launch_bounds__(WARPS * 32) lse_merge_kernel(const AttnParams p) {
     constexpr int VEC = D / 32;
-    constexpr int GMAX = 8;
-    __shared__ float sm_o[WARPS][GMAX][D];
-    __shared__ float2 sm_ml[WARPS][GMAX];
+    constexpr int UNROLL = 8;
+    __shared__ float sm_o[WARPS][D];
+    __shared__ float2 sm_ml[WARPS];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int pair = blockIdx.x;
-    const int b = pair / p.Hkv, kvh = pair - b * p.Hkv;
+    const int row = blockIdx.x;
+    grid_dependency_wait();  // partials, prefix sums and the plan come from the split kernel
+    launch_dependents();
+    const int b = row / p.Hq, h = row - b * p.Hq;
     const int G = p.G;
+    const int kvh = h / G, r = h - kvh * G;
     const int c0 = p.cum_pages[b], np = p.cum_pages[b + 1] - c0;
-    __nv_bfloat16 *obase = p.out + (static_cast<size_t>(b) * p.Hq + kvh * G) * D;
-    if (np == 0) {  // empty context: zero rows, lse = -inf
-        for (int i = threadIdx.x; i < G * D; i += WARPS * 32) obase[i] = __float2bfloat16(0.f);
-        if (p.lse != nullptr && threadIdx.x < G) p.lse[static_cast<size_t>(b) * p.Hq + kvh * G + threadIdx.x] = -INFINITY;
+    __nv_bfloat16 *orow = p.out + static_cast<size_t>(row) * D + lane * VEC;
+    if (np == 0) {  // empty context: zero row, lse = -inf
+        if (warp == 0) {
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) orow[v] = __float2bfloat16(0.f);
+            if (p.lse != nullptr && lane == 0) p.lse[row] = -INFINITY;
+        }
         return;
     }
     const long long u0 = static_cast<long long>(p.Hkv) * c0 + static_cast<long long>(kvh) * np;
     const long long first = range_of_unit(p.plan, u0), last = range_of_unit(p.plan, u0 + np - 1);
     if (first == last) return;  // written directly by the split kernel
     const int n = static_cast<int>(last - first) + 1;
-    const size_t slot0 = static_cast<size_t>(first) + pair;
+    const size_t slot0 = static_cast<size_t>(first) + static_cast<size_t>(b) * p.Hkv + kvh;
 
-    float m[GMAX], l[GMAX], acc[GMAX][VEC];
+    float m = -INFINITY, l = 0.f, acc[VEC];
 #pragma unroll
-    for (int r = 0; r < GMAX; ++r) {
-        m[r] = -INFINITY;
-        l[r] = 0.f;
+    for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
+    for (int i0 = warp; i0 < n; i0 += WARPS * UNROLL) {
+        float2 ml[UNROLL];
+        float o[UNROLL][VEC];
 #pragma unroll
-        for (int v = 0; v < VEC; ++v) acc[r][v] = 0.f;
-    }
-    for (int i = warp; i < n; i += WARPS) {
-        const float2 *ml_src = p.part_ml + (slot0 + i) * G;
-        const float *o_src = p.part_o + (slot0 + i) * G * D + lane * VEC;
-        float2 ml[GMAX];
-        float o[GMAX][VEC];
-#pragma unroll
-        for (int r = 0; r < GMAX; ++r) {
-            if (r < G) {
-                ml[r] = ml_src[r];
+        for (int u = 0; u < UNROLL; ++u) {
+            const int i = i0 + u * WARPS;
+            if (i < n) {
+                const size_t rec = (slot0 + i) * G + r;
+                ml[u] = p.part_ml[rec];
+                const float *src = p.part_o + rec * D + lane * VEC;
                 if (VEC == 4) {
-                    const float4 t = *reinterpret_cast<const float4 *>(o_src + r * D);
-                    o[r][0] = t.x; o[r][1] = t.y; o[r][VEC - 2] = t.z; o[r][VEC - 1] = t.w;
+                    const float4 t = *reinterpret_cast<const float4 *>(src);
+                    o[u][0] = t.x; o[u][1] = t.y; o[u][VEC - 2] = t.z; o[u][VEC - 1] = t.w;
                 } else {
-                    const float2 t = *reinterpret_cast<const float2 *>(o_src + r * D);
-                    o[r][0] = t.x; o[r][1] = t.y;
+                    const float2 t = *reinterpret_cast<const float2 *>(src);
+                    o[u][0] = t.x; o[u][1] = t.y;
                 }
+            } else {
+                ml[u] = make_float2(-INFINITY, 0.f);
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) o[u][v] = 0.f;
             }
         }
+        float m_new = m;
 #pragma unroll
-        for (int r = 0; r < GMAX; ++r) {
-            if (r < G) {
-                const float m_new = fmaxf(m[r], ml[r].x);
-                const float a = exp2f(m[r] - m_new), w = exp2f(ml[r].x - m_new);
-                l[r] = l[r] * a + w * ml[r].y;
+        for (int u = 0; u < UNROLL; ++u) m_new = fmaxf(m_new, ml[u].x);
+        const float a = exp2f(m - m_new);  // m_new is finite: the first record of every batch exists
+        l *= a;
 #pragma unroll
-                for (int v = 0; v < VEC; ++v) acc[r][v] = acc[r][v] * a + w * o[r][v];
-                m[r] = m_new;
-            }
+        for (int v = 0; v < VEC; ++v) acc[v] *= a;
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const float w = exp2f(ml[u].x - m_new);
+            l += w * ml[u].y;
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) acc[v] += w * o[u][v];
         }
+        m = m_new;
     }
 #pragma unroll
-    for (int r = 0; r < GMAX; ++r) {
-        if (r < G) {
-#pragma unroll
-            for (int v = 0; v < VEC; ++v) sm_o[warp][r][lane * VEC + v] = acc[r][v];
-            if (lane == 0) sm_ml[warp][r] = make_float2(m[r], l[r]);
-        }
-    }
+    for (int v = 0; v < VEC; ++v) sm_o[warp][lane * VEC + v] = acc[v];
+    if (lane == 0) sm_ml[warp] = make_float2(m, l);
     __syncthreads();
-    for (int r = warp; r < G; r += WARPS) {
+    if (warp == 0) {
         float M = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < WARPS; ++w) M = fmaxf(M, sm_ml[w][r].x);
+        for (int w = 0; w < WARPS; ++w) M = fmaxf(M, sm_ml[w].x);
         float Lsum = 0.f, out[VEC];
 #pragma unroll
         for (int v = 0; v < VEC; ++v) out[v] = 0.f;
 #pragma unroll
         for (int w = 0; w < WARPS; ++w) {
-            const float wt = exp2f(sm_ml[w][r].x - M);
-            Lsum += wt * sm_ml[w][r].y;
+            const float wt = exp2f(sm_ml[w].x - M);  // warps without records carry m = -inf, weight 0
+            Lsum += wt * sm_ml[w].y;
 #pragma unroll
-            for (int v = 0; v < VEC; ++v) out[v] += wt * sm_o[w][r][lane * VEC + v];
+            for (int v = 0; v < VEC; ++v) out[v] += wt * sm_o[w][lane * VEC + v];
         }
         const float inv = 1.f / Lsum;
-        __nv_bfloat16 *orow = obase + static_cast<size_t>(r) * D + lane * VEC;
 #pragma unroll
         for (int v = 0; v < VEC; v += 2)
             *reinterpret_cast<__nv_bfloat162 *>(orow + v) = __floats2bfloat162_rn(out[v] * inv, out[v + 1] * inv);
-        if (p.lse != nullptr && lane == 0)
-            p.lse[static_cast<size_t>(b) * p.Hq + kvh * G + r] = (M + log2f(Lsum)) * kLn2;
+        if (p.lse != nullptr && lane == 0) p.lse[row] = (M + log2f(Lsum)) * kLn2;
     }
 }
 
@@ -658,22 +663,20 @@ cudaError_t prepare_decode_attn(const AttnVariant &v, size_t *smem_bytes) {
 cudaError_t launch_decode_attn(const AttnVariant &v, const CUtensorMap &tm_k, const CUtensorMap &tm_v,
                                const AttnParams &p, int num_ctas, size_t smem_bytes, cudaStream_t stream) {
     return dispatch(v, [&](auto kernel, size_t) {
-        kernel<<<num_ctas, v.warps * 32, smem_bytes, stream>>>(tm_k, tm_v, p);
-        return cudaGetLastError();
+        return launch_pdl(kernel, dim3(num_ctas), dim3(v.warps * 32), smem_bytes, stream, p.pdl != 0, tm_k, tm_v, p);
     });
 }
 
 cudaError_t launch_lse_merge(int head_dim, const AttnParams &p, cudaStream_t stream) {
-    // few pairs (low decode concurrency) mean many partials per pair: give each pair more warps
-    const int pairs = p.B * p.Hkv;
+    // few rows (low decode concurrency) mean many partials per row: give each row more warps
+    const int rows = p.B * p.Hq;
+    const bool pdl = p.pdl != 0;
     if (head_dim == 128) {
-        if (pairs <= 1024) lse_merge_kernel<128, 8><<<pairs, 256, 0, stream>>>(p);
-        else lse_merge_kernel<128, 4><<<pairs, 128, 0, stream>>>(p);
-    } else {
-        if (pairs <= 1024) lse_merge_kernel<64, 8><<<pairs, 256, 0, stream>>>(p);
-        else lse_merge_kernel<64, 4><<<pairs, 128, 0, stream>>>(p);
+        if (rows <= 4096) return launch_pdl(lse_merge_kernel<128, 8>, dim3(rows), dim3(256), 0, stream, pdl, p);
+        return launch_pdl(lse_merge_kernel<128, 2>, dim3(rows), dim3(64), 0, stream, pdl, p);
     }
-    return cudaGetLastError();
+    if (rows <= 4096) return launch_pdl(lse_merge_kernel<64, 8>, dim3(rows), dim3(256), 0, stream, pdl, p);
+    return launch_pdl(lse_merge_kernel<64, 2>, dim3(rows), dim3(64), 0, stream, pdl, p);
 }
 
 }  // namespace pd

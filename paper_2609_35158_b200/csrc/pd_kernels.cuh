@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 namespace pd {
 
 constexpr int kPageSize = 16;       // tokens per page
@@ -43,6 +45,7 @@ struct AttnParams {
     int32_t min_pages_auto;     // lower bound on pages per range in automatic mode
     int32_t halving_levels;     // automatic plan: number of levels whose ranges halve the remaining fair share
     int32_t tail_pages;         // automatic plan: pages per range of the last level
+    int32_t pdl;                // launch with programmatic stream serialization
     unsigned long long *trace;  // optional [workers][4] ns timestamps: kernel entry, first data, last data, exit
 };
 
@@ -55,12 +58,32 @@ struct AppendParams {
     int32_t B, Hkv, D, MP;
     int32_t num_pages;
     int32_t advance;
+    int32_t pdl;  // launch with programmatic stream serialization
 };
 
 // Shape of one compiled variant of the split kernel.
 struct AttnVariant {
     int head_dim, warps, stages, hilo;
 };
+
+// Launches `kernel` so that it may overlap the tail of the previous kernel in the stream (programmatic
+// dependent launch); every kernel of this library waits on the grid dependency before its first read
+// of global memory, so this is safe after any predecessor.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool pdl,
+                       Args &&...args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // Launchers (defined next to their kernels). They return the CUDA error of the launch.
 cudaError_t launch_kv_append(const AppendParams &p, cudaStream_t stream);

@@ -5,6 +5,7 @@
 // chunk of one KV head's K or V row. The destination slot follows from the
 // sequence's current length and its page-table row.
 #include "pd_kernels.cuh"
+#include "pd_ptx.cuh"
 
 namespace pd {
 
@@ -12,6 +13,8 @@ namespace {
 
 __global__ void __launch_bounds__(256) kv_append_kernel(const AppendParams p) {
     const int b = blockIdx.x;
+    grid_dependency_wait();  // the previous step's kernels still read the pools and the lengths
+    launch_dependents();
     const int pos = p.ctx_lens[b];
     __syncthreads();  // everyone has read the length before thread 0 advances it
     const int logical = pos / kPageSize, slot = pos % kPageSize;
@@ -46,8 +49,7 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const AppendParams p) {
 
 cudaError_t launch_kv_append(const AppendParams &p, cudaStream_t stream) {
     if (p.B == 0) return cudaSuccess;
-    kv_append_kernel<<<p.B, 256, 0, stream>>>(p);
-    return cudaGetLastError();
+    return launch_pdl(kv_append_kernel, dim3(p.B), dim3(256), 0, stream, p.pdl != 0, p);
 }
 
 }  // namespace pd

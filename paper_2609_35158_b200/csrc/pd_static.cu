@@ -144,7 +144,7 @@ extern "C" int pd_decode_attn_static(const pd_config *cfg, const void *q, const 
     if (encode_map(*cfg, k_pages, &tm_k) != PD_OK || encode_map(*cfg, v_pages, &tm_v) != PD_OK) return PD_ERR_CUDA;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // the array keeps the previous call's contents; the status latch is the one thing that must start at zero
+    // the array keeps the previous call's contents; the status latch and the range-claim counters must start at zero
     if (cudaMemsetAsync(local.scratch + off_status, 0, pd::kStatusWords * sizeof(int32_t), s) != cudaSuccess)
         return PD_ERR_CUDA;
 
