@@ -29,10 +29,15 @@
 // 128-byte swizzle, so ldmatrix reads are bank-conflict free. K and V of a page
 // complete on separate mbarriers.
 //
-// Math. The query group (g <= 8 heads sharing the KV head) is the M dimension
-// of mma.sync.m16n8k16 (rows g..15 are zero): S = Q K^T per page, online
-// softmax in fp32 in log2 units with a lazy rescale, then O += P V with P split
-// into a bf16 high and low part (two MMAs) so that P carries ~16 mantissa bits.
+// Math. Tokens are the M dimension of mma.sync.m16n8k16 and the query group
+// (g <= 8 heads sharing the KV head, zero-padded to 8) is N, so no MMA row is
+// wasted: S^T = K Q^T (one page = 16 tokens x 8 heads, 8 MMAs at D = 128), then
+// O^T += V^T P^T (8 more). Softmax runs in fp32 in log2 units; the running max
+// of a head is refreshed only when a logit exceeds it by more than 8 (a factor
+// 256 of headroom), so the steady state needs one warp vote per page and no
+// shuffles. P is split into a bf16 high and low part (two MMAs) so that it
+// carries ~16 mantissa bits; movmatrix turns the S^T fragments into the B
+// operand of the second product.
 #include "pd_kernels.cuh"
 #include "pd_ptx.cuh"
 
@@ -41,6 +46,7 @@ namespace pd {
 namespace {
 
 constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleSlack = 8.f;  // log2 units a logit may exceed the running max before a rescale
 constexpr int kClaimAhead = 2;  // pages left to issue in a range when the next range is claimed
 
 struct Cursor {
@@ -213,7 +219,7 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     constexpr int TILE_BYTES = HALVES * HALF_BYTES;
     constexpr int STAGE_BYTES = 2 * TILE_BYTES;  // K tile then V tile
     constexpr int KSTEPS = D / 16;
-    constexpr int NTILES = D / 8;
+    constexpr int MTILES = D / 16;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -270,15 +276,15 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     const uint32_t bar0 = smem_u32(bars + warp * STAGES * 2);
     int32_t *my_stage_range = stage_range + warp * STAGES;
     const uint64_t policy = l2_policy_evict_first();
-    const int quad_row = lane >> 2;  // query head inside the group handled by this lane
-    const int quad_col = (lane & 3) * 2;
+    const int quad_row = lane >> 2;        // B-fragment column of this lane: the query head whose Q it holds
+    const int quad_col = (lane & 3) * 2;   // accumulator columns of this lane: heads quad_col and quad_col + 1
     const int G = p.G;
     // ldmatrix lane addressing inside a tile (row = token, 16-byte chunk index swizzled by row & 7)
     const int mat = lane >> 3, r8 = lane & 7;
-    const uint32_t k_row_off = (((mat >> 1) * 8 + r8) * 128);
-    const int k_sel = mat & 1;
-    const uint32_t v_row_off = (((mat & 1) * 8 + r8) * 128);
-    const int v_sel = mat >> 1;
+    const uint32_t k_row_off = (((mat & 1) * 8 + r8) * 128);   // A operand: K tile, tokens x d
+    const int k_sel = mat >> 1;
+    const uint32_t v_row_off = (((mat >> 1) * 8 + r8) * 128);  // A operand: V tile read transposed, d x tokens
+    const int v_sel = mat & 1;
 
     PageIdCache pt;
     pt.b = -1; pt.blk = -1; pt.val = -1; pt.nval = -1;
@@ -352,9 +358,9 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     uint32_t stage = 0, parity = 0;  // ring position of the next page to consume
     bool alive = true, seg_open = false;
     int seg_page0 = 0, L = 0;
-    uint32_t qa[KSTEPS][2];
-    float O[NTILES][4];
-    float m_run = -INFINITY, l_run = 0.f;
+    uint32_t qb[KSTEPS][2];     // Q^T as the B operand: head quad_row, d = 16 kk + quad_col (+1), and +8
+    float O[MTILES][4];          // O^T: rows d = 16 j + quad_row (+8), columns heads quad_col, quad_col + 1
+    float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;  // per head (a = quad_col, b = quad_col + 1)
 
     while (inflight > 0) {
         if (c_left == 0) {  // first page of a range
@@ -371,17 +377,17 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
 #pragma unroll
             for (int kk = 0; kk < KSTEPS; ++kk) {
                 if (quad_row < G) {
-                    qa[kk][0] = __ldg(reinterpret_cast<const uint32_t *>(qrow + kk * 16 + quad_col));
-                    qa[kk][1] = __ldg(reinterpret_cast<const uint32_t *>(qrow + kk * 16 + 8 + quad_col));
+                    qb[kk][0] = __ldg(reinterpret_cast<const uint32_t *>(qrow + kk * 16 + quad_col));
+                    qb[kk][1] = __ldg(reinterpret_cast<const uint32_t *>(qrow + kk * 16 + 8 + quad_col));
                 } else {
-                    qa[kk][0] = 0u;
-                    qa[kk][1] = 0u;
+                    qb[kk][0] = 0u;
+                    qb[kk][1] = 0u;
                 }
             }
 #pragma unroll
-            for (int j = 0; j < NTILES; ++j) { O[j][0] = 0.f; O[j][1] = 0.f; O[j][2] = 0.f; O[j][3] = 0.f; }
-            m_run = -INFINITY;
-            l_run = 0.f;
+            for (int j = 0; j < MTILES; ++j) { O[j][0] = 0.f; O[j][1] = 0.f; O[j][2] = 0.f; O[j][3] = 0.f; }
+            m_a = -INFINITY; m_b = -INFINITY;
+            l_a = 0.f; l_b = 0.f;
         }
 
         const uint32_t kbase = ring + stage * STAGE_BYTES;
@@ -395,52 +401,55 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
             if (t_first == 0ull) t_first = t_last;
         }
 
-        // S = Q K^T for 16 tokens: two 8-token column tiles, two accumulators each
-        float Sa[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-        float Sb[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        // S^T = K Q^T for the 16 tokens of the page (two accumulators shorten the dependent chain)
+        float Se[4] = {0.f, 0.f, 0.f, 0.f}, So[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int kk = 0; kk < KSTEPS; ++kk) {
-            uint32_t b0, b1, b2, b3;
-            ldmatrix_x4(b0, b1, b2, b3,
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4(a0, a1, a2, a3,
                         kbase + (kk >> 2) * HALF_BYTES + k_row_off + ((((kk & 3) * 2 + k_sel) ^ r8) << 4));
-            if (kk & 1) {
-                mma_bf16_16816(Sb[0], qa[kk][0], 0u, qa[kk][1], 0u, b0, b1);
-                mma_bf16_16816(Sb[1], qa[kk][0], 0u, qa[kk][1], 0u, b2, b3);
-            } else {
-                mma_bf16_16816(Sa[0], qa[kk][0], 0u, qa[kk][1], 0u, b0, b1);
-                mma_bf16_16816(Sa[1], qa[kk][0], 0u, qa[kk][1], 0u, b2, b3);
-            }
+            if (kk & 1) mma_bf16_16816(So, a0, a1, a2, a3, qb[kk][0], qb[kk][1]);
+            else mma_bf16_16816(Se, a0, a1, a2, a3, qb[kk][0], qb[kk][1]);
         }
-        // this lane: row quad_row, tokens quad_col, +1, +8, +9 (log2 units)
-        float s0 = (Sa[0][0] + Sb[0][0]) * p.scale_log2, s1 = (Sa[0][1] + Sb[0][1]) * p.scale_log2;
-        float s2 = (Sa[1][0] + Sb[1][0]) * p.scale_log2, s3 = (Sa[1][1] + Sb[1][1]) * p.scale_log2;
+        // this lane: tokens quad_row and quad_row + 8, heads quad_col (a) and quad_col + 1 (b); log2 units
+        float s0 = (Se[0] + So[0]) * p.scale_log2, s1 = (Se[1] + So[1]) * p.scale_log2;
+        float s2 = (Se[2] + So[2]) * p.scale_log2, s3 = (Se[3] + So[3]) * p.scale_log2;
         if (valid < kPageSize) {  // last page of the context: mask, never multiply
-            if (quad_col >= valid) s0 = -INFINITY;
-            if (quad_col + 1 >= valid) s1 = -INFINITY;
-            if (quad_col + 8 >= valid) s2 = -INFINITY;
-            if (quad_col + 9 >= valid) s3 = -INFINITY;
+            if (quad_row >= valid) { s0 = -INFINITY; s1 = -INFINITY; }
+            if (quad_row + 8 >= valid) { s2 = -INFINITY; s3 = -INFINITY; }
         }
-        float mx = fmaxf(fmaxf(s0, s1), fmaxf(s2, s3));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        const float m_new = fmaxf(m_run, mx);
-        if (__any_sync(0xffffffffu, m_new > m_run)) {  // lazy rescale of the running state
-            const float alpha = fast_exp2(m_run - m_new);
-            l_run *= alpha;
+        float mx_a = fmaxf(s0, s2), mx_b = fmaxf(s1, s3);
+        if (__any_sync(0xffffffffu, mx_a > m_a + kRescaleSlack || mx_b > m_b + kRescaleSlack)) {
+            // some logit left the headroom of a running max: refresh both maxima over the page, rescale
 #pragma unroll
-            for (int j = 0; j < NTILES; ++j) { O[j][0] *= alpha; O[j][1] *= alpha; }
-            m_run = m_new;
+            for (int o = 4; o < 32; o <<= 1) {
+                mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, o));
+                mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, o));
+            }
+            const float new_a = fmaxf(m_a, mx_a), new_b = fmaxf(m_b, mx_b);
+            const float alpha_a = fast_exp2(m_a - new_a), alpha_b = fast_exp2(m_b - new_b);
+            l_a *= alpha_a;
+            l_b *= alpha_b;
+#pragma unroll
+            for (int j = 0; j < MTILES; ++j) {
+                O[j][0] *= alpha_a; O[j][2] *= alpha_a;
+                O[j][1] *= alpha_b; O[j][3] *= alpha_b;
+            }
+            m_a = new_a;
+            m_b = new_b;
         }
-        const float p0 = fast_exp2(s0 - m_run), p1 = fast_exp2(s1 - m_run);
-        const float p2 = fast_exp2(s2 - m_run), p3 = fast_exp2(s3 - m_run);
-        l_run += (p0 + p1) + (p2 + p3);
+        const float p0 = fast_exp2(s0 - m_a), p1 = fast_exp2(s1 - m_b);
+        const float p2 = fast_exp2(s2 - m_a), p3 = fast_exp2(s3 - m_b);
+        l_a += p0 + p2;
+        l_b += p1 + p3;
+        // P^T as the B operand: transpose the (token x head) fragments to (head x token)
         const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1), h23 = __floats2bfloat162_rn(p2, p3);
-        const uint32_t pa0 = *reinterpret_cast<const uint32_t *>(&h01);
-        const uint32_t pa2 = *reinterpret_cast<const uint32_t *>(&h23);
-        uint32_t pl0 = 0u, pl2 = 0u;
+        const uint32_t pb0 = movmatrix_trans(*reinterpret_cast<const uint32_t *>(&h01));
+        const uint32_t pb1 = movmatrix_trans(*reinterpret_cast<const uint32_t *>(&h23));
+        uint32_t pl0 = 0u, pl1 = 0u;
         if (HILO) {
-            pl0 = pack_bf16x2(p0 - __low2float(h01), p1 - __high2float(h01));
-            pl2 = pack_bf16x2(p2 - __low2float(h23), p3 - __high2float(h23));
+            pl0 = movmatrix_trans(pack_bf16x2(p0 - __low2float(h01), p1 - __high2float(h01)));
+            pl1 = movmatrix_trans(pack_bf16x2(p2 - __low2float(h23), p3 - __high2float(h23)));
         }
 
         if (!__all_sync(0xffffffffu, mbar_wait(bv, parity))) { alive = false; break; }
@@ -451,18 +460,14 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                     st_shared_zero16(vbase + (lane >> 3) * HALF_BYTES + row * 128 + (lane & 7) * 16);
             __syncwarp();
         }
-        // O += P V : 16 tokens (k) x D columns
+        // O^T += V^T P^T : D rows (16 per MMA) x 8 heads, contraction over the 16 tokens
 #pragma unroll
-        for (int j = 0; j < NTILES / 2; ++j) {
-            uint32_t v0, v1, v2, v3;
-            ldmatrix_x4_trans(v0, v1, v2, v3,
+        for (int j = 0; j < MTILES; ++j) {
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4_trans(a0, a1, a2, a3,
                               vbase + (j >> 2) * HALF_BYTES + v_row_off + ((((j & 3) * 2 + v_sel) ^ r8) << 4));
-            mma_bf16_16816(O[2 * j], pa0, 0u, pa2, 0u, v0, v1);
-            mma_bf16_16816(O[2 * j + 1], pa0, 0u, pa2, 0u, v2, v3);
-            if (HILO) {
-                mma_bf16_16816(O[2 * j], pl0, 0u, pl2, 0u, v0, v1);
-                mma_bf16_16816(O[2 * j + 1], pl0, 0u, pl2, 0u, v2, v3);
-            }
+            mma_bf16_16816(O[j], a0, a1, a2, a3, pb0, pb1);
+            if (HILO) mma_bf16_16816(O[j], a0, a1, a2, a3, pl0, pl1);
         }
         __syncwarp();  // every lane has read this stage
         if (valid < kPageSize) fence_proxy_async();  // generic-proxy stores before the next TMA write
@@ -474,26 +479,42 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         --c_left;
         const bool pair_end = cons.page + 1 == cons.np;
         if (c_left == 0 || pair_end) {
-            float l_tot = l_run + __shfl_xor_sync(0xffffffffu, l_run, 1);
-            l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 2);
-            if (quad_row < G) {
-                const int h = cons.kvh * G + quad_row;
-                if (seg_page0 == 0 && pair_end) {
-                    const float inv = 1.f / l_tot;
-                    __nv_bfloat16 *orow = p.out + (static_cast<size_t>(cons.b) * p.Hq + h) * D + quad_col;
 #pragma unroll
-                    for (int j = 0; j < NTILES; ++j)
-                        *reinterpret_cast<__nv_bfloat162 *>(orow + j * 8) =
-                            __floats2bfloat162_rn(O[j][0] * inv, O[j][1] * inv);
-                    if (p.lse != nullptr && (lane & 3) == 0)
-                        p.lse[static_cast<size_t>(cons.b) * p.Hq + h] = (m_run + log2f(l_tot)) * kLn2;
-                } else {
-                    const size_t slot = static_cast<size_t>(c_rid) + static_cast<size_t>(cons.b) * p.Hkv + cons.kvh;
-                    float *orow = p.part_o + (slot * G + quad_row) * D + quad_col;
+            for (int o = 4; o < 32; o <<= 1) {
+                l_a += __shfl_xor_sync(0xffffffffu, l_a, o);
+                l_b += __shfl_xor_sync(0xffffffffu, l_b, o);
+            }
+            const size_t row0 = static_cast<size_t>(cons.b) * p.Hq + cons.kvh * G + quad_col;
+            const bool has_a = quad_col < G, has_b = quad_col + 1 < G;
+            if (seg_page0 == 0 && pair_end) {
+                const float inv_a = 1.f / l_a, inv_b = 1.f / l_b;
+                __nv_bfloat16 *oa = p.out + row0 * D + quad_row, *ob = oa + D;
 #pragma unroll
-                    for (int j = 0; j < NTILES; ++j)
-                        *reinterpret_cast<float2 *>(orow + j * 8) = make_float2(O[j][0], O[j][1]);
-                    if ((lane & 3) == 0) p.part_ml[slot * G + quad_row] = make_float2(m_run, l_tot);
+                for (int j = 0; j < MTILES; ++j) {
+                    if (has_a) {
+                        oa[16 * j] = __float2bfloat16(O[j][0] * inv_a);
+                        oa[16 * j + 8] = __float2bfloat16(O[j][2] * inv_a);
+                    }
+                    if (has_b) {
+                        ob[16 * j] = __float2bfloat16(O[j][1] * inv_b);
+                        ob[16 * j + 8] = __float2bfloat16(O[j][3] * inv_b);
+                    }
+                }
+                if (p.lse != nullptr && quad_row == 0) {
+                    if (has_a) p.lse[row0] = (m_a + log2f(l_a)) * kLn2;
+                    if (has_b) p.lse[row0 + 1] = (m_b + log2f(l_b)) * kLn2;
+                }
+            } else {
+                const size_t slot = static_cast<size_t>(c_rid) + static_cast<size_t>(cons.b) * p.Hkv + cons.kvh;
+                float *oa = p.part_o + (slot * G + quad_col) * D + quad_row, *ob = oa + D;
+#pragma unroll
+                for (int j = 0; j < MTILES; ++j) {
+                    if (has_a) { oa[16 * j] = O[j][0]; oa[16 * j + 8] = O[j][2]; }
+                    if (has_b) { ob[16 * j] = O[j][1]; ob[16 * j + 8] = O[j][3]; }
+                }
+                if (quad_row == 0) {
+                    if (has_a) p.part_ml[slot * G + quad_col] = make_float2(m_a, l_a);
+                    if (has_b) p.part_ml[slot * G + quad_col + 1] = make_float2(m_b, l_b);
                 }
             }
             seg_open = false;

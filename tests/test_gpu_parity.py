@@ -145,6 +145,38 @@ def test_closed_forms_on_gpu():
     np.testing.assert_allclose(l[1:4, 0], [math.log1p(math.e), math.log(Z), 1024.0], rtol=1e-6)
 
 
+@pytest.mark.parametrize("shape", ["rising", "falling", "jumps"])
+def test_running_max_refresh_paths(shape):
+    """Logits that drift far from the first page's maximum: slowly (inside the rescale slack for several
+    pages, then beyond it), downwards (never beyond it), and in jumps of tens of log2 units."""
+    Hq, Hkv, d = 8, 1, 64
+    L = 2000
+    lens = np.array([L, L // 3], dtype=np.int32)
+    cache = wl.build_paged_cache(lens, Hkv, d, seed=80, device=DEV, poison=True)
+    t = np.arange(L)
+    if shape == "rising":
+        a = np.floor(t * (30.0 / L) * 8) / 8          # logits 0 .. 60 (natural units), bf16-exact steps
+    elif shape == "falling":
+        a = np.floor((L - 1 - t) * (30.0 / L) * 8) / 8
+    else:
+        rng = np.random.default_rng(81)
+        a = np.repeat(rng.integers(-120, 120, size=L // 50 + 1), 50)[:L] / 4.0  # plateaus of 50 tokens
+    q = torch.zeros((2, Hq, d), dtype=torch.bfloat16, device=DEV)
+    q[:, :, 0] = 16.0                                  # s_t = 0.125 * 16 * a_t = 2 a_t
+    q[:, :, 1:] = (0.05 * wl.random_bf16((2, Hq, d - 1), 82, DEV).float()).to(torch.bfloat16)
+    for b in range(2):
+        n = int(lens[b])
+        pages = torch.from_numpy(cache.page_table_host[b, np.arange(n) // 16].astype(np.int64)).to(DEV)
+        slots = torch.from_numpy(np.arange(n) % 16).to(DEV)
+        cache.k_pages[pages, 0, slots, 0] = torch.from_numpy(a[:n].astype(np.float32)).to(DEV).to(torch.bfloat16)
+    with ctx_for(cache, Hq) as ctx:
+        for split in (0, 5, 100000):
+            out, lse = run_attn(ctx, cache, q, cache.ctx_lens, 0.125, split_pages=split)
+            ref, ref_lse = oracle_on_cache(q, cache, lens, 0.125)
+            assert_parity(out, ref, f"{shape} split {split}")
+            np.testing.assert_allclose(lse.cpu().numpy(), ref_lse, rtol=2e-5, atol=2e-5)
+
+
 def test_gqa_mapping_and_identical_keys_on_gpu():
     Hq, Hkv, d = 8, 2, 64
     lens = np.array([77, 200], dtype=np.int32)
