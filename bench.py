@@ -161,14 +161,24 @@ def run_cuda(args):
     lens = lens0.astype(np.int64).copy()
     bpt = w.kv_bytes_per_token
 
+    # page-table updates of one step travel in one pinned staging row: (sequence, logical page, physical page)
+    stage_rows = 2 * (W + K) + 8
+    staging = torch.empty((stage_rows, 3, B), dtype=torch.int64).pin_memory() if dynamic_alloc else None
+    alloc_calls = [0]
+
     def allocate_pages():
         if not dynamic_alloc:
             return
         need, logical, phys = alloc.assign(lens)
-        if len(need):
-            cache.page_table[torch.from_numpy(need).to(dev, non_blocking=True),
-                             torch.from_numpy(logical).to(dev, non_blocking=True)] = \
-                torch.from_numpy(phys).to(dev, non_blocking=True)
+        n = len(need)
+        if n:
+            row = staging[alloc_calls[0] % stage_rows]
+            alloc_calls[0] += 1
+            row[0, :n] = torch.from_numpy(need)
+            row[1, :n] = torch.from_numpy(logical)
+            row[2, :n] = torch.from_numpy(phys.astype(np.int64))
+            upd = row[:, :n].to(dev, non_blocking=True)
+            cache.page_table[upd[0], upd[1]] = upd[2].to(torch.int32)
 
     def device_step(i):
         nonlocal lens

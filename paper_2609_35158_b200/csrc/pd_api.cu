@@ -42,6 +42,7 @@ struct pd_ctx {
     int halving_levels = 0;
     int tail_pages = 16;
     int pdl = 1;
+    int merge_rows = 0;
     size_t slots = 0;
     // device workspace (one allocation)
     void *workspace = nullptr;
@@ -168,6 +169,7 @@ int pd_create(const pd_config *cfg, pd_ctx **out) {
     ctx->halving_levels = env_int("PD_TUNE_LEVELS", 6);
     ctx->tail_pages = env_int("PD_TUNE_TAIL", 16);
     ctx->pdl = env_int("PD_TUNE_PDL", 1);
+    ctx->merge_rows = env_int("PD_TUNE_MERGE_ROWS", 0);
     if (ctx->halving_levels < 0 || ctx->halving_levels > pd::kMaxLevels - 2 || ctx->tail_pages < 1) {
         delete ctx;
         return PD_ERR_INVALID_ARG;
@@ -315,6 +317,7 @@ int pd_decode_attn(pd_ctx *ctx, const void *q, const void *k_pages, const void *
     p.tail_pages = ctx->tail_pages;
     const bool hooked = ctx->ev_before != nullptr;
     p.pdl = hooked ? 0 : ctx->pdl;  // timing events must bracket the split kernel alone: no overlap with neighbours
+    p.merge_rows = ctx->merge_rows;
     p.trace = ctx->trace;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (hooked) cudaEventRecord(ctx->ev_before, s);

@@ -548,26 +548,36 @@ __device__ __forceinline__ long long range_of_unit(const int32_t *plan, long lon
     return rec[4 * l + 3] + (x - start_of(l)) / rec[4 * l + 2];
 }
 
-// One CTA per (sequence, query head): its warps take the row's partials round-robin, eight loads in
-// flight each, keeping a running (max, sum, output); the per-warp results are then combined through
-// shared memory in warp order. The order of operations is fixed, so reruns are bit-identical.
-template <int D, int WARPS>
+// Each CTA merges R consecutive rows (query heads of one KV head; R divides the group size). Warp w
+// works on row w % R and takes every (WARPS / R)-th partial of it, eight loads in flight, keeping a
+// running (max, sum, output); the warps of a row are then combined through shared memory in warp
+// order. The order of operations is fixed, so reruns are bit-identical.
+template <int D, int WARPS, int R>
 __global__ void __launch_bounds__(WARPS * 32) lse_merge_kernel(const AttnParams p) {
     constexpr int VEC = D / 32;
     constexpr int UNROLL = 8;
+    constexpr int S = WARPS / R;  // warps sharing one row
+    static_assert(WARPS % R == 0, "rows per CTA must divide the warp count");
     __shared__ float sm_o[WARPS][D];
     __shared__ float2 sm_ml[WARPS];
+    __shared__ int32_t sm_plan[kPlanWords + 2];  // the plan, then the two prefix sums of this sequence
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int row = blockIdx.x;
-    grid_dependency_wait();  // partials, prefix sums and the plan come from the split kernel
-    launch_dependents();
-    const int b = row / p.Hq, h = row - b * p.Hq;
+    const int row = blockIdx.x * R + warp % R;
+    const int sub = warp / R;
+    const int b = (blockIdx.x * R) / p.Hq;  // all rows of the CTA belong to one sequence and one KV head
+    const int h = row - b * p.Hq;
     const int G = p.G;
     const int kvh = h / G, r = h - kvh * G;
-    const int c0 = p.cum_pages[b], np = p.cum_pages[b + 1] - c0;
+    grid_dependency_wait();  // partials, prefix sums and the plan come from the split kernel
+    launch_dependents();
+    // one round trip for everything the bookkeeping needs
+    for (int i = threadIdx.x; i < kPlanWords + 2; i += WARPS * 32)
+        sm_plan[i] = i < kPlanWords ? p.plan[i] : p.cum_pages[b + (i - kPlanWords)];
+    __syncthreads();
+    const int c0 = sm_plan[kPlanWords], np = sm_plan[kPlanWords + 1] - c0;
     __nv_bfloat16 *orow = p.out + static_cast<size_t>(row) * D + lane * VEC;
     if (np == 0) {  // empty context: zero row, lse = -inf
-        if (warp == 0) {
+        if (sub == 0) {
 #pragma unroll
             for (int v = 0; v < VEC; ++v) orow[v] = __float2bfloat16(0.f);
             if (p.lse != nullptr && lane == 0) p.lse[row] = -INFINITY;
@@ -575,20 +585,20 @@ __global__ void __launch_bounds__(WARPS * 32) lse_merge_kernel(const AttnParams 
         return;
     }
     const long long u0 = static_cast<long long>(p.Hkv) * c0 + static_cast<long long>(kvh) * np;
-    const long long first = range_of_unit(p.plan, u0), last = range_of_unit(p.plan, u0 + np - 1);
-    if (first == last) return;  // written directly by the split kernel
+    const long long first = range_of_unit(sm_plan, u0), last = range_of_unit(sm_plan, u0 + np - 1);
+    if (first == last) return;  // written directly by the split kernel (the same for every row of the CTA)
     const int n = static_cast<int>(last - first) + 1;
     const size_t slot0 = static_cast<size_t>(first) + static_cast<size_t>(b) * p.Hkv + kvh;
 
     float m = -INFINITY, l = 0.f, acc[VEC];
 #pragma unroll
     for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
-    for (int i0 = warp; i0 < n; i0 += WARPS * UNROLL) {
+    for (int i0 = sub; i0 < n; i0 += S * UNROLL) {
         float2 ml[UNROLL];
         float o[UNROLL][VEC];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-            const int i = i0 + u * WARPS;
+            const int i = i0 + u * S;
             if (i < n) {
                 const size_t rec = (slot0 + i) * G + r;
                 ml[u] = p.part_ml[rec];
@@ -626,19 +636,19 @@ __global__ void __launch_bounds__(WARPS * 32) lse_merge_kernel(const AttnParams 
     for (int v = 0; v < VEC; ++v) sm_o[warp][lane * VEC + v] = acc[v];
     if (lane == 0) sm_ml[warp] = make_float2(m, l);
     __syncthreads();
-    if (warp == 0) {
+    if (sub == 0) {  // warp w < R finishes row w: its partners are warps w, w + R, w + 2R, ...
         float M = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < WARPS; ++w) M = fmaxf(M, sm_ml[w].x);
+        for (int k = 0; k < S; ++k) M = fmaxf(M, sm_ml[warp + k * R].x);
         float Lsum = 0.f, out[VEC];
 #pragma unroll
         for (int v = 0; v < VEC; ++v) out[v] = 0.f;
 #pragma unroll
-        for (int w = 0; w < WARPS; ++w) {
-            const float wt = exp2f(sm_ml[w].x - M);  // warps without records carry m = -inf, weight 0
-            Lsum += wt * sm_ml[w].y;
+        for (int k = 0; k < S; ++k) {
+            const float wt = exp2f(sm_ml[warp + k * R].x - M);  // warps without records carry m = -inf, weight 0
+            Lsum += wt * sm_ml[warp + k * R].y;
 #pragma unroll
-            for (int v = 0; v < VEC; ++v) out[v] += wt * sm_o[w][lane * VEC + v];
+            for (int v = 0; v < VEC; ++v) out[v] += wt * sm_o[warp + k * R][lane * VEC + v];
         }
         const float inv = 1.f / Lsum;
 #pragma unroll
@@ -689,15 +699,19 @@ cudaError_t launch_decode_attn(const AttnVariant &v, const CUtensorMap &tm_k, co
 }
 
 cudaError_t launch_lse_merge(int head_dim, const AttnParams &p, cudaStream_t stream) {
-    // few rows (low decode concurrency) mean many partials per row: give each row more warps
+    // Few rows (low decode concurrency) mean many partials per row: all 8 warps of a CTA share one
+    // row. With many rows the partial lists are short and CTA count dominates: a CTA takes several rows.
     const int rows = p.B * p.Hq;
     const bool pdl = p.pdl != 0;
-    if (head_dim == 128) {
-        if (rows <= 4096) return launch_pdl(lse_merge_kernel<128, 8>, dim3(rows), dim3(256), 0, stream, pdl, p);
-        return launch_pdl(lse_merge_kernel<128, 2>, dim3(rows), dim3(64), 0, stream, pdl, p);
-    }
-    if (rows <= 4096) return launch_pdl(lse_merge_kernel<64, 8>, dim3(rows), dim3(256), 0, stream, pdl, p);
-    return launch_pdl(lse_merge_kernel<64, 2>, dim3(rows), dim3(64), 0, stream, pdl, p);
+    int r = p.merge_rows > 0 ? p.merge_rows : (rows <= 512 ? 1 : (rows <= 1024 ? 2 : 8));
+    while (r > 1 && p.G % r != 0) r >>= 1;
+#define PD_MERGE(D_, R_)                                                                                  \
+    if (head_dim == D_ && r == R_)                                                                        \
+        return launch_pdl(lse_merge_kernel<D_, 8, R_>, dim3(rows / R_), dim3(256), 0, stream, pdl, p);
+    PD_MERGE(128, 1) PD_MERGE(128, 2) PD_MERGE(128, 4) PD_MERGE(128, 8)
+    PD_MERGE(64, 1) PD_MERGE(64, 2) PD_MERGE(64, 4) PD_MERGE(64, 8)
+#undef PD_MERGE
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace pd

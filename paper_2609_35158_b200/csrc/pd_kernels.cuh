@@ -46,6 +46,7 @@ struct AttnParams {
     int32_t halving_levels;     // automatic plan: number of levels whose ranges halve the remaining fair share
     int32_t tail_pages;         // automatic plan: pages per range of the last level
     int32_t pdl;                // launch with programmatic stream serialization
+    int32_t merge_rows;         // rows per CTA of the merge kernel, 0 = chosen from the row count
     unsigned long long *trace;  // optional [workers][4] ns timestamps: kernel entry, first data, last data, exit
 };
 

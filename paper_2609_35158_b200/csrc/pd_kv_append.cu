@@ -40,7 +40,7 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const AppendParams p) {
         const __nv_bfloat16 *src = (which ? p.v_new : p.k_new) + (static_cast<size_t>(b) * p.Hkv + kvh) * p.D + j * 8;
         __nv_bfloat16 *dst = (which ? p.v_pages : p.k_pages) +
                              ((static_cast<size_t>(page) * p.Hkv + kvh) * kPageSize + slot) * p.D + j * 8;
-        *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
+        *reinterpret_cast<uint4 *>(dst) = __ldg(reinterpret_cast<const uint4 *>(src));
     }
     if (p.advance && threadIdx.x == 0) p.ctx_lens[b] = pos + 1;
 }
