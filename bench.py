@@ -30,9 +30,9 @@ METRIC = "decode-attn achieved HBM GB/s (% of B200 peak) and seq-steps/s per lay
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) per launch of the split kernel in the committed ncu capture
-# (profiles/decode_attn_split_config3_ncu.md: 1.577394 GB + 4.45 MB), as a ratio to the
+# (profiles/decode_attn_split_config3_ncu.md: 1.577338 GB + 7.53 MB), as a ratio to the
 # algorithmic KV bytes of that launch (1.576878 GB); traffic grows in proportion to the pages read.
-NCU_TRAFFIC_RATIO = 1.0031
+NCU_TRAFFIC_RATIO = 1.0051
 
 
 def measured_hbm_peak():
