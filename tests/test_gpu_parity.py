@@ -345,23 +345,25 @@ def test_full_size_configs_all_rows(config):
 
 
 def test_config4_multiturn_loop_with_page_allocation():
-    """Config 4 at full batch: steps of (allocate, append, attend). Appends are checked on
-    the pages they touch, attention on a sample of sequences that always includes the
-    shortest and the longest; 8 steps here, placed so that every sequence crosses a
-    page boundary in the sample at least once is not guaranteed, so boundary crossings
-    are forced by choosing the sampled sequences among those that allocate."""
+    """Config 4 at full batch: 128 steps of (allocate, append, attend) with the host free list in the
+    loop. Every append is checked on the slot it must fill; attention is checked against the oracle on
+    steps 0, 1, 63, 126 and 127 for a sample of sequences that holds the shortest, the longest and
+    several that open a new page during the loop."""
     w = wl.WORKLOADS[4]
     lens0 = wl.context_lengths(4)
-    B, steps = w.batch, 8
+    B, steps = w.batch, 128
+    check_steps = (0, 1, 63, 126, 127)
     cache = wl.build_paged_cache(lens0, w.num_kv_heads, w.head_dim, seed=4, device=DEV, reserve_tokens=steps,
                                  preassign_reserve=False, poison=False)
     alloc = wl.PageAllocator(cache)
     lens = lens0.copy()
-    will_allocate = np.nonzero((16 - lens0 % 16) % 16 < steps)[0]
-    sample = sorted(set([int(np.argmin(lens0)), int(np.argmax(lens0))] + will_allocate[:6].tolist() + [0, 1, 2]))
+    sample = sorted(set([int(np.argmin(lens0)), int(np.argmax(lens0))] + list(range(6))))
+    ar = torch.arange(B, device=DEV)
+    allocated = 0
     with ctx_for(cache, w.num_q_heads) as ctx:
         for step in range(steps):
             need, logical, phys = alloc.assign(lens)
+            allocated += len(need)
             if len(need):
                 cache.page_table[torch.from_numpy(need).to(DEV), torch.from_numpy(logical).to(DEV)] = \
                     torch.from_numpy(phys).to(DEV)
@@ -369,15 +371,51 @@ def test_config4_multiturn_loop_with_page_allocation():
             kn = wl.random_bf16((B, w.num_kv_heads, w.head_dim), 5000 + step, DEV)
             vn = wl.random_bf16((B, w.num_kv_heads, w.head_dim), 6000 + step, DEV)
             ctx.pd.pd_kv_append(ctx.h, kn, vn, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens)
-            out, _ = run_attn(ctx, cache, q, cache.ctx_lens, w.sm_scale, want_lse=False)
+            out = torch.empty((B, w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=DEV)
+            ctx.pd.pd_decode_attn(ctx.h, q, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, out,
+                                  sm_scale=w.sm_scale)
             # append: the slot of every sequence holds exactly the new rows
             pos = torch.from_numpy(lens.astype(np.int64)).to(DEV)
-            page = cache.page_table[torch.arange(B, device=DEV), pos // 16].long()
+            page = cache.page_table[ar, pos // 16].long()
             assert torch.equal(cache.k_pages[page, :, pos % 16], kn)
             assert torch.equal(cache.v_pages[page, :, pos % 16], vn)
             lens = lens + 1
-            assert np.array_equal(cache.ctx_lens.cpu().numpy(), lens)
-            if step in (0, 1, steps - 1):
+            if step in check_steps:
+                assert ctx.pd.pd_device_status(ctx.h)[0] == 0
+                assert np.array_equal(cache.ctx_lens.cpu().numpy(), lens)
                 ref, _ = oracle_on_cache(q, cache, lens, w.sm_scale, seq_ids=sample)
                 assert_parity(out[sample], ref, f"config 4 step {step}")
-    assert len(will_allocate) > 0
+        assert ctx.pd.pd_device_status(ctx.h)[0] == 0
+    assert allocated >= B * (steps // 16)  # every sequence crossed page boundaries during the loop
+
+
+def test_maximum_batch_with_empty_and_tiny_contexts():
+    """4096 sequences (the largest batch a context accepts), lengths 0..40 with many zeros."""
+    Hq, Hkv, d, B = 8, 2, 64, 4096
+    rng = np.random.default_rng(90)
+    lens = rng.integers(0, 40, size=B, endpoint=True).astype(np.int32)
+    lens[rng.integers(0, B, size=300)] = 0
+    lens[-1] = 0
+    cache = wl.build_paged_cache(lens, Hkv, d, seed=91, device=DEV, max_pages_per_seq=3)
+    q = wl.random_bf16((B, Hq, d), 92, DEV)
+    with ctx_for(cache, Hq) as ctx:
+        for split in (0, 1):
+            out, lse = run_attn(ctx, cache, q, cache.ctx_lens, 0.125, split_pages=split)
+            ref, ref_lse = oracle_on_cache(q, cache, lens, 0.125)
+            assert_parity(out, ref, f"max batch split {split}")
+            np.testing.assert_allclose(lse.cpu().numpy(), ref_lse, rtol=2e-5, atol=2e-5)
+            empty = torch.from_numpy(lens == 0).to(DEV)
+            assert torch.all(out[empty] == 0) and torch.all(torch.isinf(lse[empty]))
+
+
+def test_one_very_long_sequence_alone():
+    """Batch 1, 65 536 tokens: every worker warp reads a slice of the same (sequence, KV head) pairs."""
+    Hq, Hkv, d = 32, 8, 128
+    lens = np.array([65536], dtype=np.int32)
+    cache = wl.build_paged_cache(lens, Hkv, d, seed=93, device=DEV)
+    q = wl.random_bf16((1, Hq, d), 94, DEV)
+    with ctx_for(cache, Hq) as ctx:
+        out, lse = run_attn(ctx, cache, q, cache.ctx_lens, 1.0 / math.sqrt(d))
+    ref, ref_lse = oracle_on_cache(q, cache, lens, 1.0 / math.sqrt(d))
+    assert_parity(out, ref, "single 64K sequence")
+    np.testing.assert_allclose(lse.cpu().numpy(), ref_lse, rtol=2e-5, atol=2e-5)
