@@ -347,6 +347,123 @@ def time_oracle_once(w, cache, q, lens, max_seconds_hint: float = 30.0):
             "seconds_per_step": round(dt, 3)}
 
 
+# ------------------------------------------------------------------------------------------ KV transfer op
+
+def run_transfer(args):
+    """Gather + scatter of the pages holding every sequence's new tokens (Eq. 3's KV-transfer term).
+
+    Workload: configs[4] geometry (batch 512, 32/8 heads, d = 128); every sequence moves the pages of one
+    turn of U{256..2048} new tokens. A step packs them on the source cache and unpacks them into a
+    differently placed destination cache. Value = bytes read + written by both kernels / step time."""
+    import torch
+
+    import oracle
+    import paper_2609_35158_b200 as pd
+    import workloads as wl
+
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    w = wl.WORKLOADS[4]
+    K, W = args.steps, args.warmup
+    rng = np.random.Generator(np.random.PCG64(404))
+    new_tokens = rng.integers(256, 2048, size=w.batch, endpoint=True).astype(np.int32)
+    src = wl.build_paged_cache(new_tokens, w.num_kv_heads, w.head_dim, seed=41, device=dev)
+    dst = wl.build_paged_cache(new_tokens, w.num_kv_heads, w.head_dim, seed=42, device=dev)
+    pe = ((new_tokens + 15) // 16).astype(np.int32)
+    pb = np.zeros_like(pe)
+    off = np.concatenate([[0], np.cumsum(pe)[:-1]]).astype(np.int64)
+    total_pages = int(pe.sum())
+    page_bytes = 2 * w.num_kv_heads * 16 * w.head_dim * 2
+    to_dev = lambda a: torch.from_numpy(a).to(dev)
+    d_pb, d_pe, d_off = to_dev(pb), to_dev(pe), to_dev(off)
+    packed = torch.empty((total_pages, 2, w.num_kv_heads, 16, w.head_dim), dtype=torch.bfloat16, device=dev)
+    ctx_s = pd.pd_create(w.num_q_heads, w.num_kv_heads, w.head_dim, 16, w.batch, src.page_table.shape[1], src.num_pages, 0)
+    ctx_d = pd.pd_create(w.num_q_heads, w.num_kv_heads, w.head_dim, 16, w.batch, dst.page_table.shape[1], dst.num_pages, 0)
+
+    def step(buf):
+        pd.pd_kv_gather(ctx_s, src.k_pages, src.v_pages, src.page_table, d_pb, d_pe, d_off, buf)
+        pd.pd_kv_scatter(ctx_d, buf, d_off, dst.k_pages, dst.v_pages, dst.page_table, d_pb, d_pe)
+
+    for _ in range(W):
+        step(packed)
+    torch.cuda.synchronize()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    t0, t1 = ev(), ev()
+    hooked = [i for i in range(K) if i % 16 == min(8, K - 1)]
+    hb, ha = {i: ev() for i in hooked}, {i: ev() for i in hooked}
+    sampler = ClockSampler(0)
+    sampler.start()
+    t0.record()
+    for i in range(K):
+        if i in hb:
+            hb[i].record()
+            pd.pd_kv_gather(ctx_s, src.k_pages, src.v_pages, src.page_table, d_pb, d_pe, d_off, packed)
+            ha[i].record()
+            pd.pd_kv_scatter(ctx_d, packed, d_off, dst.k_pages, dst.v_pages, dst.page_table, d_pb, d_pe)
+        else:
+            step(packed)
+    t1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = t0.elapsed_time(t1) / K
+    gather_ms = float(np.mean([hb[i].elapsed_time(ha[i]) for i in hooked]))
+    moved = 2 * 2 * total_pages * page_bytes  # two kernels, each reads and writes every page
+    assert pd.pd_device_status(ctx_s)[0] == 0 and pd.pd_device_status(ctx_d)[0] == 0
+
+    # host-buffer variant: the packed buffer crosses PCIe in both directions (what a host-staged transport does)
+    host = torch.empty(packed.shape, dtype=torch.bfloat16).pin_memory()
+    e0, e1 = ev(), ev()
+    for i in range(W + K):
+        if i == W:
+            e0.record()
+        pd.pd_kv_gather(ctx_s, src.k_pages, src.v_pages, src.page_table, d_pb, d_pe, d_off, packed)
+        host.copy_(packed, non_blocking=True)
+        packed.copy_(host, non_blocking=True)
+        pd.pd_kv_scatter(ctx_d, packed, d_off, dst.k_pages, dst.v_pages, dst.page_table, d_pb, d_pe)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1) / K
+
+    # CPU baseline: the oracle's gather + scatter on a prefix of the batch
+    n = 64
+    sub = list(range(n))
+    sk, sv = oracle.bf16_bits(src.k_pages), oracle.bf16_bits(src.v_pages)
+    dk, dv = oracle.bf16_bits(dst.k_pages).copy(), oracle.bf16_bits(dst.v_pages).copy()
+    sub_off = np.concatenate([[0], np.cumsum(pe[:n])[:-1]]).astype(np.int64)
+    t = time.perf_counter()
+    reps = 5
+    for _ in range(reps):
+        pk, _rc = oracle.kv_gather(sk, sv, src.page_table_host[:n], pb[:n], pe[:n], sub_off, int(pe[:n].sum()))
+        oracle.kv_scatter(pk, sub_off, dk, dv, dst.page_table_host[:n], pb[:n], pe[:n])
+    cpu_s = (time.perf_counter() - t) / reps
+    cpu_bytes = 4 * int(pe[:n].sum()) * page_bytes
+    peak, peak_kind = measured_hbm_peak()
+    value = moved / (ms * 1e-3) / 1e9
+    achieved = (moved / 2) / (gather_ms * 1e-3) / 1e9
+    result = {
+        "metric": "KV page gather+scatter bytes moved (read+write) GB/s", "value": round(value, 2), "unit": "GB/s",
+        "n_gpus": 1, "steps": K, "warmup": W, "ms_per_step": round(ms, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": "KV transfer, configs[4] geometry: batch 512, 8 KV heads, d 128, one turn of U{256..2048} new tokens per sequence",
+                   "pages_moved": total_pages, "packed_bytes": total_pages * page_bytes,
+                   "kv_bytes_per_token_K": w.kv_bytes_per_token,
+                   "l2": f"{total_pages * page_bytes / 1e9:.2f} GB packed per step >> 126 MB L2"},
+        "clocks": clocks,
+        "e2e": {"value": round(moved / (e2e_ms * 1e-3) / 1e9, 2), "unit": "GB/s",
+                "h2d_bytes_per_step": total_pages * page_bytes, "d2h_bytes_per_step": total_pages * page_bytes,
+                "ms_per_step": round(e2e_ms, 5), "note": "packed buffer staged through pinned host memory between gather and scatter"},
+        "gpu_launches": 2 * K,
+        "roofline": {"bound": "hbm", "kernel": "kv_transfer_kernel<gather>", "achieved": round(achieved, 2), "peak": peak,
+                     "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "algorithmic_bytes_per_launch": moved // 2, "avg_launch_ms": round(gather_ms, 5)},
+        "cpu_baseline": {"value": round(cpu_bytes / cpu_s / 1e9, 3), "unit": "GB/s", "cores": 1, "kind": "oracle",
+                         "sample": f"gather + scatter of the first {n} sequences ({int(pe[:n].sum())} pages), {reps} repetitions"},
+    }
+    pd.pd_destroy(ctx_s)
+    pd.pd_destroy(ctx_d)
+    print(json.dumps(result), flush=True)
+
+
 # ------------------------------------------------------------------------------------------ reference arm
 
 def run_reference(args):
@@ -409,11 +526,15 @@ def main():
     ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--op", default="decode", choices=["decode", "kv_transfer"],
+                    help="decode = the headline decode step; kv_transfer = page gather + scatter")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.op == "kv_transfer":
+        run_transfer(args)
     else:
         run_cuda(args)
 

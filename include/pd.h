@@ -132,6 +132,31 @@ int pd_decode_step_host(pd_ctx *ctx, const void *q_host, const void *k_new_host,
                         void *out_host, int32_t batch, float sm_scale, int32_t split_pages, void *stream);
 
 /*
+ * KV page gather / scatter: the device-side data movement of the cross-pool KV
+ * transfer in the disaggregated prefill model (Eq. 3, the B * dL * K / BW term).
+ * The prefill side packs the pages that hold a sequence's new tokens into one
+ * contiguous buffer; the decode side unpacks such a buffer into pages it has
+ * assigned itself. The transport between the two is not part of this library.
+ *
+ * For every b < batch the logical pages [page_begin[b], page_end[b]) are moved.
+ * The packed buffer is [packed pages][2][num_kv_heads][page_size][head_dim]
+ * bf16: packed page packed_page_offset[b] + i holds the K block, then the V
+ * block, of logical page page_begin[b] + i (whole pages; slots past the
+ * sequence's length travel as they are). page_begin, page_end (int32) and
+ * packed_page_offset (int64, normally the exclusive prefix sum of the page
+ * counts) are DEVICE arrays supplied by the caller, who also sizes `packed`.
+ * Ranges of different sequences must not overlap in the packed buffer. A page
+ * id outside [0, num_pages) is skipped and latched for pd_device_status.
+ * K = 2 * num_kv_heads * head_dim * 2 bytes per token per layer.
+ */
+int pd_kv_gather(pd_ctx *ctx, const void *k_pages, const void *v_pages, const int32_t *page_table,
+                 const int32_t *page_begin, const int32_t *page_end, const int64_t *packed_page_offset,
+                 void *packed, int32_t batch, void *stream);
+int pd_kv_scatter(pd_ctx *ctx, const void *packed, const int64_t *packed_page_offset, void *k_pages,
+                  void *v_pages, const int32_t *page_table, const int32_t *page_begin,
+                  const int32_t *page_end, int32_t batch, void *stream);
+
+/*
  * Decode attention without any allocation (the paper has no counterpart; this
  * is a packaging variant of pd_decode_attn for restricted hosts).
  *

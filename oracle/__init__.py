@@ -47,6 +47,10 @@ def _load():
         lib.pd_oracle_lse_merge.restype = i
         lib.pd_oracle_kv_append.argtypes = [p, p, p, p, p, p, i, i, i, i, i, ctypes.c_int64, i]
         lib.pd_oracle_kv_append.restype = i
+        lib.pd_oracle_kv_gather.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, ctypes.c_int64]
+        lib.pd_oracle_kv_gather.restype = i
+        lib.pd_oracle_kv_scatter.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, ctypes.c_int64]
+        lib.pd_oracle_kv_scatter.restype = i
         _lib = lib
     return _lib
 
@@ -151,3 +155,36 @@ def kv_append(k_new, v_new, k_pages, v_pages, page_table, ctx_lens, *, advance: 
         k_new.ctypes.data, v_new.ctypes.data, k_pages.ctypes.data, v_pages.ctypes.data,
         page_table.ctypes.data, ctx_lens.ctypes.data, B, Hkv, d, P, page_table.shape[1], NP,
         1 if advance else 0)
+
+
+def kv_gather(k_pages, v_pages, page_table, page_begin, page_end, dst_page_offset, total_pages: int):
+    """Pack logical pages [page_begin[b], page_end[b]) of every sequence into one buffer.
+
+    Returns uint16 [total_pages, 2, Hkv, P, d]; packed page dst_page_offset[b] + i holds the K block then
+    the V block of logical page page_begin[b] + i."""
+    lib = _load()
+    k_pages, v_pages = _c(k_pages, np.uint16), _c(v_pages, np.uint16)
+    page_table = _c(page_table, np.int32)
+    pb, pe = _c(page_begin, np.int32), _c(page_end, np.int32)
+    off = _c(dst_page_offset, np.int64)
+    NP, Hkv, P, d = k_pages.shape
+    packed = np.zeros((total_pages, 2, Hkv, P, d), dtype=np.uint16)
+    rc = lib.pd_oracle_kv_gather(k_pages.ctypes.data, v_pages.ctypes.data, page_table.ctypes.data, pb.ctypes.data,
+                                 pe.ctypes.data, off.ctypes.data, packed.ctypes.data, len(pb), Hkv, d, P,
+                                 page_table.shape[1], NP)
+    return packed, rc
+
+
+def kv_scatter(packed, src_page_offset, k_pages, v_pages, page_table, page_begin, page_end) -> int:
+    """In-place unpack of a packed buffer into the pages the table names (host mirrors, uint16)."""
+    lib = _load()
+    for a in (k_pages, v_pages):
+        assert isinstance(a, np.ndarray) and a.dtype == np.uint16 and a.flags.c_contiguous and a.flags.writeable
+    packed = _c(packed, np.uint16)
+    page_table = _c(page_table, np.int32)
+    pb, pe = _c(page_begin, np.int32), _c(page_end, np.int32)
+    off = _c(src_page_offset, np.int64)
+    NP, Hkv, P, d = k_pages.shape
+    return lib.pd_oracle_kv_scatter(packed.ctypes.data, off.ctypes.data, k_pages.ctypes.data, v_pages.ctypes.data,
+                                    page_table.ctypes.data, pb.ctypes.data, pe.ctypes.data, len(pb), Hkv, d, P,
+                                    page_table.shape[1], NP)

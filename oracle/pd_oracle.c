@@ -227,3 +227,52 @@ int pd_oracle_kv_append(const uint16_t *k_new, const uint16_t *v_new,
     }
     return rc;
 }
+
+/*
+ * KV page gather / scatter: the data movement behind the cross-pool KV transfer
+ * term of the disaggregated prefill model (Eq. 3, B * dL * K / BW): the pages
+ * that hold a sequence's new tokens are packed into one contiguous buffer on the
+ * prefill side and unpacked into freshly assigned pages on the decode side.
+ *
+ * For sequence b the logical pages [page_begin[b], page_end[b]) are moved. The
+ * packed buffer holds whole pages: packed page (dst_page_offset[b] + i) is
+ *   [2][num_kv_heads][page_size][head_dim] bf16   (K block, then V block)
+ * of logical page page_begin[b] + i. Pure byte copies in index order.
+ * Return 0, or -(b+1) for the first sequence with an out-of-range page id
+ * (that sequence is skipped).
+ */
+int pd_oracle_kv_gather(const uint16_t *k_pages, const uint16_t *v_pages, const int32_t *page_table,
+                        const int32_t *page_begin, const int32_t *page_end, const int64_t *dst_page_offset,
+                        uint16_t *packed, int B, int Hkv, int d, int P, int MP, int64_t num_pages)
+{
+    int rc = 0;
+    const size_t tile = (size_t)Hkv * P * d; /* elements of one pool page */
+    for (int b = 0; b < B; ++b) {
+        for (int lp = page_begin[b]; lp < page_end[b]; ++lp) {
+            int32_t page = (lp >= 0 && lp < MP) ? page_table[(size_t)b * MP + lp] : -1;
+            if (page < 0 || (int64_t)page >= num_pages) { if (!rc) rc = -(b + 1); continue; }
+            uint16_t *dst = packed + ((size_t)dst_page_offset[b] + (size_t)(lp - page_begin[b])) * 2 * tile;
+            memcpy(dst, k_pages + (size_t)page * tile, sizeof(uint16_t) * tile);
+            memcpy(dst + tile, v_pages + (size_t)page * tile, sizeof(uint16_t) * tile);
+        }
+    }
+    return rc;
+}
+
+int pd_oracle_kv_scatter(const uint16_t *packed, const int64_t *src_page_offset, uint16_t *k_pages, uint16_t *v_pages,
+                         const int32_t *page_table, const int32_t *page_begin, const int32_t *page_end,
+                         int B, int Hkv, int d, int P, int MP, int64_t num_pages)
+{
+    int rc = 0;
+    const size_t tile = (size_t)Hkv * P * d;
+    for (int b = 0; b < B; ++b) {
+        for (int lp = page_begin[b]; lp < page_end[b]; ++lp) {
+            int32_t page = (lp >= 0 && lp < MP) ? page_table[(size_t)b * MP + lp] : -1;
+            if (page < 0 || (int64_t)page >= num_pages) { if (!rc) rc = -(b + 1); continue; }
+            const uint16_t *src = packed + ((size_t)src_page_offset[b] + (size_t)(lp - page_begin[b])) * 2 * tile;
+            memcpy(k_pages + (size_t)page * tile, src, sizeof(uint16_t) * tile);
+            memcpy(v_pages + (size_t)page * tile, src + tile, sizeof(uint16_t) * tile);
+        }
+    }
+    return rc;
+}

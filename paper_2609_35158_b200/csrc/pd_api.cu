@@ -272,6 +272,55 @@ int pd_kv_append(pd_ctx *ctx, const void *k_new, const void *v_new, void *k_page
     return PD_OK;
 }
 
+namespace {
+
+int kv_transfer(pd_ctx *ctx, bool scatter, void *k_pages, void *v_pages, const int32_t *page_table,
+                const int32_t *page_begin, const int32_t *page_end, const int64_t *packed_page_offset, void *packed,
+                int32_t batch, void *stream) {
+    if (int rc = check_batch(ctx, batch)) return rc;
+    if (!aligned16(k_pages) || !aligned16(v_pages) || !aligned16(packed) || page_table == nullptr ||
+        page_begin == nullptr || page_end == nullptr || packed_page_offset == nullptr)
+        return fail(ctx, PD_ERR_INVALID_ARG, "KV transfer: null or misaligned pointer");
+    if (batch == 0) return PD_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
+    pd::TransferParams p{};
+    p.k_pages = static_cast<__nv_bfloat16 *>(k_pages);
+    p.v_pages = static_cast<__nv_bfloat16 *>(v_pages);
+    p.packed = packed;
+    p.page_table = page_table;
+    p.page_begin = page_begin;
+    p.page_end = page_end;
+    p.packed_page_offset = reinterpret_cast<const long long *>(packed_page_offset);
+    p.status = ctx->status;
+    p.B = batch;
+    p.Hkv = ctx->cfg.num_kv_heads;
+    p.D = ctx->cfg.head_dim;
+    p.MP = ctx->cfg.max_pages_per_seq;
+    p.num_pages = static_cast<int32_t>(ctx->cfg.num_pages);
+    p.pdl = ctx->pdl;
+    const cudaError_t err = pd::launch_kv_transfer(p, scatter, ctx->num_sms, static_cast<cudaStream_t>(stream));
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, scatter ? "kv_scatter launch" : "kv_gather launch", err);
+    ctx->launches += 1;
+    return PD_OK;
+}
+
+}  // namespace
+
+int pd_kv_gather(pd_ctx *ctx, const void *k_pages, const void *v_pages, const int32_t *page_table,
+                 const int32_t *page_begin, const int32_t *page_end, const int64_t *packed_page_offset, void *packed,
+                 int32_t batch, void *stream) {
+    return kv_transfer(ctx, false, const_cast<void *>(k_pages), const_cast<void *>(v_pages), page_table, page_begin,
+                       page_end, packed_page_offset, packed, batch, stream);
+}
+
+int pd_kv_scatter(pd_ctx *ctx, const void *packed, const int64_t *packed_page_offset, void *k_pages, void *v_pages,
+                  const int32_t *page_table, const int32_t *page_begin, const int32_t *page_end, int32_t batch,
+                  void *stream) {
+    return kv_transfer(ctx, true, k_pages, v_pages, page_table, page_begin, page_end, packed_page_offset,
+                       const_cast<void *>(packed), batch, stream);
+}
+
 int pd_decode_attn(pd_ctx *ctx, const void *q, const void *k_pages, const void *v_pages, const int32_t *page_table,
                    const int32_t *ctx_lens, void *out, float *lse, int32_t batch, float sm_scale, int32_t split_pages,
                    void *stream) {

@@ -62,6 +62,18 @@ struct AppendParams {
     int32_t pdl;  // launch with programmatic stream serialization
 };
 
+struct TransferParams {
+    __nv_bfloat16 *k_pages, *v_pages;    // [NP][Hkv][16][D] (read by gather, written by scatter)
+    void *packed;                        // [packed pages][2][Hkv][16][D] (written by gather, read by scatter)
+    const int32_t *page_table;           // [B][MP]
+    const int32_t *page_begin, *page_end;    // [B] logical page range of every sequence
+    const long long *packed_page_offset;     // [B] index of the sequence's first page in the packed buffer
+    int32_t *status;
+    int32_t B, Hkv, D, MP;
+    int32_t num_pages;
+    int32_t pdl;
+};
+
 // Shape of one compiled variant of the split kernel.
 struct AttnVariant {
     int head_dim, warps, stages, hilo;
@@ -92,5 +104,6 @@ cudaError_t prepare_decode_attn(const AttnVariant &v, size_t *smem_bytes);  // o
 cudaError_t launch_decode_attn(const AttnVariant &v, const CUtensorMap &tm_k, const CUtensorMap &tm_v,
                                const AttnParams &p, int num_ctas, size_t smem_bytes, cudaStream_t stream);
 cudaError_t launch_lse_merge(int head_dim, const AttnParams &p, cudaStream_t stream);
+cudaError_t launch_kv_transfer(const TransferParams &p, bool scatter, int num_sms, cudaStream_t stream);
 
 }  // namespace pd

@@ -461,3 +461,40 @@ def test_workload_length_recipes():
     tok = [int(wl.context_lengths(1)[p].sum()) for p in parts]
     assert abs(tok[0] - tok[1]) < 16384
     assert len(list(itertools.chain(*parts))) == 64
+
+
+# ---------------------------------------------------------------- KV page gather / scatter
+
+def test_gather_matches_fancy_indexing_and_scatter_inverts_it():
+    Hkv, d, P = 2, 64, 16
+    lens = np.array([100, 16, 33, 0, 250], dtype=np.int32)
+    cache = wl.build_paged_cache(lens, Hkv, d, seed=30)
+    kp, vp = oracle.bf16_bits(cache.k_pages), oracle.bf16_bits(cache.v_pages)
+    table = cache.page_table_host
+    pages = (lens + P - 1) // P
+    pb = np.array([2, 0, 1, 0, 5], dtype=np.int32)             # only the pages of the "new" tokens
+    pe = pages.astype(np.int32)
+    cnt = np.maximum(pe - pb, 0)
+    off = np.concatenate([[0], np.cumsum(cnt)[:-1]]).astype(np.int64)
+    packed, rc = oracle.kv_gather(kp, vp, table, pb, pe, off, int(cnt.sum()))
+    assert rc == 0
+    for b in range(5):  # independent statement with NumPy fancy indexing
+        ids = table[b, pb[b]:pe[b]]
+        assert np.array_equal(packed[off[b]:off[b] + cnt[b], 0], kp[ids])
+        assert np.array_equal(packed[off[b]:off[b] + cnt[b], 1], vp[ids])
+    # scatter into a differently permuted destination cache, then compare logical contents
+    dst = wl.build_paged_cache(lens, Hkv, d, seed=31)
+    dk, dv = oracle.bf16_bits(dst.k_pages).copy(), oracle.bf16_bits(dst.v_pages).copy()
+    before_k = dk.copy()
+    assert oracle.kv_scatter(packed, off, dk, dv, dst.page_table_host, pb, pe) == 0
+    touched = np.zeros(dk.shape[0], dtype=bool)
+    for b in range(5):
+        src_ids, dst_ids = table[b, pb[b]:pe[b]], dst.page_table_host[b, pb[b]:pe[b]]
+        assert np.array_equal(dk[dst_ids], kp[src_ids]) and np.array_equal(dv[dst_ids], vp[src_ids])
+        touched[dst_ids] = True
+    assert np.array_equal(dk[~touched], before_k[~touched])  # nothing else was written
+    # an unassigned page id is reported and skipped
+    bad = table.copy()
+    bad[0, 3] = -1
+    _, rc = oracle.kv_gather(kp, vp, bad, pb, pe, off, int(cnt.sum()))
+    assert rc == -1
