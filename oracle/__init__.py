@@ -47,6 +47,10 @@ def _load():
         lib.pd_oracle_lse_merge.restype = i
         lib.pd_oracle_kv_append.argtypes = [p, p, p, p, p, p, i, i, i, i, i, ctypes.c_int64, i]
         lib.pd_oracle_kv_append.restype = i
+        lib.pd_oracle_prefill_attn.argtypes = [p, p, p, p, p, p, i, i, i, i, i, i, ctypes.c_float, p, p, i]
+        lib.pd_oracle_prefill_attn.restype = i
+        lib.pd_oracle_kv_append_tokens.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, ctypes.c_int64]
+        lib.pd_oracle_kv_append_tokens.restype = i
         lib.pd_oracle_kv_gather.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, ctypes.c_int64]
         lib.pd_oracle_kv_gather.restype = i
         lib.pd_oracle_kv_scatter.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, ctypes.c_int64]
@@ -188,3 +192,49 @@ def kv_scatter(packed, src_page_offset, k_pages, v_pages, page_table, page_begin
     return lib.pd_oracle_kv_scatter(packed.ctypes.data, off.ctypes.data, k_pages.ctypes.data, v_pages.ctypes.data,
                                     page_table.ctypes.data, pb.ctypes.data, pe.ctypes.data, len(pb), Hkv, d, P,
                                     page_table.shape[1], NP)
+
+
+def prefill_attn(q, q_indptr, k_pages, v_pages, page_table, ctx_lens, sm_scale, *, nthreads: int | None = None):
+    """Causal attention of packed new-token queries over prefix + themselves.
+
+    q: uint16 [total_q, Hq, d]; q_indptr: int32 [B+1]; the cache already holds the new tokens and
+    ctx_lens counts them. Returns (out fp64 [total_q, Hq, d], lse fp64 [total_q, Hq])."""
+    lib = _load()
+    q = _c(q, np.uint16)
+    ip = _c(q_indptr, np.int32)
+    k_pages, v_pages = _c(k_pages, np.uint16), _c(v_pages, np.uint16)
+    page_table, ctx_lens = _c(page_table, np.int32), _c(ctx_lens, np.int32)
+    total_q, Hq, d = q.shape
+    NP, Hkv, P, _ = k_pages.shape
+    B = len(ip) - 1
+    assert ip[0] == 0 and ip[-1] == total_q and np.all(np.diff(ip) >= 0)
+    for b in range(B):
+        assert ctx_lens[b] >= ip[b + 1] - ip[b], "the cache must already hold the new tokens"
+        if ctx_lens[b] > 0:
+            used = page_table[b, :(int(ctx_lens[b]) + P - 1) // P]
+            assert used.min() >= 0 and used.max() < NP, "page id out of range"
+    out = np.empty((total_q, Hq, d), dtype=np.float64)
+    lse = np.empty((total_q, Hq), dtype=np.float64)
+    if nthreads is None:
+        nthreads = os.cpu_count() or 1
+    rc = lib.pd_oracle_prefill_attn(q.ctypes.data, ip.ctypes.data, k_pages.ctypes.data, v_pages.ctypes.data,
+                                    page_table.ctypes.data, ctx_lens.ctypes.data, B, Hq, Hkv, d, P,
+                                    page_table.shape[1], ctypes.c_float(np.float32(sm_scale)), out.ctypes.data,
+                                    lse.ctypes.data, int(nthreads))
+    if rc != 0:
+        raise RuntimeError(f"pd_oracle_prefill_attn failed ({rc})")
+    return out, lse
+
+
+def kv_append_tokens(k_new, v_new, q_indptr, k_pages, v_pages, page_table, ctx_lens) -> int:
+    """In-place multi-token append on host mirrors; ctx_lens grows by each sequence's token count."""
+    lib = _load()
+    for a, dt in ((k_pages, np.uint16), (v_pages, np.uint16), (ctx_lens, np.int32)):
+        assert isinstance(a, np.ndarray) and a.dtype == dt and a.flags.c_contiguous and a.flags.writeable
+    k_new, v_new = _c(k_new, np.uint16), _c(v_new, np.uint16)
+    ip = _c(q_indptr, np.int32)
+    page_table = _c(page_table, np.int32)
+    NP, Hkv, P, d = k_pages.shape
+    return lib.pd_oracle_kv_append_tokens(k_new.ctypes.data, v_new.ctypes.data, ip.ctypes.data, k_pages.ctypes.data,
+                                          v_pages.ctypes.data, page_table.ctypes.data, ctx_lens.ctypes.data,
+                                          len(ip) - 1, Hkv, d, P, page_table.shape[1], NP)

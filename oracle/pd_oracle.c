@@ -276,3 +276,145 @@ int pd_oracle_kv_scatter(const uint16_t *packed, const int64_t *src_page_offset,
     }
     return rc;
 }
+
+/*
+ * Append-prefill attention: the step that opens every turn of a multi-turn
+ * rollout. The new turn's tokens (observation plus template, dL per trajectory
+ * in the prefill terms of Eq. 1 and Eq. 3) are appended to the cached context
+ * (Sec. 2.1) and each of them attends causally over the cached prefix and the
+ * new tokens up to and including itself; with prefix caching only these dL
+ * tokens are computed, but they read the whole context.
+ *
+ * Queries are packed: q [total_q][num_q_heads][head_dim], sequence b owns rows
+ * [q_indptr[b], q_indptr[b+1]). Its K/V (new tokens included) are already in the
+ * cache, ctx_lens[b] = L_b counts them. Query i of sequence b sits at absolute
+ * position pos = L_b - q_len_b + i and sees tokens 0 .. pos:
+ *   out[row][h] = softmax(sm_scale * q[row][h] . K_{0..pos}^T) V_{0..pos}
+ * Two passes in fp64 per (row, head), exactly as the decode definition.
+ */
+typedef struct {
+    attn_job base;          /* q points at the packed queries; B is unused here */
+    const int32_t *q_indptr;
+    int n_seq;
+    int next_item;
+} prefill_job;
+
+static void *prefill_worker(void *arg)
+{
+    prefill_job *J = (prefill_job *)arg;
+    attn_job *A = &J->base;
+    int maxlen = 1;
+    for (int b = 0; b < J->n_seq; ++b)
+        if (A->ctx_lens[b] > maxlen) maxlen = A->ctx_lens[b];
+    double *s_buf = (double *)malloc(sizeof(double) * (size_t)maxlen);
+    if (!s_buf) return (void *)1;
+    const int total_q = J->q_indptr[J->n_seq];
+    const int items = total_q * A->Hq;
+    const int d = A->d, P = A->P, g = A->Hq / A->Hkv;
+    const size_t page_stride = (size_t)A->Hkv * P * d;
+    for (;;) {
+        pthread_mutex_lock(&A->mu);
+        int it = J->next_item++;
+        pthread_mutex_unlock(&A->mu);
+        if (it >= items) break;
+        const int row = it / A->Hq, h = it % A->Hq, kvh = h / g;
+        int b = 0;
+        while (J->q_indptr[b + 1] <= row) ++b; /* sequence that owns this query row */
+        const int q_len = J->q_indptr[b + 1] - J->q_indptr[b];
+        const int pos = A->ctx_lens[b] - q_len + (row - J->q_indptr[b]);
+        double *o = A->out + ((size_t)row * A->Hq + h) * d;
+        for (int j = 0; j < d; ++j) o[j] = 0.0;
+        if (pos < 0) { A->lse[(size_t)row * A->Hq + h] = -INFINITY; continue; }
+        const uint16_t *qrow = A->q + ((size_t)row * A->Hq + h) * d;
+        double m = -INFINITY;
+        for (int t = 0; t <= pos; ++t) {
+            int32_t page = A->page_table[(size_t)b * A->MP + t / P];
+            const uint16_t *krow = A->k_pages + (size_t)page * page_stride + ((size_t)kvh * P + t % P) * d;
+            double dot = 0.0;
+            for (int j = 0; j < d; ++j) dot += bf16_to_f64(qrow[j]) * bf16_to_f64(krow[j]);
+            s_buf[t] = A->scale * dot;
+            if (s_buf[t] > m) m = s_buf[t];
+        }
+        double Z = 0.0;
+        for (int t = 0; t <= pos; ++t) {
+            double p = exp(s_buf[t] - m);
+            Z += p;
+            int32_t page = A->page_table[(size_t)b * A->MP + t / P];
+            const uint16_t *vrow = A->v_pages + (size_t)page * page_stride + ((size_t)kvh * P + t % P) * d;
+            for (int j = 0; j < d; ++j) o[j] += p * bf16_to_f64(vrow[j]);
+        }
+        for (int j = 0; j < d; ++j) o[j] /= Z;
+        A->lse[(size_t)row * A->Hq + h] = m + log(Z);
+    }
+    free(s_buf);
+    return NULL;
+}
+
+int pd_oracle_prefill_attn(const uint16_t *q, const int32_t *q_indptr, const uint16_t *k_pages, const uint16_t *v_pages,
+                           const int32_t *page_table, const int32_t *ctx_lens, int n_seq, int Hq, int Hkv, int d,
+                           int P, int MP, float sm_scale, double *out, double *lse, int nthreads)
+{
+    if (n_seq < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || d <= 0 || P <= 0 || MP <= 0) return -1;
+    if (nthreads < 1) nthreads = 1;
+    if (nthreads > 256) nthreads = 256;
+    prefill_job J;
+    memset(&J, 0, sizeof J);
+    J.base.q = q; J.base.k_pages = k_pages; J.base.v_pages = v_pages;
+    J.base.page_table = page_table; J.base.ctx_lens = ctx_lens;
+    J.base.Hq = Hq; J.base.Hkv = Hkv; J.base.d = d; J.base.P = P; J.base.MP = MP;
+    J.base.scale = (double)sm_scale;
+    J.base.out = out; J.base.lse = lse;
+    J.q_indptr = q_indptr; J.n_seq = n_seq; J.next_item = 0;
+    pthread_mutex_init(&J.base.mu, NULL);
+    int rc = 0;
+    pthread_t th[256];
+    int started = 0;
+    for (int i = 0; i < nthreads; ++i) {
+        if (pthread_create(&th[i], NULL, prefill_worker, &J) != 0) break;
+        ++started;
+    }
+    if (started == 0) rc = (prefill_worker(&J) != NULL) ? -1 : 0;
+    for (int i = 0; i < started; ++i) {
+        void *ret = NULL;
+        pthread_join(th[i], &ret);
+        if (ret != NULL) rc = -1;
+    }
+    pthread_mutex_destroy(&J.base.mu);
+    return rc;
+}
+
+/*
+ * Multi-token append: sequence b receives the rows [q_indptr[b], q_indptr[b+1])
+ * of k_new / v_new ([total][Hkv][d]) at positions ctx_lens[b], ctx_lens[b]+1, ...
+ * and its length grows by that count. Byte copies; a sequence with any position
+ * or page id out of range is skipped whole and reported as -(b+1).
+ */
+int pd_oracle_kv_append_tokens(const uint16_t *k_new, const uint16_t *v_new, const int32_t *q_indptr,
+                               uint16_t *k_pages, uint16_t *v_pages, const int32_t *page_table, int32_t *ctx_lens,
+                               int n_seq, int Hkv, int d, int P, int MP, int64_t num_pages)
+{
+    int rc = 0;
+    const size_t page_stride = (size_t)Hkv * P * d;
+    for (int b = 0; b < n_seq; ++b) {
+        const int n = q_indptr[b + 1] - q_indptr[b];
+        const int L = ctx_lens[b];
+        int ok = L >= 0 && n >= 0 && (L + n + P - 1) / P <= MP;
+        for (int i = 0; ok && i < n; ++i) {
+            int32_t page = page_table[(size_t)b * MP + (L + i) / P];
+            if (page < 0 || (int64_t)page >= num_pages) ok = 0;
+        }
+        if (!ok) { if (!rc) rc = -(b + 1); continue; }
+        for (int i = 0; i < n; ++i) {
+            const int pos = L + i;
+            const int32_t page = page_table[(size_t)b * MP + pos / P];
+            for (int kvh = 0; kvh < Hkv; ++kvh) {
+                size_t dst = (size_t)page * page_stride + ((size_t)kvh * P + pos % P) * d;
+                size_t src = ((size_t)(q_indptr[b] + i) * Hkv + kvh) * d;
+                memcpy(k_pages + dst, k_new + src, sizeof(uint16_t) * (size_t)d);
+                memcpy(v_pages + dst, v_new + src, sizeof(uint16_t) * (size_t)d);
+            }
+        }
+        ctx_lens[b] = L + n;
+    }
+    return rc;
+}

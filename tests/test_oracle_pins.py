@@ -498,3 +498,92 @@ def test_gather_matches_fancy_indexing_and_scatter_inverts_it():
     bad[0, 3] = -1
     _, rc = oracle.kv_gather(kp, vp, bad, pb, pe, off, int(cnt.sum()))
     assert rc == -1
+
+
+# ---------------------------------------------------------------- append-prefill attention
+
+def prefill_case(seed, lens, q_lens, Hq, Hkv, d):
+    lens, q_lens = np.asarray(lens, np.int32), np.asarray(q_lens, np.int32)
+    cache = wl.build_paged_cache(lens, Hkv, d, seed=seed, poison=True)
+    ip = np.concatenate([[0], np.cumsum(q_lens)]).astype(np.int32)
+    q = oracle.bf16_bits(wl.random_bf16((int(ip[-1]), Hq, d), seed + 1))
+    return cache, ip, q
+
+
+def test_prefill_equals_decode_definition_per_token_and_sdpa_causal():
+    Hq, Hkv, d = 4, 2, 64
+    lens, q_lens = [70, 33, 5, 40], [20, 33, 1, 0]
+    cache, ip, q = prefill_case(60, lens, q_lens, Hq, Hkv, d)
+    kp, vp = oracle.bf16_bits(cache.k_pages), oracle.bf16_bits(cache.v_pages)
+    out, lse = oracle.prefill_attn(q, ip, kp, vp, cache.page_table_host, np.asarray(lens, np.int32), 0.125)
+    assert np.all(np.isfinite(out)) and out.shape[0] == 54
+    kf, vf = oracle.bf16_bits_to_f64(kp), oracle.bf16_bits_to_f64(vp)
+    for b in range(4):
+        L, n = lens[b], q_lens[b]
+        if n == 0:
+            continue
+        # (1) every query token as a decode query over its visible prefix (the pinned decode definition)
+        for i in range(n):
+            vis = np.array([L - n + i + 1], np.int32)
+            o1, l1 = oracle.decode_attn(q[ip[b] + i][None], kp, vp, cache.page_table_host[b][None], vis, 0.125)
+            np.testing.assert_allclose(out[ip[b] + i], o1[0], rtol=1e-13, atol=1e-15)
+            np.testing.assert_allclose(lse[ip[b] + i], l1[0], rtol=1e-13)
+        # (2) torch SDPA on the dense layout with an explicit bottom-right-aligned causal mask
+        t = np.arange(L)
+        pages = cache.page_table_host[b, t // 16]
+        for kvh in range(Hkv):
+            Kd = torch.from_numpy(kf[pages, kvh, t % 16])      # [L, d]
+            Vd = torch.from_numpy(vf[pages, kvh, t % 16])
+            for h in range(kvh * 2, kvh * 2 + 2):
+                Qd = torch.from_numpy(oracle.bf16_bits_to_f64(q[ip[b]:ip[b + 1], h]))  # [n, d]
+                mask = torch.arange(L)[None, :] <= (L - n + torch.arange(n))[:, None]
+                ref = torch.nn.functional.scaled_dot_product_attention(Qd[None], Kd[None], Vd[None], attn_mask=mask[None],
+                                                                       scale=0.125)[0].numpy()
+                np.testing.assert_allclose(out[ip[b]:ip[b + 1], h], ref, rtol=1e-12, atol=1e-14)
+
+
+def test_prefill_first_token_of_a_fresh_sequence_sees_only_itself():
+    Hq, Hkv, d = 2, 1, 64
+    cache, ip, q = prefill_case(61, [19], [19], Hq, Hkv, d)
+    kp, vp = oracle.bf16_bits(cache.k_pages), oracle.bf16_bits(cache.v_pages)
+    out, lse = oracle.prefill_attn(q, ip, kp, vp, cache.page_table_host, np.array([19], np.int32), 0.125)
+    v0 = oracle.bf16_bits_to_f64(vp)[cache.page_table_host[0, 0], 0, 0]
+    for h in range(Hq):
+        assert np.array_equal(out[0, h], v0)
+    # the last query sees everything: equal to plain decode attention over the whole context
+    o1, _ = oracle.decode_attn(q[18][None], kp, vp, cache.page_table_host, np.array([19], np.int32), 0.125)
+    np.testing.assert_allclose(out[18], o1[0], rtol=1e-13)
+    # future tokens never leak: changing the last token's K/V leaves every earlier row untouched
+    kp2, vp2 = kp.copy(), vp.copy()
+    page = cache.page_table_host[0, 1]
+    kp2[page, :, 2] = bf16(np.full((Hkv, d), 3.0)); vp2[page, :, 2] = bf16(np.full((Hkv, d), -5.0))  # token 18
+    out2, _ = oracle.prefill_attn(q, ip, kp2, vp2, cache.page_table_host, np.array([19], np.int32), 0.125)
+    assert np.array_equal(out2[:18], out[:18]) and not np.array_equal(out2[18], out[18])
+
+
+def test_multi_token_append_then_prefill_matches_token_by_token_decode():
+    """Appending a turn at once and prefilling equals appending one token at a time and decoding."""
+    Hq, Hkv, d = 4, 1, 64
+    lens0 = np.array([30, 0, 16], np.int32)
+    q_lens = np.array([5, 18, 16], np.int32)
+    cache = wl.build_paged_cache(lens0, Hkv, d, seed=62, reserve_tokens=20)
+    ip = np.concatenate([[0], np.cumsum(q_lens)]).astype(np.int32)
+    total = int(ip[-1])
+    kn = oracle.bf16_bits(wl.random_bf16((total, Hkv, d), 63))
+    vn = oracle.bf16_bits(wl.random_bf16((total, Hkv, d), 64))
+    q = oracle.bf16_bits(wl.random_bf16((total, Hq, d), 65))
+    kp, vp = oracle.bf16_bits(cache.k_pages).copy(), oracle.bf16_bits(cache.v_pages).copy()
+    lens = lens0.copy()
+    assert oracle.kv_append_tokens(kn, vn, ip, kp, vp, cache.page_table_host, lens) == 0
+    assert np.array_equal(lens, lens0 + q_lens)
+    out, _ = oracle.prefill_attn(q, ip, kp, vp, cache.page_table_host, lens, 0.125)
+    # token by token with the single-token append and the decode definition
+    kp1, vp1 = oracle.bf16_bits(cache.k_pages).copy(), oracle.bf16_bits(cache.v_pages).copy()
+    for b in range(3):
+        cur = np.array([lens0[b]], np.int32)
+        for i in range(q_lens[b]):
+            r = ip[b] + i
+            oracle.kv_append(kn[r][None], vn[r][None], kp1, vp1, cache.page_table_host[b][None], cur)
+            o1, _ = oracle.decode_attn(q[r][None], kp1, vp1, cache.page_table_host[b][None], cur, 0.125)
+            np.testing.assert_allclose(out[r], o1[0], rtol=1e-13, atol=1e-15)
+    assert np.array_equal(kp, kp1) and np.array_equal(vp, vp1)
