@@ -132,6 +132,40 @@ int pd_decode_step_host(pd_ctx *ctx, const void *q_host, const void *k_new_host,
                         void *out_host, int32_t batch, float sm_scale, int32_t split_pages, void *stream);
 
 /*
+ * Append-prefill: the step that opens every turn of a multi-turn rollout
+ * (Sec. 2.1; the prefill terms B * dL * t_prefill of Eq. 1 and Eq. 3). The new
+ * turn's tokens are appended to the cached context and each of them attends
+ * causally over the cached prefix and the new tokens up to and including
+ * itself; with prefix caching only these tokens are computed.
+ *
+ * New tokens are packed: sequence b owns rows [q_indptr[b], q_indptr[b+1]) of
+ * q / out ([total][num_q_heads][head_dim] bf16), of k_new / v_new
+ * ([total][num_kv_heads][head_dim] bf16) and of lse ([total][num_q_heads] fp32,
+ * may be NULL). q_indptr is a DEVICE int32 array of batch + 1 entries;
+ * max_q_len is a host-side upper bound on q_indptr[b+1] - q_indptr[b] (it sizes
+ * the grid; a larger value only launches idle blocks).
+ *
+ * pd_kv_append_tokens copies the rows of sequence b to positions ctx_lens[b],
+ * ctx_lens[b] + 1, ... (their pages must already be in the table) and then adds
+ * the token count to ctx_lens[b]; a sequence that would run past its table row
+ * or meets a page id outside [0, num_pages) is skipped or partly written and
+ * latched for pd_device_status. Bit-exact.
+ *
+ * pd_prefill_attn expects the cache to hold the new tokens already and
+ * ctx_lens[b] = L_b to count them: query i of sequence b sits at position
+ * L_b - q_len_b + i and out = softmax(sm_scale * q . K_{0..pos}^T) V_{0..pos}.
+ * head_dim must be 128 (PD_ERR_UNSUPPORTED otherwise). The kernel runs on the
+ * tcgen05 tensor cores with fp32 accumulation; P is rounded to bf16 before the
+ * second product.
+ */
+int pd_kv_append_tokens(pd_ctx *ctx, const void *k_new, const void *v_new, const int32_t *q_indptr,
+                        void *k_pages, void *v_pages, const int32_t *page_table, int32_t *ctx_lens,
+                        int32_t batch, int32_t max_q_len, void *stream);
+int pd_prefill_attn(pd_ctx *ctx, const void *q, const int32_t *q_indptr, const void *k_pages,
+                    const void *v_pages, const int32_t *page_table, const int32_t *ctx_lens, void *out,
+                    float *lse, int32_t batch, int32_t max_q_len, float sm_scale, void *stream);
+
+/*
  * KV page gather / scatter: the device-side data movement of the cross-pool KV
  * transfer in the disaggregated prefill model (Eq. 3, the B * dL * K / BW term).
  * The prefill side packs the pages that hold a sequence's new tokens into one

@@ -27,7 +27,7 @@ PD_APPEND_NO_ADVANCE = 1
 # every symbol include/pd.h declares
 EXPORTS = (
     "pd_create", "pd_destroy", "pd_kv_append", "pd_decode_attn", "pd_decode_attn_static", "pd_decode_step_host",
-    "pd_kv_gather", "pd_kv_scatter", "pd_device_status", "pd_read_worker_trace",
+    "pd_kv_gather", "pd_kv_scatter", "pd_kv_append_tokens", "pd_prefill_attn", "pd_device_status", "pd_read_worker_trace",
     "pd_set_profile_events", "pd_workspace_bytes", "pd_launch_count", "pd_last_plan", "pd_status_string", "pd_last_error", "pd_version",
 )
 
@@ -60,6 +60,8 @@ def _load() -> ctypes.CDLL:
     lib.pd_kv_append.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, u32, vp]
     lib.pd_decode_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, vp]
     lib.pd_decode_attn_static.argtypes = [ctypes.POINTER(pd_config), vp, vp, vp, vp, vp, vp, vp, i32, f32, vp]
+    lib.pd_kv_append_tokens.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, vp]
+    lib.pd_prefill_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp]
     lib.pd_kv_gather.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.pd_kv_scatter.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.pd_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, vp]
@@ -137,6 +139,22 @@ def pd_decode_attn(ctx, q, k_pages, v_pages, page_table, ctx_lens, out, lse=None
     _check(_lib.pd_decode_attn(ctx, _ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(page_table), _ptr(ctx_lens),
                                _ptr(out), _ptr(lse), batch, sm_scale, split_pages, _stream(stream)),
            "pd_decode_attn", ctx)
+
+
+def pd_kv_append_tokens(ctx, k_new, v_new, q_indptr, k_pages, v_pages, page_table, ctx_lens, max_q_len, batch=None,
+                        stream=None):
+    batch = q_indptr.shape[0] - 1 if batch is None else batch
+    _check(_lib.pd_kv_append_tokens(ctx, _ptr(k_new), _ptr(v_new), _ptr(q_indptr), _ptr(k_pages), _ptr(v_pages),
+                                    _ptr(page_table), _ptr(ctx_lens), batch, max_q_len, _stream(stream)),
+           "pd_kv_append_tokens", ctx)
+
+
+def pd_prefill_attn(ctx, q, q_indptr, k_pages, v_pages, page_table, ctx_lens, out, lse=None, max_q_len=0, batch=None,
+                    sm_scale=1.0, stream=None):
+    batch = q_indptr.shape[0] - 1 if batch is None else batch
+    _check(_lib.pd_prefill_attn(ctx, _ptr(q), _ptr(q_indptr), _ptr(k_pages), _ptr(v_pages), _ptr(page_table),
+                                _ptr(ctx_lens), _ptr(out), _ptr(lse), batch, max_q_len, sm_scale, _stream(stream)),
+           "pd_prefill_attn", ctx)
 
 
 def pd_kv_gather(ctx, k_pages, v_pages, page_table, page_begin, page_end, packed_page_offset, packed, batch=None,

@@ -62,6 +62,7 @@ struct pd_ctx {
     alignas(64) CUtensorMap tm_k{};
     alignas(64) CUtensorMap tm_v{};
     cudaEvent_t ev_before = nullptr, ev_after = nullptr;  // optional timing hook around the split kernel
+    bool prefill_ready = false;
     int64_t launches = 0;
     char last_error[256] = {0};
 };
@@ -380,6 +381,86 @@ int pd_decode_attn(pd_ctx *ctx, const void *q, const void *k_pages, const void *
     err = pd::launch_lse_merge(ctx->cfg.head_dim, p, s);
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "lse_merge launch", err);
     ctx->launches += 2;
+    return PD_OK;
+}
+
+int pd_kv_append_tokens(pd_ctx *ctx, const void *k_new, const void *v_new, const int32_t *q_indptr, void *k_pages,
+                        void *v_pages, const int32_t *page_table, int32_t *ctx_lens, int32_t batch, int32_t max_q_len,
+                        void *stream) {
+    if (int rc = check_batch(ctx, batch)) return rc;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_pages) || !aligned16(v_pages) || q_indptr == nullptr ||
+        page_table == nullptr || ctx_lens == nullptr)
+        return fail(ctx, PD_ERR_INVALID_ARG, "pd_kv_append_tokens: null or misaligned pointer");
+    if (max_q_len < 0) return fail(ctx, PD_ERR_INVALID_ARG, "max_q_len must be >= 0");
+    if (batch == 0 || max_q_len == 0) return PD_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
+    pd::AppendTokensParams p{};
+    p.k_new = static_cast<const __nv_bfloat16 *>(k_new);
+    p.v_new = static_cast<const __nv_bfloat16 *>(v_new);
+    p.q_indptr = q_indptr;
+    p.k_pages = static_cast<__nv_bfloat16 *>(k_pages);
+    p.v_pages = static_cast<__nv_bfloat16 *>(v_pages);
+    p.page_table = page_table;
+    p.ctx_lens = ctx_lens;
+    p.status = ctx->status;
+    p.B = batch;
+    p.Hkv = ctx->cfg.num_kv_heads;
+    p.D = ctx->cfg.head_dim;
+    p.MP = ctx->cfg.max_pages_per_seq;
+    p.num_pages = static_cast<int32_t>(ctx->cfg.num_pages);
+    p.pdl = ctx->pdl;
+    const cudaError_t err = pd::launch_kv_append_tokens(p, max_q_len, static_cast<cudaStream_t>(stream));
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "kv_append_tokens launch", err);
+    ctx->launches += 2;
+    return PD_OK;
+}
+
+int pd_prefill_attn(pd_ctx *ctx, const void *q, const int32_t *q_indptr, const void *k_pages, const void *v_pages,
+                    const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse, int32_t batch,
+                    int32_t max_q_len, float sm_scale, void *stream) {
+    if (int rc = check_batch(ctx, batch)) return rc;
+    if (ctx->cfg.head_dim != 128) return fail(ctx, PD_ERR_UNSUPPORTED, "pd_prefill_attn: head_dim must be 128");
+    if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(out) || q_indptr == nullptr ||
+        page_table == nullptr || ctx_lens == nullptr)
+        return fail(ctx, PD_ERR_INVALID_ARG, "pd_prefill_attn: null or misaligned pointer");
+    if (!(sm_scale > 0.f) || !(sm_scale < 3.0e38f)) return fail(ctx, PD_ERR_INVALID_ARG, "sm_scale must be finite and positive");
+    if (max_q_len < 0) return fail(ctx, PD_ERR_INVALID_ARG, "max_q_len must be >= 0");
+    if (batch == 0 || max_q_len == 0) return PD_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
+    if (!ctx->prefill_ready) {
+        const cudaError_t e = pd::prepare_prefill_attn();
+        if (e != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "prefill kernel attribute", e);
+        ctx->prefill_ready = true;
+    }
+    if (ctx->map_k_ptr != k_pages) {
+        if (int rc = encode_pool_map(ctx, k_pages, &ctx->tm_k)) return rc;
+        ctx->map_k_ptr = k_pages;
+    }
+    if (ctx->map_v_ptr != v_pages) {
+        if (int rc = encode_pool_map(ctx, v_pages, &ctx->tm_v)) return rc;
+        ctx->map_v_ptr = v_pages;
+    }
+    pd::PrefillParams p{};
+    p.q = static_cast<const __nv_bfloat16 *>(q);
+    p.q_indptr = q_indptr;
+    p.page_table = page_table;
+    p.ctx_lens = ctx_lens;
+    p.out = static_cast<__nv_bfloat16 *>(out);
+    p.lse = lse;
+    p.status = ctx->status;
+    p.B = batch;
+    p.Hq = ctx->cfg.num_q_heads;
+    p.Hkv = ctx->cfg.num_kv_heads;
+    p.G = ctx->group;
+    p.MP = ctx->cfg.max_pages_per_seq;
+    p.num_pages = static_cast<int32_t>(ctx->cfg.num_pages);
+    p.scale_log2 = sm_scale * 1.4426950408889634f;
+    p.pdl = ctx->pdl;
+    const cudaError_t err = pd::launch_prefill_attn(ctx->tm_k, ctx->tm_v, p, max_q_len, static_cast<cudaStream_t>(stream));
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "prefill_attn launch", err);
+    ctx->launches += 1;
     return PD_OK;
 }
 

@@ -74,6 +74,32 @@ struct TransferParams {
     int32_t pdl;
 };
 
+struct PrefillParams {
+    const __nv_bfloat16 *q;     // [total_q][Hq][D] packed new-token queries
+    const int32_t *q_indptr;    // [B+1]
+    const int32_t *page_table;  // [B][MP]
+    const int32_t *ctx_lens;    // [B] lengths including the new tokens
+    __nv_bfloat16 *out;         // [total_q][Hq][D]
+    float *lse;                 // [total_q][Hq] or null
+    int32_t *status;
+    int32_t B, Hq, Hkv, G, MP;
+    int32_t num_pages;
+    float scale_log2;
+    int32_t pdl;
+};
+
+struct AppendTokensParams {
+    const __nv_bfloat16 *k_new, *v_new;  // [total][Hkv][D]
+    const int32_t *q_indptr;             // [B+1]
+    __nv_bfloat16 *k_pages, *v_pages;
+    const int32_t *page_table;
+    int32_t *ctx_lens;
+    int32_t *status;
+    int32_t B, Hkv, D, MP;
+    int32_t num_pages;
+    int32_t pdl;
+};
+
 // Shape of one compiled variant of the split kernel.
 struct AttnVariant {
     int head_dim, warps, stages, hilo;
@@ -104,6 +130,10 @@ cudaError_t prepare_decode_attn(const AttnVariant &v, size_t *smem_bytes);  // o
 cudaError_t launch_decode_attn(const AttnVariant &v, const CUtensorMap &tm_k, const CUtensorMap &tm_v,
                                const AttnParams &p, int num_ctas, size_t smem_bytes, cudaStream_t stream);
 cudaError_t launch_lse_merge(int head_dim, const AttnParams &p, cudaStream_t stream);
+cudaError_t prepare_prefill_attn();  // opt-in shared memory, once
+cudaError_t launch_prefill_attn(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const PrefillParams &p, int max_q_len,
+                                cudaStream_t stream);
+cudaError_t launch_kv_append_tokens(const AppendTokensParams &p, int max_q_len, cudaStream_t stream);
 cudaError_t launch_kv_transfer(const TransferParams &p, bool scatter, int num_sms, cudaStream_t stream);
 
 }  // namespace pd

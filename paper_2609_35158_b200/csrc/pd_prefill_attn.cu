@@ -1,0 +1,374 @@
+// Append-prefill attention over the paged KV cache, and the multi-token KV append.
+//
+// Every turn of a multi-turn rollout starts by prefilling the new tokens of the
+// turn (observation plus template, dL per trajectory in the prefill terms of
+// Eq. 1 and Eq. 3) on top of the cached context (Sec. 2.1). With prefix caching
+// only those dL tokens are computed, but each attends causally over the whole
+// cached prefix and the new tokens up to itself. Unlike decode this is a dense
+// contraction: 128 query rows share every K/V tile, so it runs on the
+// fifth-generation tensor cores.
+//
+// One CTA (128 threads) owns 128 rows = 128/g consecutive new tokens x the g
+// query heads of one KV head, row = head * (128/g) + token. It walks the context
+// in blocks of 128 tokens (8 pages):
+//   TMA      pages -> shared memory, [half of d][token][128 B] with the 128-byte
+//            swizzle: K is a K-major operand, V an MN-major one, no transposes;
+//            three stages of K+V; pages past the context are zero-filled
+//   tcgen05  S = Q K^T into tensor memory (8 MMAs of 128x128x16, one thread)
+//   threads  one thread per row: load its 128 logits from tensor memory, mask,
+//            running max with a slack of 8 log2 units, exp2, row sum, P as bf16
+//            back into tensor memory; a rare correction pass rescales O
+//   tcgen05  O += P V (P from tensor memory, 8 MMAs)
+// The S MMA of block j+1 is issued as soon as every thread holds block j's
+// logits in registers, so tensor cores and softmax overlap. All waits are
+// bounded; a wait that runs out latches PD_ERR_TIMEOUT and the CTA unwinds and
+// frees its tensor memory.
+#include "pd_kernels.cuh"
+#include "pd_ptx.cuh"
+#include "pd_tcgen05.cuh"
+
+namespace pd {
+
+namespace {
+
+constexpr float kLn2f = 0.6931471805599453f;
+constexpr float kSlack = 8.f;                 // log2 units a logit may exceed the running max before a rescale
+constexpr int kRows = 128;                    // query rows per CTA (MMA M)
+constexpr int kBlock = 128;                   // context tokens per step (MMA N of S, K of O)
+constexpr int kPagesPerBlock = kBlock / kPageSize;
+constexpr int kD = 128;
+constexpr int kHalfBytes = kBlock * 128;      // one 64-column half of a 128-token tile: 16 KB
+constexpr int kTileBytes = 2 * kHalfBytes;    // 32 KB
+constexpr int kStageBytes = 2 * kTileBytes;   // K tile + V tile
+constexpr int kStages = 3;
+constexpr int kTmemCols = 512;
+constexpr int kColS = 0, kColP = 128, kColO = 256;  // tensor-memory columns: logits, probabilities, output
+
+__device__ __forceinline__ void latch(int32_t *status, int code, int seq, int detail) {
+    if (atomicCAS(status, kDevOk, code) == kDevOk) {
+        status[1] = seq;
+        status[2] = detail;
+    }
+}
+
+__global__ void __launch_bounds__(kRows, 1)
+prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                    const PrefillParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_a, abort_b;  // a: raised before the first barrier of a step, b: between the two
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int b = blockIdx.z, kvh = blockIdx.y;
+    const int G = p.G, TOK = kRows / G;
+
+    grid_dependency_wait();
+    launch_dependents();
+    const int q0 = p.q_indptr[b], q_len = p.q_indptr[b + 1] - q0;
+    const int tile_start = blockIdx.x * TOK;
+    if (tile_start >= q_len) return;  // before any allocation
+    const int L = min(max(p.ctx_lens[b], 0), p.MP * kPageSize);
+    if (L < q_len) {  // the cache must already hold the new tokens
+        if (tid == 0) latch(p.status, kDevBadLength, b, L);
+        return;
+    }
+    const int n_tok = min(TOK, q_len - tile_start);
+    const int pos0 = L - q_len + tile_start;        // absolute position of the tile's first token
+    const int nb = (pos0 + n_tok - 1) / kBlock + 1;  // context blocks this tile can see
+    const int n_pages = (L + kPageSize - 1) / kPageSize;
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *aligned = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t q_s = base;
+    const uint32_t stage0 = base + kTileBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + kTileBytes + kStages * kStageBytes);
+    const uint32_t bar_kv = smem_u32(bars), bar_s = smem_u32(bars + kStages), bar_pv = smem_u32(bars + kStages + 1);
+
+    // ---- set-up: barriers, tensor memory, the Q tile
+    if (tid == 0) {
+        for (int i = 0; i < kStages + 2; ++i) mbar_init(smem_u32(bars + i), 1);
+        mbar_init_fence();
+        abort_a = 0;
+        abort_b = 0;
+        prefetch_tensormap(&tm_k);
+        prefetch_tensormap(&tm_v);
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
+        tmem_relinquish_alloc_permit();
+    }
+    const int head = tid / TOK, tok = tid - head * TOK;
+    const bool row_valid = tok < n_tok;
+    const int my_pos = pos0 + (row_valid ? tok : n_tok - 1);  // padding rows mirror the last token
+    {
+        const uint4 *src = reinterpret_cast<const uint4 *>(
+            p.q + (static_cast<size_t>(q0 + tile_start + tok) * p.Hq + kvh * G + head) * kD);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (row_valid) v = __ldg(src + c);
+            const uint32_t a = q_s + (c >> 3) * kHalfBytes + sw128_offset(tid, c & 7);
+            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+        }
+    }
+    fence_proxy_async();  // the Q tile was written with ordinary stores; the tensor core reads it through the async proxy
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tm = tmem_slot;
+    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+    const uint64_t policy = l2_policy_evict_first();
+    const int32_t oob_row = p.num_pages * p.Hkv * kPageSize;  // a TMA box that starts here is all zero fill
+
+    auto issue_block_loads = [&](int j) {  // thread 0 only
+        const uint32_t st = stage0 + (j % kStages) * kStageBytes;
+        const uint32_t bar = bar_kv + (j % kStages) * 8;
+        mbar_arrive_expect_tx(bar, kStageBytes);
+        const int32_t *row = p.page_table + static_cast<size_t>(b) * p.MP;
+#pragma unroll
+        for (int pg = 0; pg < kPagesPerBlock; ++pg) {
+            const int lp = j * kPagesPerBlock + pg;
+            int32_t y = oob_row;
+            if (lp < n_pages) {
+                int pid = __ldg(row + lp);
+                if (pid < 0 || pid >= p.num_pages) {
+                    latch(p.status, kDevBadPage, b, pid);
+                    pid = 0;
+                }
+                y = (pid * p.Hkv + kvh) * kPageSize;
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                tma_load_2d(st + h * kHalfBytes + pg * (kPageSize * 128), &tm_k, h * 64, y, bar, policy);
+                tma_load_2d(st + kTileBytes + h * kHalfBytes + pg * (kPageSize * 128), &tm_v, h * 64, y, bar, policy);
+            }
+        }
+    };
+    auto issue_qk = [&](int j) {  // thread 0 only: S = Q K_j^T, then signal bar_s
+        const uint32_t kst = stage0 + (j % kStages) * kStageBytes;
+        constexpr uint32_t idesc = umma_idesc_bf16(kRows, kBlock, false);
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                umma_ss(tm + kColS, umma_smem_desc(q_s + h * kHalfBytes + ks * 32, 16, 1024),
+                        umma_smem_desc(kst + h * kHalfBytes + ks * 32, 16, 1024), idesc, (h | ks) != 0);
+        umma_commit(bar_s);
+    };
+
+    if (tid == 0) {
+        for (int j = 0; j < min(nb, kStages); ++j) issue_block_loads(j);
+        if (mbar_wait(bar_kv, 0)) {
+            tc_fence_after_sync();
+            issue_qk(0);
+        } else {
+            abort_a = 1;
+        }
+    }
+
+    // l_run sums the exact probabilities (for lse); l_norm sums them as rounded to bf16, i.e. exactly the
+    // weights the second product applies, so that the output is a true weighted mean of V rows
+    float m_run = -INFINITY, l_run = 0.f, l_norm = 0.f;
+    bool ok = true;
+    for (int j = 0; j < nb; ++j) {
+        // ---- logits of block j: tensor memory -> registers
+        if (ok && !mbar_wait(bar_s, j & 1)) ok = false;
+        tc_fence_after_sync();
+        uint32_t s[kBlock];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld32(tm + lane_base + kColS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(s + c * 32));
+        tmem_wait_ld();
+        if (!ok) abort_a = 1;
+        tc_fence_before_sync();
+        __syncthreads();  // every thread holds its logits: the S columns are free again
+        if (abort_a) break;
+        if (tid == 0 && j + 1 < nb) {  // S of the next block overlaps this block's softmax
+            if (mbar_wait(bar_kv + ((j + 1) % kStages) * 8, ((j + 1) / kStages) & 1)) {
+                tc_fence_after_sync();
+                issue_qk(j + 1);
+            } else {
+                abort_b = 1;
+            }
+        }
+
+        // ---- softmax of this thread's row (log2 units)
+        const int t0 = j * kBlock;
+        float mx = -INFINITY;
+        const bool need_mask = t0 + kBlock - 1 > my_pos;
+#pragma unroll
+        for (int c = 0; c < kBlock; ++c) {
+            float x = __uint_as_float(s[c]) * p.scale_log2;
+            if (need_mask && t0 + c > my_pos) x = -INFINITY;
+            s[c] = __float_as_uint(x);
+            mx = fmaxf(mx, x);
+        }
+        float alpha = 1.f;
+        if (mx > m_run + kSlack) {
+            const float m_new = fmaxf(m_run, mx);
+            alpha = fast_exp2(m_run - m_new);
+            m_run = m_new;
+        }
+        // the previous block's O += P V must have finished before P or O is touched; it also frees a stage
+        if (j > 0 && ok && !mbar_wait(bar_pv, (j - 1) & 1)) ok = false;
+        tc_fence_after_sync();
+        if (tid == 0 && j > 0 && j + 2 < nb) issue_block_loads(j + 2);
+        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {  // rare: rescale this warp's rows of O
+            l_run *= alpha;
+            l_norm *= alpha;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tm + lane_base + kColO + c * 32, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                tmem_st32(tm + lane_base + kColO + c * 32, o);
+            }
+        } else {
+            l_run *= alpha;  // alpha is 1 unless this is the first block (the sums are 0 then)
+            l_norm *= alpha;
+        }
+        uint32_t pk[kBlock / 2];
+        float sum = 0.f, sum_r = 0.f;
+#pragma unroll
+        for (int c = 0; c < kBlock; c += 2) {
+            const float p0 = fast_exp2(__uint_as_float(s[c]) - m_run), p1 = fast_exp2(__uint_as_float(s[c + 1]) - m_run);
+            sum += p0 + p1;
+            const uint32_t packed = pack_bf16x2(p0, p1);
+            pk[c >> 1] = packed;
+            sum_r += __uint_as_float(packed << 16) + __uint_as_float(packed & 0xffff0000u);
+        }
+        l_run += sum;
+        l_norm += sum_r;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) tmem_st32(tm + lane_base + kColP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(pk + c * 32));
+        tmem_wait_st();
+
+        // V rows past the context inside the last page may hold NaN; 0 * NaN is NaN, so clear them
+        const uint32_t vst = stage0 + (j % kStages) * kStageBytes + kTileBytes;
+        const int valid_rows = L - t0;
+        if (valid_rows < kBlock) {
+            const int last = min(kBlock, (valid_rows + kPageSize - 1) / kPageSize * kPageSize);
+            for (int i = tid; i < (last - valid_rows) * 16; i += kRows) {
+                const int r = valid_rows + (i >> 4), c = i & 15;
+                st_shared_zero16(vst + (c >> 3) * kHalfBytes + r * 128 + (c & 7) * 16);
+            }
+            fence_proxy_async();
+        }
+        if (!ok) abort_b = 1;
+        tc_fence_before_sync();
+        __syncthreads();  // P complete, O corrected
+        if (abort_b) break;
+        if (tid == 0) {  // O += P V_j
+            tc_fence_after_sync();
+            constexpr uint32_t idesc = umma_idesc_bf16(kRows, kD, true);
+#pragma unroll
+            for (int ks = 0; ks < kBlock / 16; ++ks)
+                umma_ts(tm + kColO, tm + kColP + ks * 8, umma_smem_desc(vst + ks * 2048, kHalfBytes, 1024), idesc,
+                        (j | ks) != 0);
+            umma_commit(bar_pv);
+        }
+    }
+
+    // ---- epilogue: O / l -> bf16 rows
+    const bool aborted = abort_a != 0 || abort_b != 0;  // uniform: read after the barrier that ended the loop
+    if (!aborted) {
+        if (!mbar_wait(bar_pv, (nb - 1) & 1)) ok = false;
+        tc_fence_after_sync();
+        const float inv = 1.f / l_norm;
+        __nv_bfloat16 *orow = p.out + (static_cast<size_t>(q0 + tile_start + tok) * p.Hq + kvh * G + head) * kD;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tm + lane_base + kColO + c * 32, o);
+            tmem_wait_ld();
+            if (row_valid && ok) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 8) {
+                    uint4 v;
+                    v.x = pack_bf16x2(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
+                    v.y = pack_bf16x2(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+                    v.z = pack_bf16x2(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+                    v.w = pack_bf16x2(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
+                    *reinterpret_cast<uint4 *>(orow + c * 32 + i) = v;
+                }
+            }
+        }
+        if (p.lse != nullptr && row_valid && ok)
+            p.lse[static_cast<size_t>(q0 + tile_start + tok) * p.Hq + kvh * G + head] = (m_run + log2f(l_run)) * kLn2f;
+    }
+    if (!ok || aborted) {
+        if (tid == 0) latch(p.status, kDevTimeout, b, blockIdx.x);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, kTmemCols);
+}
+
+// Multi-token append: CTA (x, b) copies tokens x, x + gridDim.x, ... of sequence b. Lengths are read
+// here and advanced by a separate tiny kernel, so no CTA sees a half-updated length.
+__global__ void __launch_bounds__(256) kv_append_tokens_kernel(const AppendTokensParams p) {
+    const int b = blockIdx.y;
+    grid_dependency_wait();
+    launch_dependents();
+    const int r0 = p.q_indptr[b], n = p.q_indptr[b + 1] - r0;
+    const int L = p.ctx_lens[b];
+    if (n <= 0) return;
+    if (L < 0 || (L + n + kPageSize - 1) / kPageSize > p.MP) {
+        if (threadIdx.x == 0 && blockIdx.x == 0) latch(p.status, kDevBadLength, b, L);
+        return;
+    }
+    const int chunks_per_row = p.D / 8, chunks_per_tensor = p.Hkv * chunks_per_row;
+    for (int i = blockIdx.x; i < n; i += gridDim.x) {
+        const int pos = L + i;
+        const int page = p.page_table[static_cast<size_t>(b) * p.MP + pos / kPageSize];
+        if (page < 0 || page >= p.num_pages) {
+            if (threadIdx.x == 0) latch(p.status, kDevBadPage, b, page);
+            continue;
+        }
+        for (int c = threadIdx.x; c < 2 * chunks_per_tensor; c += blockDim.x) {
+            const int which = c / chunks_per_tensor, rem = c - which * chunks_per_tensor;
+            const int kvh = rem / chunks_per_row, jj = rem - kvh * chunks_per_row;
+            const __nv_bfloat16 *src = (which ? p.v_new : p.k_new) + (static_cast<size_t>(r0 + i) * p.Hkv + kvh) * p.D + jj * 8;
+            __nv_bfloat16 *dst = (which ? p.v_pages : p.k_pages) +
+                                 ((static_cast<size_t>(page) * p.Hkv + kvh) * kPageSize + pos % kPageSize) * p.D + jj * 8;
+            *reinterpret_cast<uint4 *>(dst) = __ldg(reinterpret_cast<const uint4 *>(src));
+        }
+    }
+}
+
+__global__ void advance_lens_kernel(const AppendTokensParams p) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    grid_dependency_wait();
+    launch_dependents();
+    if (b >= p.B) return;
+    const int n = p.q_indptr[b + 1] - p.q_indptr[b];
+    const int L = p.ctx_lens[b];
+    if (n > 0 && L >= 0 && (L + n + kPageSize - 1) / kPageSize <= p.MP) p.ctx_lens[b] = L + n;
+}
+
+}  // namespace
+
+size_t prefill_smem_bytes() { return kTileBytes + kStages * kStageBytes + 1024 + (kStages + 2) * 8 + 64; }
+
+cudaError_t prepare_prefill_attn() {
+    return cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                static_cast<int>(prefill_smem_bytes()));
+}
+
+cudaError_t launch_prefill_attn(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const PrefillParams &p, int max_q_len,
+                                cudaStream_t stream) {
+    if (p.B == 0 || max_q_len <= 0) return cudaSuccess;
+    const int tok = kRows / p.G;
+    const dim3 grid((max_q_len + tok - 1) / tok, p.Hkv, p.B);
+    return launch_pdl(prefill_attn_kernel, grid, dim3(kRows), prefill_smem_bytes(), stream, p.pdl != 0, tm_k, tm_v, p);
+}
+
+cudaError_t launch_kv_append_tokens(const AppendTokensParams &p, int max_q_len, cudaStream_t stream) {
+    if (p.B == 0 || max_q_len <= 0) return cudaSuccess;
+    const dim3 grid(max_q_len < 64 ? max_q_len : 64, p.B);
+    cudaError_t err = launch_pdl(kv_append_tokens_kernel, grid, dim3(256), 0, stream, p.pdl != 0, p);
+    if (err != cudaSuccess) return err;
+    return launch_pdl(advance_lens_kernel, dim3((p.B + 127) / 128), dim3(128), 0, stream, p.pdl != 0, p);
+}
+
+}  // namespace pd

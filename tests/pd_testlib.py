@@ -23,9 +23,15 @@ def error_metrics(out_gpu_bf16: torch.Tensor, out_ref: np.ndarray):
     return max_abs, float(rel.max()) if rel.size else 0.0
 
 
-def assert_parity(out_gpu_bf16, out_ref, what=""):
+def assert_parity(out_gpu_bf16, out_ref, what="", scale_abs_by_magnitude=False):
+    """``scale_abs_by_magnitude``: the absolute bound becomes 1e-2 * max(1, |ref|) per element. bf16 cannot
+    hold a value of magnitude 4 to better than 1.6e-2, so outputs that are single V rows (contexts of a
+    handful of tokens, as the first queries of a prefill see) need the bound to follow the magnitude."""
     assert torch.isfinite(out_gpu_bf16.float()).all(), f"{what}: non-finite output"
     max_abs, rel = error_metrics(out_gpu_bf16, out_ref)
+    if scale_abs_by_magnitude:
+        got = out_gpu_bf16.detach().float().cpu().numpy().astype(np.float64)
+        max_abs = float((np.abs(got - out_ref) / np.maximum(1.0, np.abs(out_ref))).max())
     assert max_abs <= MAX_ABS_TOL, f"{what}: max abs error {max_abs:.3e} > {MAX_ABS_TOL}"
     assert rel <= REL_L2_TOL, f"{what}: per-row relative L2 {rel:.3e} > {REL_L2_TOL}"
     return max_abs, rel
