@@ -464,6 +464,133 @@ def run_transfer(args):
     print(json.dumps(result), flush=True)
 
 
+# ------------------------------------------------------------------------------------------ prefill op
+
+def run_prefill(args):
+    """Append-prefill of one turn: multi-token append + causal attention of the new tokens over prefix + themselves.
+
+    Workload: Qwen3-8B geometry, 32 sequences whose cached prefix is U{2048..16384} tokens and whose new turn
+    is U{256..2048} tokens. Value = attention TFLOP/s of the whole step (append + attention), where the
+    attention of query i at position pos costs 4 * H_q * d * (pos + 1) flops."""
+    import torch
+
+    import oracle
+    import paper_2609_35158_b200 as pd
+    import workloads as wl
+
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    w = wl.WORKLOADS[1]
+    K, W = args.steps, args.warmup
+    B = 32
+    rng = np.random.Generator(np.random.PCG64(505))
+    q_lens = rng.integers(256, 2048, size=B, endpoint=True).astype(np.int32)
+    prefix = rng.integers(2048, 16384, size=B, endpoint=True).astype(np.int32)
+    ip = np.concatenate([[0], np.cumsum(q_lens)]).astype(np.int32)
+    total_q = int(ip[-1])
+    cache = wl.build_paged_cache(prefix, w.num_kv_heads, w.head_dim, seed=51, device=dev,
+                                 reserve_tokens=int(q_lens.max()))
+    ctx = pd.pd_create(w.num_q_heads, w.num_kv_heads, w.head_dim, 16, B, cache.page_table.shape[1], cache.num_pages, 0)
+    q = wl.random_bf16((total_q, w.num_q_heads, w.head_dim), 52, dev)
+    kn = wl.random_bf16((total_q, w.num_kv_heads, w.head_dim), 53, dev)
+    vn = wl.random_bf16((total_q, w.num_kv_heads, w.head_dim), 54, dev)
+    out = torch.empty_like(q)
+    ip_dev = torch.from_numpy(ip).to(dev)
+    prefix_dev = torch.from_numpy(prefix).to(dev)
+    max_q = int(q_lens.max())
+    flops = float(sum(4.0 * w.num_q_heads * w.head_dim * (int(n) * int(p0) + int(n) * (int(n) + 1) / 2)
+                      for n, p0 in zip(q_lens, prefix)))
+
+    def step():
+        cache.ctx_lens.copy_(prefix_dev)  # every step prefills the same turn onto the same prefix
+        pd.pd_kv_append_tokens(ctx, kn, vn, ip_dev, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, max_q)
+        pd.pd_prefill_attn(ctx, q, ip_dev, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, out,
+                           max_q_len=max_q, sm_scale=w.sm_scale)
+
+    for _ in range(W):
+        step()
+    torch.cuda.synchronize()
+    assert pd.pd_device_status(ctx)[0] == 0
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    t0, t1 = ev(), ev()
+    hooked = [i for i in range(K) if i % 4 == min(2, K - 1)]
+    hb, ha = {i: ev() for i in hooked}, {i: ev() for i in hooked}
+    sampler = ClockSampler(0)
+    sampler.start()
+    t0.record()
+    for i in range(K):
+        if i in hb:
+            cache.ctx_lens.copy_(prefix_dev)
+            pd.pd_kv_append_tokens(ctx, kn, vn, ip_dev, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, max_q)
+            hb[i].record()
+            pd.pd_prefill_attn(ctx, q, ip_dev, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, out,
+                               max_q_len=max_q, sm_scale=w.sm_scale)
+            ha[i].record()
+        else:
+            step()
+    t1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    assert pd.pd_device_status(ctx)[0] == 0
+    ms = t0.elapsed_time(t1) / K
+    attn_ms = float(np.mean([hb[i].elapsed_time(ha[i]) for i in hooked]))
+
+    # host-buffer variant: q, k_new, v_new from pinned host memory, out back to the host, every step
+    hq, hk, hv = q.cpu().pin_memory(), kn.cpu().pin_memory(), vn.cpu().pin_memory()
+    hout = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+    e0, e1 = ev(), ev()
+    for i in range(W + K):
+        if i == W:
+            e0.record()
+        q.copy_(hq, non_blocking=True)
+        kn.copy_(hk, non_blocking=True)
+        vn.copy_(hv, non_blocking=True)
+        step()
+        hout.copy_(out, non_blocking=True)
+        torch.cuda.synchronize()
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1) / K
+
+    # CPU baseline: the oracle on a sample of query rows (first, middle, last of a few sequences)
+    cores = os.cpu_count() or 1
+    kp, vp = oracle.bf16_bits(cache.k_pages), oracle.bf16_bits(cache.v_pages)
+    lens_after = (prefix + q_lens).astype(np.int32)
+    nseq = 2
+    sub_ip = np.concatenate([[0], np.cumsum(q_lens[:nseq])]).astype(np.int32)
+    t = time.perf_counter()
+    oracle.prefill_attn(oracle.bf16_bits(q[:int(sub_ip[-1])]), sub_ip, kp, vp, cache.page_table_host[:nseq], lens_after[:nseq],
+                        w.sm_scale, nthreads=cores)
+    cpu_s = time.perf_counter() - t
+    cpu_flops = float(sum(4.0 * w.num_q_heads * w.head_dim * (int(n) * int(p0) + int(n) * (int(n) + 1) / 2)
+                          for n, p0 in zip(q_lens[:nseq], prefix[:nseq])))
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak, peak_kind = float(json.load(f)["bf16_tflops"]), "measured (cuBLAS bf16 burst)"
+    except Exception:
+        peak, peak_kind = 1590.0, "fallback"
+    achieved = flops / (attn_ms * 1e-3) / 1e12
+    result = {
+        "metric": "append-prefill attention TFLOP/s", "value": round(flops / (ms * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
+        "n_gpus": 1, "steps": K, "warmup": W, "ms_per_step": round(ms, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "one prefill turn, Qwen3-8B geometry (32/8 heads, d 128), 32 sequences, prefix U{2048..16384}, new tokens U{256..2048}",
+                   "new_tokens_total": total_q, "prefix_tokens_total": int(prefix.sum()), "flops_per_step": flops},
+        "clocks": clocks,
+        "e2e": {"value": round(flops / (e2e_ms * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
+                "h2d_bytes_per_step": int((hq.numel() + hk.numel() + hv.numel()) * 2), "d2h_bytes_per_step": int(hout.numel() * 2),
+                "ms_per_step": round(e2e_ms, 5)},
+        "gpu_launches": 3 * K,
+        "roofline": {"bound": "tensor", "kernel": "prefill_attn_kernel", "achieved": round(achieved, 2), "peak": peak,
+                     "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "avg_launch_ms": round(attn_ms, 5)},
+        "cpu_baseline": {"value": round(cpu_flops / cpu_s / 1e12, 5), "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+                         "sample": f"all query rows of the first {nseq} sequences ({int(sub_ip[-1])} new tokens), {cpu_s:.1f} s"},
+    }
+    pd.pd_destroy(ctx)
+    print(json.dumps(result), flush=True)
+
+
 # ------------------------------------------------------------------------------------------ reference arm
 
 def run_reference(args):
@@ -526,8 +653,9 @@ def main():
     ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--op", default="decode", choices=["decode", "kv_transfer"],
-                    help="decode = the headline decode step; kv_transfer = page gather + scatter")
+    ap.add_argument("--op", default="decode", choices=["decode", "kv_transfer", "prefill"],
+                    help="decode = the headline decode step; kv_transfer = page gather + scatter; "
+                         "prefill = one append-prefill turn")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
@@ -535,6 +663,8 @@ def main():
         run_reference(args)
     elif args.op == "kv_transfer":
         run_transfer(args)
+    elif args.op == "prefill":
+        run_prefill(args)
     else:
         run_cuda(args)
 

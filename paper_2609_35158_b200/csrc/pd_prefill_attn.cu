@@ -165,9 +165,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         }
     }
 
-    // l_run sums the exact probabilities (for lse); l_norm sums them as rounded to bf16, i.e. exactly the
-    // weights the second product applies, so that the output is a true weighted mean of V rows
-    float m_run = -INFINITY, l_run = 0.f, l_norm = 0.f;
+    float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
     for (int j = 0; j < nb; ++j) {
         // ---- logits of block j: tensor memory -> registers
@@ -190,17 +188,21 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             }
         }
 
-        // ---- softmax of this thread's row (log2 units)
+        // ---- softmax of this thread's row. Logits stay raw; sm_scale * log2(e) > 0 is folded into the
+        // exponent's FMA, so the row maximum can be taken on the raw values.
         const int t0 = j * kBlock;
         float mx = -INFINITY;
-        const bool need_mask = t0 + kBlock - 1 > my_pos;
+        if (t0 + kBlock - 1 > my_pos) {  // the block reaches past this row's position: mask by select
 #pragma unroll
-        for (int c = 0; c < kBlock; ++c) {
-            float x = __uint_as_float(s[c]) * p.scale_log2;
-            if (need_mask && t0 + c > my_pos) x = -INFINITY;
-            s[c] = __float_as_uint(x);
-            mx = fmaxf(mx, x);
+            for (int c = 0; c < kBlock; ++c) {
+                if (t0 + c > my_pos) s[c] = 0xff800000u;  // -inf
+                mx = fmaxf(mx, __uint_as_float(s[c]));
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < kBlock; c += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(s[c]), __uint_as_float(s[c + 1])));
         }
+        mx *= p.scale_log2;
         float alpha = 1.f;
         if (mx > m_run + kSlack) {
             const float m_new = fmaxf(m_run, mx);
@@ -213,7 +215,6 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         if (tid == 0 && j > 0 && j + 2 < nb) issue_block_loads(j + 2);
         if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {  // rare: rescale this warp's rows of O
             l_run *= alpha;
-            l_norm *= alpha;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t o[32];
@@ -224,21 +225,20 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 tmem_st32(tm + lane_base + kColO + c * 32, o);
             }
         } else {
-            l_run *= alpha;  // alpha is 1 unless this is the first block (the sums are 0 then)
-            l_norm *= alpha;
+            l_run *= alpha;  // alpha is 1 unless this is the first block (l_run is 0 then)
         }
         uint32_t pk[kBlock / 2];
-        float sum = 0.f, sum_r = 0.f;
+        float sum0 = 0.f, sum1 = 0.f;
+        const float neg_m = -m_run;
 #pragma unroll
         for (int c = 0; c < kBlock; c += 2) {
-            const float p0 = fast_exp2(__uint_as_float(s[c]) - m_run), p1 = fast_exp2(__uint_as_float(s[c + 1]) - m_run);
-            sum += p0 + p1;
-            const uint32_t packed = pack_bf16x2(p0, p1);
-            pk[c >> 1] = packed;
-            sum_r += __uint_as_float(packed << 16) + __uint_as_float(packed & 0xffff0000u);
+            const float p0 = fast_exp2(fmaf(__uint_as_float(s[c]), p.scale_log2, neg_m));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, neg_m));
+            sum0 += p0;
+            sum1 += p1;
+            pk[c >> 1] = pack_bf16x2(p0, p1);
         }
-        l_run += sum;
-        l_norm += sum_r;
+        l_run += sum0 + sum1;
 #pragma unroll
         for (int c = 0; c < 2; ++c) tmem_st32(tm + lane_base + kColP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(pk + c * 32));
         tmem_wait_st();
@@ -274,7 +274,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     if (!aborted) {
         if (!mbar_wait(bar_pv, (nb - 1) & 1)) ok = false;
         tc_fence_after_sync();
-        const float inv = 1.f / l_norm;
+        const float inv = 1.f / l_run;
         __nv_bfloat16 *orow = p.out + (static_cast<size_t>(q0 + tile_start + tok) * p.Hq + kvh * G + head) * kD;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
