@@ -10,17 +10,18 @@
 //
 // One CTA (128 threads) owns 128 rows = 128/g consecutive new tokens x the g
 // query heads of one KV head, row = head * (128/g) + token. It walks the context
-// in blocks of 128 tokens (8 pages):
+// in blocks of 64 tokens (4 pages):
 //   TMA      pages -> shared memory, [half of d][token][128 B] with the 128-byte
 //            swizzle: K is a K-major operand, V an MN-major one, no transposes;
-//            three stages of K+V; pages past the context are zero-filled
-//   tcgen05  S = Q K^T into tensor memory (8 MMAs of 128x128x16, one thread)
-//   threads  one thread per row: load its 128 logits from tensor memory, mask,
+//            two stages of K+V; pages past the context are zero-filled
+//   tcgen05  S = Q K^T into tensor memory (8 MMAs of 128x64x16, one thread)
+//   threads  one thread per row: load its 64 logits from tensor memory, mask,
 //            running max with a slack of 8 log2 units, exp2, row sum, P as bf16
 //            back into tensor memory; a rare correction pass rescales O
-//   tcgen05  O += P V (P from tensor memory, 8 MMAs)
+//   tcgen05  O += P V (P from tensor memory, 4 MMAs of 128x128x16)
 // The S MMA of block j+1 is issued as soon as every thread holds block j's
-// logits in registers, so tensor cores and softmax overlap. All waits are
+// logits in registers, and two CTAs share each SM (96 KB of shared memory, 256
+// tensor-memory columns each), so one CTA's softmax overlaps the other's MMAs. All waits are
 // bounded; a wait that runs out latches PD_ERR_TIMEOUT and the CTA unwinds and
 // frees its tensor memory.
 #include "pd_kernels.cuh"
@@ -34,15 +35,18 @@ namespace {
 constexpr float kLn2f = 0.6931471805599453f;
 constexpr float kSlack = 8.f;                 // log2 units a logit may exceed the running max before a rescale
 constexpr int kRows = 128;                    // query rows per CTA (MMA M)
-constexpr int kBlock = 128;                   // context tokens per step (MMA N of S, K of O)
+constexpr int kBlock = 64;                    // context tokens per step (MMA N of S, K of O)
 constexpr int kPagesPerBlock = kBlock / kPageSize;
 constexpr int kD = 128;
-constexpr int kHalfBytes = kBlock * 128;      // one 64-column half of a 128-token tile: 16 KB
-constexpr int kTileBytes = 2 * kHalfBytes;    // 32 KB
-constexpr int kStageBytes = 2 * kTileBytes;   // K tile + V tile
-constexpr int kStages = 3;
-constexpr int kTmemCols = 512;
-constexpr int kColS = 0, kColP = 128, kColO = 256;  // tensor-memory columns: logits, probabilities, output
+constexpr int kQHalfBytes = kRows * 128;      // one 64-column half of the 128-row Q tile: 16 KB
+constexpr int kQBytes = 2 * kQHalfBytes;
+constexpr int kHalfBytes = kBlock * 128;      // one 64-column half of a K or V tile of kBlock tokens
+constexpr int kTileBytes = 2 * kHalfBytes;
+constexpr int kStages = 2;                    // K ring and V ring have two tiles each
+// Two CTAs share an SM (96 KB of shared memory and 256 tensor-memory columns each): while one runs its
+// softmax on the CUDA cores the other's MMAs keep the tensor cores busy.
+constexpr int kTmemCols = 256;
+constexpr int kColS = 0, kColP = kBlock, kColO = 128;  // tensor-memory columns: logits, probabilities, output
 
 __device__ __forceinline__ void latch(int32_t *status, int code, int seq, int detail) {
     if (atomicCAS(status, kDevOk, code) == kDevOk) {
@@ -51,7 +55,7 @@ __device__ __forceinline__ void latch(int32_t *status, int code, int seq, int de
     }
 }
 
-__global__ void __launch_bounds__(kRows, 1)
+__global__ void __launch_bounds__(kRows, 2)
 prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                     const PrefillParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -79,13 +83,15 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *aligned = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t q_s = base;
-    const uint32_t stage0 = base + kTileBytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + kTileBytes + kStages * kStageBytes);
-    const uint32_t bar_kv = smem_u32(bars), bar_s = smem_u32(bars + kStages), bar_pv = smem_u32(bars + kStages + 1);
+    const uint32_t stage0 = base + kQBytes;
+    const uint32_t k_ring = stage0, v_ring = stage0 + kStages * kTileBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + kQBytes + 2 * kStages * kTileBytes);
+    const uint32_t bar_k = smem_u32(bars), bar_v = smem_u32(bars + kStages);
+    const uint32_t bar_s = smem_u32(bars + 2 * kStages), bar_pv = smem_u32(bars + 2 * kStages + 1);
 
     // ---- set-up: barriers, tensor memory, the Q tile
     if (tid == 0) {
-        for (int i = 0; i < kStages + 2; ++i) mbar_init(smem_u32(bars + i), 1);
+        for (int i = 0; i < 2 * kStages + 2; ++i) mbar_init(smem_u32(bars + i), 1);
         mbar_init_fence();
         abort_a = 0;
         abort_b = 0;
@@ -106,7 +112,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         for (int c = 0; c < 16; ++c) {
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
             if (row_valid) v = __ldg(src + c);
-            const uint32_t a = q_s + (c >> 3) * kHalfBytes + sw128_offset(tid, c & 7);
+            const uint32_t a = q_s + (c >> 3) * kQHalfBytes + sw128_offset(tid, c & 7);
             asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
         }
     }
@@ -119,10 +125,12 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     const uint64_t policy = l2_policy_evict_first();
     const int32_t oob_row = p.num_pages * p.Hkv * kPageSize;  // a TMA box that starts here is all zero fill
 
-    auto issue_block_loads = [&](int j) {  // thread 0 only
-        const uint32_t st = stage0 + (j % kStages) * kStageBytes;
-        const uint32_t bar = bar_kv + (j % kStages) * 8;
-        mbar_arrive_expect_tx(bar, kStageBytes);
+    // K and V travel separately: a K tile is free again as soon as its S MMA has completed, a V tile only
+    // after its O MMA, so K can be requested two blocks ahead
+    auto issue_tile_loads = [&](int j, const CUtensorMap *map, uint32_t ring, uint32_t bar0) {  // thread 0 only
+        const uint32_t st = ring + (j % kStages) * kTileBytes;
+        const uint32_t bar = bar0 + (j % kStages) * 8;
+        mbar_arrive_expect_tx(bar, kTileBytes);
         const int32_t *row = p.page_table + static_cast<size_t>(b) * p.MP;
 #pragma unroll
         for (int pg = 0; pg < kPagesPerBlock; ++pg) {
@@ -137,27 +145,28 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 y = (pid * p.Hkv + kvh) * kPageSize;
             }
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                tma_load_2d(st + h * kHalfBytes + pg * (kPageSize * 128), &tm_k, h * 64, y, bar, policy);
-                tma_load_2d(st + kTileBytes + h * kHalfBytes + pg * (kPageSize * 128), &tm_v, h * 64, y, bar, policy);
-            }
+            for (int h = 0; h < 2; ++h)
+                tma_load_2d(st + h * kHalfBytes + pg * (kPageSize * 128), map, h * 64, y, bar, policy);
         }
     };
     auto issue_qk = [&](int j) {  // thread 0 only: S = Q K_j^T, then signal bar_s
-        const uint32_t kst = stage0 + (j % kStages) * kStageBytes;
+        const uint32_t kst = k_ring + (j % kStages) * kTileBytes;
         constexpr uint32_t idesc = umma_idesc_bf16(kRows, kBlock, false);
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-                umma_ss(tm + kColS, umma_smem_desc(q_s + h * kHalfBytes + ks * 32, 16, 1024),
+                umma_ss(tm + kColS, umma_smem_desc(q_s + h * kQHalfBytes + ks * 32, 16, 1024),
                         umma_smem_desc(kst + h * kHalfBytes + ks * 32, 16, 1024), idesc, (h | ks) != 0);
         umma_commit(bar_s);
     };
 
     if (tid == 0) {
-        for (int j = 0; j < min(nb, kStages); ++j) issue_block_loads(j);
-        if (mbar_wait(bar_kv, 0)) {
+        for (int j = 0; j < min(nb, kStages); ++j) {
+            issue_tile_loads(j, &tm_k, k_ring, bar_k);
+            issue_tile_loads(j, &tm_v, v_ring, bar_v);
+        }
+        if (mbar_wait(bar_k, 0)) {
             tc_fence_after_sync();
             issue_qk(0);
         } else {
@@ -173,14 +182,16 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         tc_fence_after_sync();
         uint32_t s[kBlock];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld32(tm + lane_base + kColS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(s + c * 32));
+        for (int c = 0; c < kBlock / 32; ++c)
+            tmem_ld32(tm + lane_base + kColS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(s + c * 32));
         tmem_wait_ld();
         if (!ok) abort_a = 1;
         tc_fence_before_sync();
         __syncthreads();  // every thread holds its logits: the S columns are free again
         if (abort_a) break;
+        if (tid == 0 && j + kStages < nb) issue_tile_loads(j + kStages, &tm_k, k_ring, bar_k);  // S_j is done: its K tile is free
         if (tid == 0 && j + 1 < nb) {  // S of the next block overlaps this block's softmax
-            if (mbar_wait(bar_kv + ((j + 1) % kStages) * 8, ((j + 1) / kStages) & 1)) {
+            if (mbar_wait(bar_k + ((j + 1) % kStages) * 8, ((j + 1) / kStages) & 1)) {
                 tc_fence_after_sync();
                 issue_qk(j + 1);
             } else {
@@ -212,7 +223,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         // the previous block's O += P V must have finished before P or O is touched; it also frees a stage
         if (j > 0 && ok && !mbar_wait(bar_pv, (j - 1) & 1)) ok = false;
         tc_fence_after_sync();
-        if (tid == 0 && j > 0 && j + 2 < nb) issue_block_loads(j + 2);
+        if (tid == 0 && j > 0 && j - 1 + kStages < nb) issue_tile_loads(j - 1 + kStages, &tm_v, v_ring, bar_v);
         if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {  // rare: rescale this warp's rows of O
             l_run *= alpha;
 #pragma unroll
@@ -240,13 +251,17 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         }
         l_run += sum0 + sum1;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) tmem_st32(tm + lane_base + kColP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(pk + c * 32));
+        for (int c = 0; c < kBlock / 64; ++c)
+            tmem_st32(tm + lane_base + kColP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(pk + c * 32));
         tmem_wait_st();
 
         // V rows past the context inside the last page may hold NaN; 0 * NaN is NaN, so clear them
-        const uint32_t vst = stage0 + (j % kStages) * kStageBytes + kTileBytes;
+        const uint32_t vst = v_ring + (j % kStages) * kTileBytes;
+        const uint32_t bar_vj = bar_v + (j % kStages) * 8;
+        const uint32_t par_vj = (j / kStages) & 1;
         const int valid_rows = L - t0;
         if (valid_rows < kBlock) {
+            if (ok && !mbar_wait(bar_vj, par_vj)) ok = false;  // the tile must have landed before it is patched
             const int last = min(kBlock, (valid_rows + kPageSize - 1) / kPageSize * kPageSize);
             for (int i = tid; i < (last - valid_rows) * 16; i += kRows) {
                 const int r = valid_rows + (i >> 4), c = i & 15;
@@ -259,6 +274,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         __syncthreads();  // P complete, O corrected
         if (abort_b) break;
         if (tid == 0) {  // O += P V_j
+            if (!mbar_wait(bar_vj, par_vj)) abort_a = 1;  // seen by everyone after the next step's first barrier
             tc_fence_after_sync();
             constexpr uint32_t idesc = umma_idesc_bf16(kRows, kD, true);
 #pragma unroll
@@ -348,7 +364,7 @@ __global__ void advance_lens_kernel(const AppendTokensParams p) {
 
 }  // namespace
 
-size_t prefill_smem_bytes() { return kTileBytes + kStages * kStageBytes + 1024 + (kStages + 2) * 8 + 64; }
+size_t prefill_smem_bytes() { return kQBytes + 2 * kStages * kTileBytes + 1024 + (2 * kStages + 2) * 8 + 64; }
 
 cudaError_t prepare_prefill_attn() {
     return cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
