@@ -8,7 +8,7 @@
 // contraction: 128 query rows share every K/V tile, so it runs on the
 // fifth-generation tensor cores.
 //
-// One CTA (128 threads) owns 128 rows = 128/g consecutive new tokens x the g
+// One CTA (128 softmax threads + one issuing warp) owns 128 rows = 128/g consecutive new tokens x the g
 // query heads of one KV head, row = head * (128/g) + token. It walks the context
 // in blocks of 64 tokens (4 pages):
 //   TMA      pages -> shared memory, [half of d][token][128 B] with the 128-byte
@@ -19,8 +19,10 @@
 //            running max with a slack of 8 log2 units, exp2, row sum, P as bf16
 //            back into tensor memory; a rare correction pass rescales O
 //   tcgen05  O += P V (P from tensor memory, 4 MMAs of 128x128x16)
-// The S MMA of block j+1 is issued as soon as every thread holds block j's
-// logits in registers, and two CTAs share each SM (96 KB of shared memory, 256
+// A separate warp issues every TMA load and MMA, so the row threads never run
+// issue code or meet at a CTA barrier: they hand over through mbarriers (logits
+// read, probabilities written). The S MMA of block j+1 is issued as soon as
+// every row holds block j's logits in registers, and two CTAs share each SM (96 KB of shared memory, 256
 // tensor-memory columns each), so one CTA's softmax overlaps the other's MMAs. All waits are
 // bounded; a wait that runs out latches PD_ERR_TIMEOUT and the CTA unwinds and
 // frees its tensor memory.
@@ -34,7 +36,8 @@ namespace {
 
 constexpr float kLn2f = 0.6931471805599453f;
 constexpr float kSlack = 8.f;                 // log2 units a logit may exceed the running max before a rescale
-constexpr int kRows = 128;                    // query rows per CTA (MMA M)
+constexpr int kRows = 128;                    // query rows per CTA (MMA M), one softmax thread each
+constexpr int kThreads = kRows + 32;          // plus the warp whose first lane issues TMA and MMA
 constexpr int kBlock = 64;                    // context tokens per step (MMA N of S, K of O)
 constexpr int kPagesPerBlock = kBlock / kPageSize;
 constexpr int kD = 128;
@@ -55,12 +58,11 @@ __device__ __forceinline__ void latch(int32_t *status, int code, int seq, int de
     }
 }
 
-__global__ void __launch_bounds__(kRows, 2)
+__global__ void __launch_bounds__(kThreads, 2)
 prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                     const PrefillParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_slot;
-    __shared__ int abort_a, abort_b;  // a: raised before the first barrier of a step, b: between the two
     const int tid = threadIdx.x, warp = tid >> 5;
     const int b = blockIdx.z, kvh = blockIdx.y;
     const int G = p.G, TOK = kRows / G;
@@ -83,18 +85,20 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *aligned = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t q_s = base;
-    const uint32_t stage0 = base + kQBytes;
-    const uint32_t k_ring = stage0, v_ring = stage0 + kStages * kTileBytes;
+    const uint32_t k_ring = base + kQBytes, v_ring = k_ring + kStages * kTileBytes;
     uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + kQBytes + 2 * kStages * kTileBytes);
     const uint32_t bar_k = smem_u32(bars), bar_v = smem_u32(bars + kStages);
-    const uint32_t bar_s = smem_u32(bars + 2 * kStages), bar_pv = smem_u32(bars + 2 * kStages + 1);
+    const uint32_t bar_s = smem_u32(bars + 2 * kStages);          // S_j is in tensor memory (MMA commit)
+    const uint32_t bar_pv = smem_u32(bars + 2 * kStages + 1);     // O += P_j V_j has completed (MMA commit)
+    const uint32_t bar_s_read = smem_u32(bars + 2 * kStages + 2); // all 128 rows hold S_j in registers
+    const uint32_t bar_p_full = smem_u32(bars + 2 * kStages + 3); // all 128 rows wrote P_j
 
     // ---- set-up: barriers, tensor memory, the Q tile
     if (tid == 0) {
         for (int i = 0; i < 2 * kStages + 2; ++i) mbar_init(smem_u32(bars + i), 1);
+        mbar_init(bar_s_read, kRows);
+        mbar_init(bar_p_full, kRows);
         mbar_init_fence();
-        abort_a = 0;
-        abort_b = 0;
         prefetch_tensormap(&tm_k);
         prefetch_tensormap(&tm_v);
     }
@@ -102,10 +106,10 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
         tmem_relinquish_alloc_permit();
     }
-    const int head = tid / TOK, tok = tid - head * TOK;
+    const int head = (tid & (kRows - 1)) / TOK, tok = (tid & (kRows - 1)) - head * TOK;
     const bool row_valid = tok < n_tok;
     const int my_pos = pos0 + (row_valid ? tok : n_tok - 1);  // padding rows mirror the last token
-    {
+    if (tid < kRows) {
         const uint4 *src = reinterpret_cast<const uint4 *>(
             p.q + (static_cast<size_t>(q0 + tile_start + tok) * p.Hq + kvh * G + head) * kD);
 #pragma unroll
@@ -121,174 +125,171 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tm = tmem_slot;
-    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
-    const uint64_t policy = l2_policy_evict_first();
-    const int32_t oob_row = p.num_pages * p.Hkv * kPageSize;  // a TMA box that starts here is all zero fill
-
-    // K and V travel separately: a K tile is free again as soon as its S MMA has completed, a V tile only
-    // after its O MMA, so K can be requested two blocks ahead
-    auto issue_tile_loads = [&](int j, const CUtensorMap *map, uint32_t ring, uint32_t bar0) {  // thread 0 only
-        const uint32_t st = ring + (j % kStages) * kTileBytes;
-        const uint32_t bar = bar0 + (j % kStages) * 8;
-        mbar_arrive_expect_tx(bar, kTileBytes);
-        const int32_t *row = p.page_table + static_cast<size_t>(b) * p.MP;
-#pragma unroll
-        for (int pg = 0; pg < kPagesPerBlock; ++pg) {
-            const int lp = j * kPagesPerBlock + pg;
-            int32_t y = oob_row;
-            if (lp < n_pages) {
-                int pid = __ldg(row + lp);
-                if (pid < 0 || pid >= p.num_pages) {
-                    latch(p.status, kDevBadPage, b, pid);
-                    pid = 0;
-                }
-                y = (pid * p.Hkv + kvh) * kPageSize;
-            }
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-                tma_load_2d(st + h * kHalfBytes + pg * (kPageSize * 128), map, h * 64, y, bar, policy);
-        }
-    };
-    auto issue_qk = [&](int j) {  // thread 0 only: S = Q K_j^T, then signal bar_s
-        const uint32_t kst = k_ring + (j % kStages) * kTileBytes;
-        constexpr uint32_t idesc = umma_idesc_bf16(kRows, kBlock, false);
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-                umma_ss(tm + kColS, umma_smem_desc(q_s + h * kQHalfBytes + ks * 32, 16, 1024),
-                        umma_smem_desc(kst + h * kHalfBytes + ks * 32, 16, 1024), idesc, (h | ks) != 0);
-        umma_commit(bar_s);
-    };
-
-    if (tid == 0) {
-        for (int j = 0; j < min(nb, kStages); ++j) {
-            issue_tile_loads(j, &tm_k, k_ring, bar_k);
-            issue_tile_loads(j, &tm_v, v_ring, bar_v);
-        }
-        if (mbar_wait(bar_k, 0)) {
-            tc_fence_after_sync();
-            issue_qk(0);
-        } else {
-            abort_a = 1;
-        }
-    }
-
-    float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
-    for (int j = 0; j < nb; ++j) {
-        // ---- logits of block j: tensor memory -> registers
-        if (ok && !mbar_wait(bar_s, j & 1)) ok = false;
-        tc_fence_after_sync();
-        uint32_t s[kBlock];
-#pragma unroll
-        for (int c = 0; c < kBlock / 32; ++c)
-            tmem_ld32(tm + lane_base + kColS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(s + c * 32));
-        tmem_wait_ld();
-        if (!ok) abort_a = 1;
-        tc_fence_before_sync();
-        __syncthreads();  // every thread holds its logits: the S columns are free again
-        if (abort_a) break;
-        if (tid == 0 && j + kStages < nb) issue_tile_loads(j + kStages, &tm_k, k_ring, bar_k);  // S_j is done: its K tile is free
-        if (tid == 0 && j + 1 < nb) {  // S of the next block overlaps this block's softmax
-            if (mbar_wait(bar_k + ((j + 1) % kStages) * 8, ((j + 1) / kStages) & 1)) {
-                tc_fence_after_sync();
-                issue_qk(j + 1);
-            } else {
-                abort_b = 1;
-            }
-        }
 
-        // ---- softmax of this thread's row. Logits stay raw; sm_scale * log2(e) > 0 is folded into the
-        // exponent's FMA, so the row maximum can be taken on the raw values.
-        const int t0 = j * kBlock;
-        float mx = -INFINITY;
-        if (t0 + kBlock - 1 > my_pos) {  // the block reaches past this row's position: mask by select
+    if (warp == kRows / 32) {
+        // ================= issuing warp: one thread feeds TMA and the tensor cores =================
+        if ((tid & 31) == 0) {
+            const uint64_t policy = l2_policy_evict_first();
+            const int32_t oob_row = p.num_pages * p.Hkv * kPageSize;  // a TMA box that starts here is all zero fill
+            // K and V travel separately: a K tile is free again once its S MMA has completed, a V tile only
+            // after its O MMA, so K is requested two blocks ahead
+            auto issue_tile_loads = [&](int j, const CUtensorMap *map, uint32_t ring, uint32_t bar0) {
+                const uint32_t st = ring + (j % kStages) * kTileBytes;
+                const uint32_t bar = bar0 + (j % kStages) * 8;
+                mbar_arrive_expect_tx(bar, kTileBytes);
+                const int32_t *row = p.page_table + static_cast<size_t>(b) * p.MP;
 #pragma unroll
-            for (int c = 0; c < kBlock; ++c) {
-                if (t0 + c > my_pos) s[c] = 0xff800000u;  // -inf
-                mx = fmaxf(mx, __uint_as_float(s[c]));
+                for (int pg = 0; pg < kPagesPerBlock; ++pg) {
+                    const int lp = j * kPagesPerBlock + pg;
+                    int32_t y = oob_row;
+                    if (lp < n_pages) {
+                        int pid = __ldg(row + lp);
+                        if (pid < 0 || pid >= p.num_pages) {
+                            latch(p.status, kDevBadPage, b, pid);
+                            pid = 0;
+                        }
+                        y = (pid * p.Hkv + kvh) * kPageSize;
+                    }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_2d(st + h * kHalfBytes + pg * (kPageSize * 128), map, h * 64, y, bar, policy);
+                }
+            };
+            auto issue_qk = [&](int j) {  // S = Q K_j^T, then signal bar_s
+                const uint32_t kst = k_ring + (j % kStages) * kTileBytes;
+                constexpr uint32_t idesc = umma_idesc_bf16(kRows, kBlock, false);
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_ss(tm + kColS, umma_smem_desc(q_s + h * kQHalfBytes + ks * 32, 16, 1024),
+                                umma_smem_desc(kst + h * kHalfBytes + ks * 32, 16, 1024), idesc, (h | ks) != 0);
+                umma_commit(bar_s);
+            };
+            for (int j = 0; j < min(nb, kStages); ++j) {
+                issue_tile_loads(j, &tm_k, k_ring, bar_k);
+                issue_tile_loads(j, &tm_v, v_ring, bar_v);
             }
-        } else {
-#pragma unroll
-            for (int c = 0; c < kBlock; c += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(s[c]), __uint_as_float(s[c + 1])));
-        }
-        mx *= p.scale_log2;
-        float alpha = 1.f;
-        if (mx > m_run + kSlack) {
-            const float m_new = fmaxf(m_run, mx);
-            alpha = fast_exp2(m_run - m_new);
-            m_run = m_new;
-        }
-        // the previous block's O += P V must have finished before P or O is touched; it also frees a stage
-        if (j > 0 && ok && !mbar_wait(bar_pv, (j - 1) & 1)) ok = false;
-        tc_fence_after_sync();
-        if (tid == 0 && j > 0 && j - 1 + kStages < nb) issue_tile_loads(j - 1 + kStages, &tm_v, v_ring, bar_v);
-        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {  // rare: rescale this warp's rows of O
-            l_run *= alpha;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t o[32];
-                tmem_ld32(tm + lane_base + kColO + c * 32, o);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                tmem_st32(tm + lane_base + kColO + c * 32, o);
-            }
-        } else {
-            l_run *= alpha;  // alpha is 1 unless this is the first block (l_run is 0 then)
-        }
-        uint32_t pk[kBlock / 2];
-        float sum0 = 0.f, sum1 = 0.f;
-        const float neg_m = -m_run;
-#pragma unroll
-        for (int c = 0; c < kBlock; c += 2) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(s[c]), p.scale_log2, neg_m));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, neg_m));
-            sum0 += p0;
-            sum1 += p1;
-            pk[c >> 1] = pack_bf16x2(p0, p1);
-        }
-        l_run += sum0 + sum1;
-#pragma unroll
-        for (int c = 0; c < kBlock / 64; ++c)
-            tmem_st32(tm + lane_base + kColP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(pk + c * 32));
-        tmem_wait_st();
-
-        // V rows past the context inside the last page may hold NaN; 0 * NaN is NaN, so clear them
-        const uint32_t vst = v_ring + (j % kStages) * kTileBytes;
-        const uint32_t bar_vj = bar_v + (j % kStages) * 8;
-        const uint32_t par_vj = (j / kStages) & 1;
-        const int valid_rows = L - t0;
-        if (valid_rows < kBlock) {
-            if (ok && !mbar_wait(bar_vj, par_vj)) ok = false;  // the tile must have landed before it is patched
-            const int last = min(kBlock, (valid_rows + kPageSize - 1) / kPageSize * kPageSize);
-            for (int i = tid; i < (last - valid_rows) * 16; i += kRows) {
-                const int r = valid_rows + (i >> 4), c = i & 15;
-                st_shared_zero16(vst + (c >> 3) * kHalfBytes + r * 128 + (c & 7) * 16);
-            }
-            fence_proxy_async();
-        }
-        if (!ok) abort_b = 1;
-        tc_fence_before_sync();
-        __syncthreads();  // P complete, O corrected
-        if (abort_b) break;
-        if (tid == 0) {  // O += P V_j
-            if (!mbar_wait(bar_vj, par_vj)) abort_a = 1;  // seen by everyone after the next step's first barrier
+            ok = mbar_wait(bar_k, 0);
             tc_fence_after_sync();
-            constexpr uint32_t idesc = umma_idesc_bf16(kRows, kD, true);
+            if (ok) issue_qk(0);
+            for (int j = 0; j < nb && ok; ++j) {
+                if (j > 0) {  // O MMA of block j-1 done: its V tile is free
+                    ok = mbar_wait(bar_pv, (j - 1) & 1);
+                    if (ok && j - 1 + kStages < nb) issue_tile_loads(j - 1 + kStages, &tm_v, v_ring, bar_v);
+                }
+                // every row holds S_j in registers: the S columns and K tile j are free
+                ok = ok && mbar_wait(bar_s_read, j & 1);
+                if (!ok) break;
+                if (j + kStages < nb) issue_tile_loads(j + kStages, &tm_k, k_ring, bar_k);
+                if (j + 1 < nb) {  // S of the next block overlaps this block's softmax
+                    ok = mbar_wait(bar_k + ((j + 1) % kStages) * 8, ((j + 1) / kStages) & 1);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    issue_qk(j + 1);
+                }
+                ok = mbar_wait(bar_p_full, j & 1) && mbar_wait(bar_v + (j % kStages) * 8, (j / kStages) & 1);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t vst = v_ring + (j % kStages) * kTileBytes;
+                constexpr uint32_t idesc = umma_idesc_bf16(kRows, kD, true);
 #pragma unroll
-            for (int ks = 0; ks < kBlock / 16; ++ks)
-                umma_ts(tm + kColO, tm + kColP + ks * 8, umma_smem_desc(vst + ks * 2048, kHalfBytes, 1024), idesc,
-                        (j | ks) != 0);
-            umma_commit(bar_pv);
+                for (int ks = 0; ks < kBlock / 16; ++ks)  // O += P V_j
+                    umma_ts(tm + kColO, tm + kColP + ks * 8, umma_smem_desc(vst + ks * 2048, kHalfBytes, 1024), idesc,
+                            (j | ks) != 0);
+                umma_commit(bar_pv);
+            }
+            if (!ok) latch(p.status, kDevTimeout, b, blockIdx.x);
         }
-    }
+    } else {
+        // ================= softmax warps: one thread per query row =================
+        const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+        float m_run = -INFINITY, l_run = 0.f;
+        for (int j = 0; j < nb && ok; ++j) {
+            // ---- logits of block j: tensor memory -> registers
+            ok = mbar_wait(bar_s, j & 1);
+            tc_fence_after_sync();
+            uint32_t s[kBlock];
+#pragma unroll
+            for (int c = 0; c < kBlock / 32; ++c)
+                tmem_ld32(tm + lane_base + kColS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(s + c * 32));
+            tmem_wait_ld();
+            tc_fence_before_sync();
+            mbar_arrive(bar_s_read);
+            if (!ok) break;
 
-    // ---- epilogue: O / l -> bf16 rows
-    const bool aborted = abort_a != 0 || abort_b != 0;  // uniform: read after the barrier that ended the loop
-    if (!aborted) {
-        if (!mbar_wait(bar_pv, (nb - 1) & 1)) ok = false;
+            // ---- softmax of this thread's row. Logits stay raw; sm_scale * log2(e) > 0 is folded into the
+            // exponent's FMA, so the row maximum can be taken on the raw values.
+            const int t0 = j * kBlock;
+            float mx = -INFINITY;
+            if (t0 + kBlock - 1 > my_pos) {  // the block reaches past this row's position: mask by select
+#pragma unroll
+                for (int c = 0; c < kBlock; ++c) {
+                    if (t0 + c > my_pos) s[c] = 0xff800000u;  // -inf
+                    mx = fmaxf(mx, __uint_as_float(s[c]));
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < kBlock; c += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(s[c]), __uint_as_float(s[c + 1])));
+            }
+            mx *= p.scale_log2;
+            float alpha = 1.f;
+            if (mx > m_run + kSlack) {
+                const float m_new = fmaxf(m_run, mx);
+                alpha = fast_exp2(m_run - m_new);
+                m_run = m_new;
+            }
+            uint32_t pk[kBlock / 2];
+            float sum0 = 0.f, sum1 = 0.f;
+            const float neg_m = -m_run;
+#pragma unroll
+            for (int c = 0; c < kBlock; c += 2) {
+                const float p0 = fast_exp2(fmaf(__uint_as_float(s[c]), p.scale_log2, neg_m));
+                const float p1 = fast_exp2(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, neg_m));
+                sum0 += p0;
+                sum1 += p1;
+                pk[c >> 1] = pack_bf16x2(p0, p1);
+            }
+            l_run = l_run * alpha + (sum0 + sum1);
+            // the previous block's O += P V must have finished before P or O is touched
+            if (j > 0) {
+                ok = mbar_wait(bar_pv, (j - 1) & 1);
+                tc_fence_after_sync();
+                if (__any_sync(0xffffffffu, alpha != 1.f)) {  // rare: rescale this warp's rows of O
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tm + lane_base + kColO + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(tm + lane_base + kColO + c * 32, o);
+                    }
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < kBlock / 64; ++c)
+                tmem_st32(tm + lane_base + kColP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(pk + c * 32));
+            tmem_wait_st();
+            // V rows past the context inside the last page may hold NaN; 0 * NaN is NaN, so clear them
+            const int valid_rows = L - t0;
+            if (valid_rows < kBlock) {
+                const uint32_t vst = v_ring + (j % kStages) * kTileBytes;
+                ok = ok && mbar_wait(bar_v + (j % kStages) * 8, (j / kStages) & 1);  // the tile must have landed
+                const int last = min(kBlock, (valid_rows + kPageSize - 1) / kPageSize * kPageSize);
+                for (int i = tid; i < (last - valid_rows) * 16; i += kRows) {
+                    const int r = valid_rows + (i >> 4), c = i & 15;
+                    st_shared_zero16(vst + (c >> 3) * kHalfBytes + r * 128 + (c & 7) * 16);
+                }
+                fence_proxy_async();
+            }
+            tc_fence_before_sync();
+            mbar_arrive(bar_p_full);
+        }
+
+        // ---- epilogue: O / l -> bf16 rows
+        if (ok) ok = mbar_wait(bar_pv, (nb - 1) & 1);
         tc_fence_after_sync();
         const float inv = 1.f / l_run;
         __nv_bfloat16 *orow = p.out + (static_cast<size_t>(q0 + tile_start + tok) * p.Hq + kvh * G + head) * kD;
@@ -311,9 +312,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         }
         if (p.lse != nullptr && row_valid && ok)
             p.lse[static_cast<size_t>(q0 + tile_start + tok) * p.Hq + kvh * G + head] = (m_run + log2f(l_run)) * kLn2f;
-    }
-    if (!ok || aborted) {
-        if (tid == 0) latch(p.status, kDevTimeout, b, blockIdx.x);
+        if (!ok && (tid & 31) == 0) latch(p.status, kDevTimeout, b, blockIdx.x);
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -364,7 +363,7 @@ __global__ void advance_lens_kernel(const AppendTokensParams p) {
 
 }  // namespace
 
-size_t prefill_smem_bytes() { return kQBytes + 2 * kStages * kTileBytes + 1024 + (2 * kStages + 2) * 8 + 64; }
+size_t prefill_smem_bytes() { return kQBytes + 2 * kStages * kTileBytes + 1024 + (2 * kStages + 4) * 8 + 64; }
 
 cudaError_t prepare_prefill_attn() {
     return cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -376,7 +375,7 @@ cudaError_t launch_prefill_attn(const CUtensorMap &tm_k, const CUtensorMap &tm_v
     if (p.B == 0 || max_q_len <= 0) return cudaSuccess;
     const int tok = kRows / p.G;
     const dim3 grid((max_q_len + tok - 1) / tok, p.Hkv, p.B);
-    return launch_pdl(prefill_attn_kernel, grid, dim3(kRows), prefill_smem_bytes(), stream, p.pdl != 0, tm_k, tm_v, p);
+    return launch_pdl(prefill_attn_kernel, grid, dim3(kThreads), prefill_smem_bytes(), stream, p.pdl != 0, tm_k, tm_v, p);
 }
 
 cudaError_t launch_kv_append_tokens(const AppendTokensParams &p, int max_q_len, cudaStream_t stream) {
