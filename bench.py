@@ -591,6 +591,63 @@ def run_prefill(args):
     print(json.dumps(result), flush=True)
 
 
+# ------------------------------------------------------------------------------------------ fitting b
+
+def run_fit_b(args):
+    """Measures the decode step (append + attention) at several batch sizes with 8192-token contexts and fits
+    step_seconds = A_attn + b * concurrency: b is the per-sequence, per-layer KV-read cost of Eq. 1, as this
+    library delivers it on this GPU. The fit feeds pd_decide in an example with assumed remaining parameters."""
+    import torch
+
+    import paper_2609_35158_b200 as pd
+    import workloads as wl
+
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    w = wl.WORKLOADS[1]
+    K, W = args.steps, args.warmup
+    ctx_len = 8192
+    batches = [8, 16, 32, 64, 128, 256]
+    times = []
+    for B in batches:
+        lens = np.full(B, ctx_len, dtype=np.int32)
+        cache = wl.build_paged_cache(lens, w.num_kv_heads, w.head_dim, seed=60 + B, device=dev, reserve_tokens=W + K + 2)
+        ctx = pd.pd_create(w.num_q_heads, w.num_kv_heads, w.head_dim, 16, B, cache.page_table.shape[1], cache.num_pages, 0)
+        q = wl.random_bf16((B, w.num_q_heads, w.head_dim), 61, dev)
+        kn = wl.random_bf16((B, w.num_kv_heads, w.head_dim), 62, dev)
+        out = torch.empty_like(q)
+
+        def step():
+            pd.pd_kv_append(ctx, kn, kn, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens)
+            pd.pd_decode_attn(ctx, q, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, out, sm_scale=w.sm_scale)
+
+        for _ in range(W):
+            step()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t0.record()
+        for _ in range(K):
+            step()
+        t1.record()
+        torch.cuda.synchronize()
+        times.append(t0.elapsed_time(t1) / K * 1e-3)
+        pd.pd_destroy(ctx)
+        del cache
+    A_attn, b = pd.pd_fit_decode_cost(batches, times)
+    layers = 36  # Qwen3-8B has 36 layers (public model card); b per iteration = layers * b per layer
+    model = pd.pd_cost_model(64, 10, 200, 1000, 0.5, 0.02, b * layers, 1e-5, 0.01, 5.0, w.kv_bytes_per_token * layers, 50e9,
+                             32768.0 * w.kv_bytes_per_token * layers, 120e9, 0)
+    tgt = pd.pd_decide(model, 16)
+    print(json.dumps({
+        "metric": "decode cost per concurrent sequence per layer (b of Eq. 1)", "value": round(b * 1e6, 4), "unit": "us",
+        "fixed_us_per_layer": round(A_attn * 1e6, 3), "context_tokens": ctx_len, "batches": batches,
+        "step_us": [round(t * 1e6, 2) for t in times],
+        "ideal_us_per_sequence_at_measured_copy_bw": round(ctx_len * w.kv_bytes_per_token / measured_hbm_peak()[0] / 1e3, 4),
+        "example_decision": {"assumed": "B=64 S=10 r=200 dL=1000 theta=0.5 A=20ms t_prefill=10us T_env=5s BW=50GB/s H_max=120GB, 36 layers",
+                             "N_k": 16, "N_P": tgt.N_P, "N_D": tgt.N_D, "N_C": tgt.N_C, "makespan_s": round(tgt.makespan, 3)},
+    }), flush=True)
+
+
 # ------------------------------------------------------------------------------------------ reference arm
 
 def run_reference(args):
@@ -653,9 +710,9 @@ def main():
     ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--op", default="decode", choices=["decode", "kv_transfer", "prefill"],
+    ap.add_argument("--op", default="decode", choices=["decode", "kv_transfer", "prefill", "fit_b"],
                     help="decode = the headline decode step; kv_transfer = page gather + scatter; "
-                         "prefill = one append-prefill turn")
+                         "prefill = one append-prefill turn; fit_b = decode step time over batch size, fitted to A + b * B")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
@@ -665,6 +722,8 @@ def main():
         run_transfer(args)
     elif args.op == "prefill":
         run_prefill(args)
+    elif args.op == "fit_b":
+        run_fit_b(args)
     else:
         run_cuda(args)
 

@@ -273,6 +273,67 @@ int pd_launch_count(const pd_ctx *ctx, int64_t *launches);
 int pd_last_plan(pd_ctx *ctx, void *stream, int64_t *total_units, int32_t *pages_per_range,
                  int32_t *num_ranges, int32_t *num_workers);
 
+/*
+ * ---- PD decision engine (host-only, no CUDA): the paper's makespan models and plan arithmetic.
+ * The decode-side inputs b and K are quantities this library measures: b is the slope of the decode
+ * step time over the number of concurrent sequences (pd_fit_decode_cost on timings of pd_decode_attn),
+ * K the KV bytes per token that pd_kv_gather / pd_kv_scatter move. Times in seconds, sizes in bytes.
+ */
+typedef struct pd_cost_model {
+    double B;          /* trajectories in the rollout batch                                          */
+    double S;          /* interaction turns on the slowest trajectory                                 */
+    double r;          /* tokens generated per turn                                                   */
+    double dL;         /* prompt tokens added per turn                                                */
+    double theta;      /* bubble ratio (1 - f) / f, f = fraction of trajectories actively decoding    */
+    double A;          /* fixed cost of a decode iteration (weight reads, kernel dispatch)            */
+    double b;          /* marginal cost of one more concurrent sequence (KV-cache HBM reads)          */
+    double t_prefill;  /* prefill time per token                                                      */
+    double T_over;     /* per-turn overhead of colocation (prefill/decode switching)                  */
+    double T_env;      /* environment interaction time                                                */
+    double K_bytes;    /* KV transfer volume per token                                                */
+    double BW;         /* bandwidth between the prefill and decode pools, bytes per second            */
+    double K_seq_bytes;/* KV-cache size per trajectory                                                */
+    double H_max_bytes;/* HBM capacity per worker available to the KV cache                           */
+    double prefill_tokens_per_worker; /* tokens a prefill worker absorbs per step; 0 = do not check   */
+} pd_cost_model;
+
+typedef struct pd_target {
+    int32_t N_P, N_D, N_C; /* prefill, decode, colocated workers: fully colocated or fully disaggregated */
+    double makespan;       /* predicted batch makespan of this configuration                             */
+} pd_target;
+
+/* Eq. 1: colocated makespan on N workers. NaN on invalid input. */
+double pd_makespan_coloc(const pd_cost_model *m, int32_t N);
+/* Eq. 2-3: T_dis = max(T_prefill, T_decode) + T_env; the two paths are returned if the pointers are set. */
+double pd_makespan_disagg(const pd_cost_model *m, int32_t N_P, int32_t N_D, double *T_prefill, double *T_decode);
+/* Capacity constraints of Sec. 4.2: B K_seq <= N_D H_max, and B S dL <= N_P prefill_tokens_per_worker. */
+int32_t pd_feasible_disagg(const pd_cost_model *m, int32_t N_P, int32_t N_D);
+/*
+ * Online decision (Sec. 4.3.2): enumerates N_P in [1, N_k - 1] over the feasible splits, compares the
+ * best with colocation and returns the configuration of minimal predicted makespan. With `current` set,
+ * mode-dependent hysteresis applies: the switch is taken only if the relative gain over the current
+ * configuration exceeds ratio_threshold (same mode) or mode_threshold (colocation <-> disaggregation);
+ * a current configuration that is infeasible or sized for another N_k forces the switch. The paper
+ * publishes no threshold values; they are parameters.
+ */
+int pd_decide(const pd_cost_model *m, int32_t N_k, const pd_target *current, double ratio_threshold,
+              double mode_threshold, pd_target *out);
+/*
+ * Minimal-change plan (Eq. 5-6). Slots are stable worker ids 0 .. n_slots-1; cur_active / dst_active
+ * flag membership in the current and target active sets, cur_role[w] in [0, n_roles) is the role of a
+ * currently active worker, dst_role_count[r] the number of workers role r needs (their sum must equal
+ * the target set's size). new_role[w] receives the role of every target worker (-1 elsewhere):
+ * survivors keep their role up to its target count, the rest of the deficits go to survivors that must
+ * switch and then to joining workers. *d_worker = joins + departures, *d_role = survivors that switch.
+ */
+int pd_min_change_plan(const int32_t *cur_active, const int32_t *cur_role, const int32_t *dst_active,
+                       int32_t n_slots, const int32_t *dst_role_count, int32_t n_roles, int32_t *new_role,
+                       int32_t *d_worker, int32_t *d_role);
+/* Eq. 7: borrow training GPUs iff (R / B) (T_ded - T_full) > T_toggle. */
+int32_t pd_toggle_gate(double R, double B, double T_ded, double T_full, double T_toggle);
+/* Least-squares line step_seconds = A + b * concurrency over n >= 2 measurements. */
+int pd_fit_decode_cost(const double *concurrency, const double *step_seconds, int32_t n, double *A, double *b);
+
 const char *pd_status_string(int status);
 
 /* Text of the most recent failure recorded by this context (CUDA error string

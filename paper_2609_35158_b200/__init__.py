@@ -40,6 +40,17 @@ class pd_config(ctypes.Structure):
     ]
 
 
+class pd_cost_model(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_double) for n in (
+        "B", "S", "r", "dL", "theta", "A", "b", "t_prefill", "T_over", "T_env", "K_bytes", "BW", "K_seq_bytes",
+        "H_max_bytes", "prefill_tokens_per_worker")]
+
+
+class pd_target(ctypes.Structure):
+    _fields_ = [("N_P", ctypes.c_int32), ("N_D", ctypes.c_int32), ("N_C", ctypes.c_int32),
+                ("makespan", ctypes.c_double)]
+
+
 class PdError(RuntimeError):
     def __init__(self, code: int, where: str, detail: str = ""):
         self.code = code
@@ -72,13 +83,24 @@ def _load() -> ctypes.CDLL:
     lib.pd_launch_count.argtypes = [vp, ctypes.POINTER(i64)]
     lib.pd_last_plan.argtypes = [vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i32), ctypes.POINTER(i32),
                                  ctypes.POINTER(i32)]
+    dbl = ctypes.c_double
+    pm, pt = ctypes.POINTER(pd_cost_model), ctypes.POINTER(pd_target)
+    lib.pd_makespan_coloc.argtypes = [pm, i32]
+    lib.pd_makespan_coloc.restype = dbl
+    lib.pd_makespan_disagg.argtypes = [pm, i32, i32, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
+    lib.pd_makespan_disagg.restype = dbl
+    lib.pd_feasible_disagg.argtypes = [pm, i32, i32]
+    lib.pd_decide.argtypes = [pm, i32, pt, dbl, dbl, pt]
+    lib.pd_min_change_plan.argtypes = [vp, vp, vp, i32, vp, i32, vp, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    lib.pd_toggle_gate.argtypes = [dbl, dbl, dbl, dbl, dbl]
+    lib.pd_fit_decode_cost.argtypes = [vp, vp, i32, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
     lib.pd_status_string.argtypes = [ctypes.c_int]
     lib.pd_status_string.restype = ctypes.c_char_p
     lib.pd_last_error.argtypes = [vp]
     lib.pd_last_error.restype = ctypes.c_char_p
     lib.pd_version.argtypes = []
     for name in EXPORTS:
-        if name not in ("pd_status_string", "pd_last_error"):
+        if name not in ("pd_status_string", "pd_last_error", "pd_makespan_coloc", "pd_makespan_disagg"):
             getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -240,3 +262,57 @@ def pd_last_plan(ctx, stream=None) -> dict:
                              ctypes.byref(workers)), "pd_last_plan", ctx)
     return {"total_units": total.value, "pages_per_range": per.value, "num_ranges": ranges.value,
             "num_workers": workers.value}
+
+
+# ---- PD decision engine (host-only)
+
+def pd_makespan_coloc(model: pd_cost_model, N: int) -> float:
+    return _lib.pd_makespan_coloc(ctypes.byref(model), N)
+
+
+def pd_makespan_disagg(model: pd_cost_model, N_P: int, N_D: int):
+    """Returns (T_dis, T_prefill, T_decode)."""
+    tp, td = ctypes.c_double(), ctypes.c_double()
+    t = _lib.pd_makespan_disagg(ctypes.byref(model), N_P, N_D, ctypes.byref(tp), ctypes.byref(td))
+    return t, tp.value, td.value
+
+
+def pd_feasible_disagg(model: pd_cost_model, N_P: int, N_D: int) -> bool:
+    return bool(_lib.pd_feasible_disagg(ctypes.byref(model), N_P, N_D))
+
+
+def pd_decide(model: pd_cost_model, N_k: int, current: pd_target | None = None, ratio_threshold=0.0,
+              mode_threshold=0.0) -> pd_target:
+    out = pd_target()
+    _check(_lib.pd_decide(ctypes.byref(model), N_k, None if current is None else ctypes.byref(current),
+                          ratio_threshold, mode_threshold, ctypes.byref(out)), "pd_decide")
+    return out
+
+
+def pd_min_change_plan(cur_active, cur_role, dst_active, dst_role_count):
+    """NumPy int32 arrays in, (new_role, d_worker, d_role) out."""
+    import numpy as np
+
+    ca, cr, da = (np.ascontiguousarray(a, dtype=np.int32) for a in (cur_active, cur_role, dst_active))
+    rc = np.ascontiguousarray(dst_role_count, dtype=np.int32)
+    new_role = np.full(len(ca), -1, dtype=np.int32)
+    dw, dr = ctypes.c_int32(), ctypes.c_int32()
+    _check(_lib.pd_min_change_plan(ca.ctypes.data, cr.ctypes.data, da.ctypes.data, len(ca), rc.ctypes.data, len(rc),
+                                   new_role.ctypes.data, ctypes.byref(dw), ctypes.byref(dr)), "pd_min_change_plan")
+    return new_role, dw.value, dr.value
+
+
+def pd_toggle_gate(R, B, T_ded, T_full, T_toggle) -> bool:
+    return bool(_lib.pd_toggle_gate(R, B, T_ded, T_full, T_toggle))
+
+
+def pd_fit_decode_cost(concurrency, step_seconds):
+    """Least-squares (A, b) of step_seconds = A + b * concurrency."""
+    import numpy as np
+
+    x = np.ascontiguousarray(concurrency, dtype=np.float64)
+    y = np.ascontiguousarray(step_seconds, dtype=np.float64)
+    A, b = ctypes.c_double(), ctypes.c_double()
+    _check(_lib.pd_fit_decode_cost(x.ctypes.data, y.ctypes.data, len(x), ctypes.byref(A), ctypes.byref(b)),
+           "pd_fit_decode_cost")
+    return A.value, b.value
