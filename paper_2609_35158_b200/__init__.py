@@ -28,6 +28,8 @@ PD_APPEND_NO_ADVANCE = 1
 EXPORTS = (
     "pd_create", "pd_destroy", "pd_kv_append", "pd_decode_attn", "pd_decode_attn_static", "pd_decode_step_host",
     "pd_kv_gather", "pd_kv_scatter", "pd_kv_append_tokens", "pd_prefill_attn", "pd_device_status", "pd_read_worker_trace",
+    "pd_makespan_coloc", "pd_makespan_disagg", "pd_feasible_disagg", "pd_decide", "pd_min_change_plan", "pd_toggle_gate",
+    "pd_fit_decode_cost",
     "pd_set_profile_events", "pd_workspace_bytes", "pd_launch_count", "pd_last_plan", "pd_status_string", "pd_last_error", "pd_version",
 )
 
