@@ -229,9 +229,16 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                     if (t0 + c > my_pos) s[c] = 0xff800000u;  // -inf
                     mx = fmaxf(mx, __uint_as_float(s[c]));
                 }
-            } else {
+            } else {  // four independent chains instead of one 64-long dependency
+                float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < kBlock; c += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(s[c]), __uint_as_float(s[c + 1])));
+                for (int c = 0; c < kBlock; c += 4) {
+                    m0 = fmaxf(m0, __uint_as_float(s[c]));
+                    m1 = fmaxf(m1, __uint_as_float(s[c + 1]));
+                    m2 = fmaxf(m2, __uint_as_float(s[c + 2]));
+                    m3 = fmaxf(m3, __uint_as_float(s[c + 3]));
+                }
+                mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
             }
             mx *= p.scale_log2;
             float alpha = 1.f;
@@ -241,16 +248,21 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 m_run = m_new;
             }
             uint32_t pk[kBlock / 2];
-            float sum0 = 0.f, sum1 = 0.f;
-            const float neg_m = -m_run;
+            // packed fp32x2 arithmetic: one FMA and one add per pair of logits
+            const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-m_run, -m_run);
+            float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 #pragma unroll
-            for (int c = 0; c < kBlock; c += 2) {
-                const float p0 = fast_exp2(fmaf(__uint_as_float(s[c]), p.scale_log2, neg_m));
-                const float p1 = fast_exp2(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, neg_m));
-                sum0 += p0;
-                sum1 += p1;
-                pk[c >> 1] = pack_bf16x2(p0, p1);
+            for (int c = 0; c < kBlock; c += 4) {
+                const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, nm2);
+                const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), sc2, nm2);
+                const float2 e0 = make_float2(fast_exp2(x0.x), fast_exp2(x0.y));
+                const float2 e1 = make_float2(fast_exp2(x1.x), fast_exp2(x1.y));
+                acc0 = __fadd2_rn(acc0, e0);
+                acc1 = __fadd2_rn(acc1, e1);
+                pk[c >> 1] = pack_bf16x2(e0.x, e0.y);
+                pk[(c >> 1) + 1] = pack_bf16x2(e1.x, e1.y);
             }
+            const float sum0 = acc0.x + acc0.y, sum1 = acc1.x + acc1.y;
             l_run = l_run * alpha + (sum0 + sum1);
             // the previous block's O += P V must have finished before P or O is touched
             if (j > 0) {
