@@ -254,7 +254,10 @@ int pd_set_profile_events(pd_ctx *ctx, void *before, void *after);
  * PD_ERR_UNSUPPORTED). Waits for `stream`, then copies up to max_workers
  * records of four uint64 nanosecond values (%globaltimer: kernel entry, first
  * tile landed, last tile landed, exit) to host_out (HOST pointer) and stores
- * the number of records in *num_workers.
+ * the number of records in *num_workers. After a pd_prefill_attn the same
+ * buffer holds, per CTA (in launch order) and as four consecutive records, the
+ * SM-clock cycles row thread 0 spent waiting for S, loading S, in the softmax
+ * arithmetic, waiting for O, storing P, in total, and its block count.
  */
 int pd_read_worker_trace(pd_ctx *ctx, void *stream, uint64_t *host_out, int32_t max_workers, int32_t *num_workers);
 

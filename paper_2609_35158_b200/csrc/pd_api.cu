@@ -458,6 +458,9 @@ int pd_prefill_attn(pd_ctx *ctx, const void *q, const int32_t *q_indptr, const v
     p.num_pages = static_cast<int32_t>(ctx->cfg.num_pages);
     p.scale_log2 = sm_scale * 1.4426950408889634f;
     p.pdl = ctx->pdl;
+    p.trace = ctx->trace;                    // the worker-trace buffer doubles as [CTA][16] phase counters
+    p.trace_ctas = ctx->trace_workers / 4;
+    if (ctx->trace != nullptr) cudaMemsetAsync(ctx->trace, 0, static_cast<size_t>(ctx->trace_workers) * 32, static_cast<cudaStream_t>(stream));
     const cudaError_t err = pd::launch_prefill_attn(ctx->tm_k, ctx->tm_v, p, max_q_len, static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "prefill_attn launch", err);
     ctx->launches += 1;

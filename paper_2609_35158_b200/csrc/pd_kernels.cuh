@@ -86,6 +86,8 @@ struct PrefillParams {
     int32_t num_pages;
     float scale_log2;
     int32_t pdl;
+    unsigned long long *trace;  // optional [trace_ctas][8] SM-clock cycles per phase of row thread 0
+    int32_t trace_ctas;
 };
 
 struct AppendTokensParams {

@@ -19,8 +19,8 @@
 //            running max with a slack of 8 log2 units, exp2, row sum, P as bf16
 //            back into tensor memory; a rare correction pass rescales O
 //   tcgen05  O += P V (P from tensor memory, 4 MMAs of 128x128x16)
-// A separate warp issues every TMA load and MMA, so the row threads never run
-// issue code or meet at a CTA barrier: they hand over through mbarriers (logits
+// One extra warp issues every MMA and another every TMA load (one box per
+// lane), so the row threads never run issue code or meet at a CTA barrier: they hand over through mbarriers (logits
 // read, probabilities written). The S MMA of block j+1 is issued as soon as
 // every row holds block j's logits in registers, and two CTAs share each SM (96 KB of shared memory, 256
 // tensor-memory columns each), so one CTA's softmax overlaps the other's MMAs. All waits are
@@ -37,7 +37,7 @@ namespace {
 constexpr float kLn2f = 0.6931471805599453f;
 constexpr float kSlack = 8.f;                 // log2 units a logit may exceed the running max before a rescale
 constexpr int kRows = 128;                    // query rows per CTA (MMA M), one softmax thread each
-constexpr int kThreads = kRows + 32;          // plus the warp whose first lane issues TMA and MMA
+constexpr int kThreads = kRows + 64;          // plus one warp that issues the MMAs and one that issues the TMA loads
 constexpr int kBlock = 64;                    // context tokens per step (MMA N of S, K of O)
 constexpr int kPagesPerBlock = kBlock / kPageSize;
 constexpr int kD = 128;
@@ -92,12 +92,15 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     const uint32_t bar_pv = smem_u32(bars + 2 * kStages + 1);     // O += P_j V_j has completed (MMA commit)
     const uint32_t bar_s_read = smem_u32(bars + 2 * kStages + 2); // all 128 rows hold S_j in registers
     const uint32_t bar_p_full = smem_u32(bars + 2 * kStages + 3); // all 128 rows wrote P_j
+    const uint32_t bar_k_free = smem_u32(bars + 2 * kStages + 4); // [kStages] the S MMA that read this K tile is done
+    const uint32_t bar_v_free = bar_k_free + kStages * 8;         // [kStages] the O MMA that read this V tile is done
 
     // ---- set-up: barriers, tensor memory, the Q tile
     if (tid == 0) {
         for (int i = 0; i < 2 * kStages + 2; ++i) mbar_init(smem_u32(bars + i), 1);
         mbar_init(bar_s_read, kRows);
         mbar_init(bar_p_full, kRows);
+        for (int i = 0; i < 2 * kStages; ++i) mbar_init(bar_k_free + i * 8, 1);
         mbar_init_fence();
         prefetch_tensormap(&tm_k);
         prefetch_tensormap(&tm_v);
@@ -128,34 +131,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     bool ok = true;
 
     if (warp == kRows / 32) {
-        // ================= issuing warp: one thread feeds TMA and the tensor cores =================
+        // ================= MMA warp: lane 0 feeds the tensor cores =================
         if ((tid & 31) == 0) {
-            const uint64_t policy = l2_policy_evict_first();
-            const int32_t oob_row = p.num_pages * p.Hkv * kPageSize;  // a TMA box that starts here is all zero fill
-            // K and V travel separately: a K tile is free again once its S MMA has completed, a V tile only
-            // after its O MMA, so K is requested two blocks ahead
-            auto issue_tile_loads = [&](int j, const CUtensorMap *map, uint32_t ring, uint32_t bar0) {
-                const uint32_t st = ring + (j % kStages) * kTileBytes;
-                const uint32_t bar = bar0 + (j % kStages) * 8;
-                mbar_arrive_expect_tx(bar, kTileBytes);
-                const int32_t *row = p.page_table + static_cast<size_t>(b) * p.MP;
-#pragma unroll
-                for (int pg = 0; pg < kPagesPerBlock; ++pg) {
-                    const int lp = j * kPagesPerBlock + pg;
-                    int32_t y = oob_row;
-                    if (lp < n_pages) {
-                        int pid = __ldg(row + lp);
-                        if (pid < 0 || pid >= p.num_pages) {
-                            latch(p.status, kDevBadPage, b, pid);
-                            pid = 0;
-                        }
-                        y = (pid * p.Hkv + kvh) * kPageSize;
-                    }
-#pragma unroll
-                    for (int h = 0; h < 2; ++h)
-                        tma_load_2d(st + h * kHalfBytes + pg * (kPageSize * 128), map, h * 64, y, bar, policy);
-                }
-            };
             auto issue_qk = [&](int j) {  // S = Q K_j^T, then signal bar_s
                 const uint32_t kst = k_ring + (j % kStages) * kTileBytes;
                 constexpr uint32_t idesc = umma_idesc_bf16(kRows, kBlock, false);
@@ -166,49 +143,110 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                         umma_ss(tm + kColS, umma_smem_desc(q_s + h * kQHalfBytes + ks * 32, 16, 1024),
                                 umma_smem_desc(kst + h * kHalfBytes + ks * 32, 16, 1024), idesc, (h | ks) != 0);
                 umma_commit(bar_s);
+                umma_commit(bar_k_free + (j % kStages) * 8);
             };
-            for (int j = 0; j < min(nb, kStages); ++j) {
-                issue_tile_loads(j, &tm_k, k_ring, bar_k);
-                issue_tile_loads(j, &tm_v, v_ring, bar_v);
-            }
             ok = mbar_wait(bar_k, 0);
             tc_fence_after_sync();
             if (ok) issue_qk(0);
             for (int j = 0; j < nb && ok; ++j) {
-                if (j > 0) {  // O MMA of block j-1 done: its V tile is free
-                    ok = mbar_wait(bar_pv, (j - 1) & 1);
-                    if (ok && j - 1 + kStages < nb) issue_tile_loads(j - 1 + kStages, &tm_v, v_ring, bar_v);
-                }
-                // every row holds S_j in registers: the S columns and K tile j are free
-                ok = ok && mbar_wait(bar_s_read, j & 1);
+                // once every row holds S_j in registers the S columns are free: start S of the next block
+                ok = mbar_wait(bar_s_read, j & 1);
                 if (!ok) break;
-                if (j + kStages < nb) issue_tile_loads(j + kStages, &tm_k, k_ring, bar_k);
-                if (j + 1 < nb) {  // S of the next block overlaps this block's softmax
+                if (j + 1 < nb) {
                     ok = mbar_wait(bar_k + ((j + 1) % kStages) * 8, ((j + 1) / kStages) & 1);
                     if (!ok) break;
                     tc_fence_after_sync();
                     issue_qk(j + 1);
                 }
+                // O += P V_j as soon as the rows have written P_j
                 ok = mbar_wait(bar_p_full, j & 1) && mbar_wait(bar_v + (j % kStages) * 8, (j / kStages) & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t vst = v_ring + (j % kStages) * kTileBytes;
                 constexpr uint32_t idesc = umma_idesc_bf16(kRows, kD, true);
 #pragma unroll
-                for (int ks = 0; ks < kBlock / 16; ++ks)  // O += P V_j
+                for (int ks = 0; ks < kBlock / 16; ++ks)
                     umma_ts(tm + kColO, tm + kColP + ks * 8, umma_smem_desc(vst + ks * 2048, kHalfBytes, 1024), idesc,
                             (j | ks) != 0);
                 umma_commit(bar_pv);
+                umma_commit(bar_v_free + (j % kStages) * 8);
             }
             if (!ok) latch(p.status, kDevTimeout, b, blockIdx.x);
         }
+    } else if (warp == kRows / 32 + 1) {
+        // ================= TMA warp: one box per lane =================
+        // A tile of 64 tokens is 4 pages x 2 halves = 8 boxes of 2 KB. Issued one after another by a single
+        // thread they cost ~170 cycles each; here lane l issues box l of the tile in one warp instruction.
+        // Page ids are fetched 32 at a time (one per lane), a group ahead of need.
+        const int lane = tid & 31;
+        const uint64_t policy = l2_policy_evict_first();
+        const int32_t oob_row = p.num_pages * p.Hkv * kPageSize;  // a TMA box that starts here is all zero fill
+        const int32_t *pt_row = p.page_table + static_cast<size_t>(b) * p.MP;
+        struct IdCache { int grp, val, nval; };
+        auto load_group = [&](int grp) {
+            const int idx = grp * 32 + lane;
+            return (idx < n_pages) ? __ldg(pt_row + idx) : -1;
+        };
+        auto issue_tile_loads = [&](int j, const CUtensorMap *map, uint32_t ring, uint32_t bar0, IdCache &c) {
+            const uint32_t st = ring + (j % kStages) * kTileBytes;
+            const uint32_t bar = bar0 + (j % kStages) * 8;
+            const int grp = (j * kPagesPerBlock) >> 5;  // the 4 pages of a block never straddle a group of 32
+            if (grp != c.grp) {
+                c.val = (grp == c.grp + 1) ? c.nval : load_group(grp);
+                c.grp = grp;
+                c.nval = load_group(grp + 1);
+            }
+            const int pg = (lane >> 1) & (kPagesPerBlock - 1), h = lane & 1;
+            const int lp = j * kPagesPerBlock + pg;
+            int pid = __shfl_sync(0xffffffffu, c.val, lp & 31);
+            int32_t y = oob_row;
+            if (lp < n_pages) {
+                if (pid < 0 || pid >= p.num_pages) {
+                    if (lane < 2 * kPagesPerBlock && h == 0) latch(p.status, kDevBadPage, b, pid);
+                    pid = 0;
+                }
+                y = (pid * p.Hkv + kvh) * kPageSize;
+            }
+            if (lane == 0) mbar_arrive_expect_tx(bar, kTileBytes);
+            __syncwarp();
+            if (lane < 2 * kPagesPerBlock)
+                tma_load_2d(st + h * kHalfBytes + pg * (kPageSize * 128), map, h * 64, y, bar, policy);
+        };
+        IdCache ck{-2, -1, -1}, cv{-2, -1, -1};
+        for (int j = 0; j < min(nb, kStages); ++j) {
+            issue_tile_loads(j, &tm_k, k_ring, bar_k, ck);
+            issue_tile_loads(j, &tm_v, v_ring, bar_v, cv);
+        }
+        // A tile is reloaded once the MMA that read it has completed; each ring slot has its own barrier,
+        // whose next phase cannot complete before this warp has reloaded the slot
+        for (int j = 0; j + kStages < nb && ok; ++j) {
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_k_free + (j % kStages) * 8, (j / kStages) & 1));
+            if (!ok) break;
+            issue_tile_loads(j + kStages, &tm_k, k_ring, bar_k, ck);
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_v_free + (j % kStages) * 8, (j / kStages) & 1));
+            if (!ok) break;
+            issue_tile_loads(j + kStages, &tm_v, v_ring, bar_v, cv);
+        }
+        if (!ok && lane == 0) latch(p.status, kDevTimeout, b, blockIdx.x);
     } else {
         // ================= softmax warps: one thread per query row =================
         const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
         float m_run = -INFINITY, l_run = 0.f;
+        const bool tracing = p.trace != nullptr;
+        long long ph[6] = {0, 0, 0, 0, 0, 0};  // cycles: wait S, load S, math, wait O, store P, total
+        const long long t_begin = tracing ? clock64() : 0;
         for (int j = 0; j < nb && ok; ++j) {
+            long long tc = tracing ? clock64() : 0;
+            auto lap = [&](int i) {
+                if (tracing) {
+                    const long long now = clock64();
+                    ph[i] += now - tc;
+                    tc = now;
+                }
+            };
             // ---- logits of block j: tensor memory -> registers
             ok = mbar_wait(bar_s, j & 1);
+            lap(0);
             tc_fence_after_sync();
             uint32_t s[kBlock];
 #pragma unroll
@@ -217,6 +255,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             tmem_wait_ld();
             tc_fence_before_sync();
             mbar_arrive(bar_s_read);
+            lap(1);
             if (!ok) break;
 
             // ---- softmax of this thread's row. Logits stay raw; sm_scale * log2(e) > 0 is folded into the
@@ -264,10 +303,12 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             }
             const float sum0 = acc0.x + acc0.y, sum1 = acc1.x + acc1.y;
             l_run = l_run * alpha + (sum0 + sum1);
+            lap(2);
             // the previous block's O += P V must have finished before P or O is touched
             if (j > 0) {
                 ok = mbar_wait(bar_pv, (j - 1) & 1);
                 tc_fence_after_sync();
+                lap(3);
                 if (__any_sync(0xffffffffu, alpha != 1.f)) {  // rare: rescale this warp's rows of O
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
@@ -298,6 +339,16 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             }
             tc_fence_before_sync();
             mbar_arrive(bar_p_full);
+            lap(4);
+        }
+        if (tracing && tid == 0) {
+            const int cta = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+            if (cta < p.trace_ctas) {
+                unsigned long long *t = p.trace + static_cast<size_t>(cta) * 16;
+                for (int i = 0; i < 5; ++i) t[i] = static_cast<unsigned long long>(ph[i]);
+                t[5] = static_cast<unsigned long long>(clock64() - t_begin);
+                t[6] = static_cast<unsigned long long>(nb);
+            }
         }
 
         // ---- epilogue: O / l -> bf16 rows
@@ -375,7 +426,7 @@ __global__ void advance_lens_kernel(const AppendTokensParams p) {
 
 }  // namespace
 
-size_t prefill_smem_bytes() { return kQBytes + 2 * kStages * kTileBytes + 1024 + (2 * kStages + 4) * 8 + 64; }
+size_t prefill_smem_bytes() { return kQBytes + 2 * kStages * kTileBytes + 1024 + (4 * kStages + 4) * 8 + 64; }
 
 cudaError_t prepare_prefill_attn() {
     return cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
