@@ -19,8 +19,8 @@
 //            running max with a slack of 8 log2 units, exp2, row sum, P as bf16
 //            back into tensor memory; a rare correction pass rescales O
 //   tcgen05  O += P V (P from tensor memory, 4 MMAs of 128x128x16)
-// One extra warp issues every MMA and another every TMA load (one box per
-// lane), so the row threads never run issue code or meet at a CTA barrier: they hand over through mbarriers (logits
+// Four service warps issue the S MMAs, the O MMAs, the TMA loads of K and those
+// of V (one box per lane), so the row threads never run issue code or meet at a CTA barrier: they hand over through mbarriers (logits
 // read, probabilities written). The S MMA of block j+1 is issued as soon as
 // every row holds block j's logits in registers, and two CTAs share each SM (96 KB of shared memory, 256
 // tensor-memory columns each), so one CTA's softmax overlaps the other's MMAs. All waits are
@@ -37,7 +37,7 @@ namespace {
 constexpr float kLn2f = 0.6931471805599453f;
 constexpr float kSlack = 8.f;                 // log2 units a logit may exceed the running max before a rescale
 constexpr int kRows = 128;                    // query rows per CTA (MMA M), one softmax thread each
-constexpr int kThreads = kRows + 64;          // plus one warp that issues the MMAs and one that issues the TMA loads
+constexpr int kThreads = kRows + 128;         // plus four service warps: S MMAs, O MMAs, K loads, V loads
 constexpr int kBlock = 64;                    // context tokens per step (MMA N of S, K of O)
 constexpr int kPagesPerBlock = kBlock / kPageSize;
 constexpr int kD = 128;
@@ -46,10 +46,13 @@ constexpr int kQBytes = 2 * kQHalfBytes;
 constexpr int kHalfBytes = kBlock * 128;      // one 64-column half of a K or V tile of kBlock tokens
 constexpr int kTileBytes = 2 * kHalfBytes;
 constexpr int kStages = 2;                    // K ring and V ring have two tiles each
+static_assert(kStages == 2, "ring slots and logit buffers share the index j % 2 and its barriers");
 // Two CTAs share an SM (96 KB of shared memory and 256 tensor-memory columns each): while one runs its
 // softmax on the CUDA cores the other's MMAs keep the tensor cores busy.
 constexpr int kTmemCols = 256;
-constexpr int kColS = 0, kColP = kBlock, kColO = 128;  // tensor-memory columns: logits, probabilities, output
+// Tensor-memory columns: two logit buffers of kBlock columns (block j uses buffer j % 2; its probabilities
+// overwrite the first kBlock / 2 columns of the same buffer once the logits are in registers), then the output.
+constexpr int kColS = 0, kColO = 128;
 
 __device__ __forceinline__ void latch(int32_t *status, int code, int seq, int detail) {
     if (atomicCAS(status, kDevOk, code) == kDevOk) {
@@ -88,19 +91,16 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     const uint32_t k_ring = base + kQBytes, v_ring = k_ring + kStages * kTileBytes;
     uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + kQBytes + 2 * kStages * kTileBytes);
     const uint32_t bar_k = smem_u32(bars), bar_v = smem_u32(bars + kStages);
-    const uint32_t bar_s = smem_u32(bars + 2 * kStages);          // S_j is in tensor memory (MMA commit)
-    const uint32_t bar_pv = smem_u32(bars + 2 * kStages + 1);     // O += P_j V_j has completed (MMA commit)
-    const uint32_t bar_s_read = smem_u32(bars + 2 * kStages + 2); // all 128 rows hold S_j in registers
-    const uint32_t bar_p_full = smem_u32(bars + 2 * kStages + 3); // all 128 rows wrote P_j
-    const uint32_t bar_k_free = smem_u32(bars + 2 * kStages + 4); // [kStages] the S MMA that read this K tile is done
-    const uint32_t bar_v_free = bar_k_free + kStages * 8;         // [kStages] the O MMA that read this V tile is done
+    // [2] each: S_j is in logit buffer j % 2 and K tile j % 2 is free again (commit after the S MMA);
+    // O += P_j V_j has completed and V tile j % 2 and logit buffer j % 2 are free again (commit after the O MMA)
+    const uint32_t bar_s = smem_u32(bars + 2 * kStages);
+    const uint32_t bar_pv = smem_u32(bars + 2 * kStages + 2);
+    const uint32_t bar_p_full = smem_u32(bars + 2 * kStages + 4);  // all 128 rows wrote P_j
 
     // ---- set-up: barriers, tensor memory, the Q tile
     if (tid == 0) {
-        for (int i = 0; i < 2 * kStages + 2; ++i) mbar_init(smem_u32(bars + i), 1);
-        mbar_init(bar_s_read, kRows);
+        for (int i = 0; i < 2 * kStages + 4; ++i) mbar_init(smem_u32(bars + i), 1);
         mbar_init(bar_p_full, kRows);
-        for (int i = 0; i < 2 * kStages; ++i) mbar_init(bar_k_free + i * 8, 1);
         mbar_init_fence();
         prefetch_tensormap(&tm_k);
         prefetch_tensormap(&tm_v);
@@ -131,50 +131,48 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     bool ok = true;
 
     if (warp == kRows / 32) {
-        // ================= MMA warp: lane 0 feeds the tensor cores =================
+        // ================= S-MMA warp: lane 0 issues S_j = Q K_j^T into logit buffer j % 2 =================
+        // Issuing a tcgen05.mma costs the issuing thread ~70 cycles; with the S and the O products issued by
+        // one thread that thread was the bottleneck of the whole CTA, so each product has its own warp. The
+        // only ordering the hardware would not give across two issuing threads is "O MMA of block j-2 before
+        // the S MMA of block j" (same logit buffer), hence the wait on bar_pv.
         if ((tid & 31) == 0) {
-            auto issue_qk = [&](int j) {  // S = Q K_j^T, then signal bar_s
+            constexpr uint32_t idesc = umma_idesc_bf16(kRows, kBlock, false);
+            for (int j = 0; j < nb && ok; ++j) {
+                if (j >= 2) ok = mbar_wait(bar_pv + (j & 1) * 8, ((j - 2) >> 1) & 1);
+                ok = ok && mbar_wait(bar_k + (j % kStages) * 8, (j / kStages) & 1);
+                if (!ok) break;
+                tc_fence_after_sync();
                 const uint32_t kst = k_ring + (j % kStages) * kTileBytes;
-                constexpr uint32_t idesc = umma_idesc_bf16(kRows, kBlock, false);
 #pragma unroll
                 for (int h = 0; h < 2; ++h)
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
-                        umma_ss(tm + kColS, umma_smem_desc(q_s + h * kQHalfBytes + ks * 32, 16, 1024),
+                        umma_ss(tm + kColS + (j & 1) * kBlock, umma_smem_desc(q_s + h * kQHalfBytes + ks * 32, 16, 1024),
                                 umma_smem_desc(kst + h * kHalfBytes + ks * 32, 16, 1024), idesc, (h | ks) != 0);
-                umma_commit(bar_s);
-                umma_commit(bar_k_free + (j % kStages) * 8);
-            };
-            ok = mbar_wait(bar_k, 0);
-            tc_fence_after_sync();
-            if (ok) issue_qk(0);
-            for (int j = 0; j < nb && ok; ++j) {
-                // once every row holds S_j in registers the S columns are free: start S of the next block
-                ok = mbar_wait(bar_s_read, j & 1);
-                if (!ok) break;
-                if (j + 1 < nb) {
-                    ok = mbar_wait(bar_k + ((j + 1) % kStages) * 8, ((j + 1) / kStages) & 1);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    issue_qk(j + 1);
-                }
-                // O += P V_j as soon as the rows have written P_j
-                ok = mbar_wait(bar_p_full, j & 1) && mbar_wait(bar_v + (j % kStages) * 8, (j / kStages) & 1);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint32_t vst = v_ring + (j % kStages) * kTileBytes;
-                constexpr uint32_t idesc = umma_idesc_bf16(kRows, kD, true);
-#pragma unroll
-                for (int ks = 0; ks < kBlock / 16; ++ks)
-                    umma_ts(tm + kColO, tm + kColP + ks * 8, umma_smem_desc(vst + ks * 2048, kHalfBytes, 1024), idesc,
-                            (j | ks) != 0);
-                umma_commit(bar_pv);
-                umma_commit(bar_v_free + (j % kStages) * 8);
+                umma_commit(bar_s + (j & 1) * 8);
             }
             if (!ok) latch(p.status, kDevTimeout, b, blockIdx.x);
         }
     } else if (warp == kRows / 32 + 1) {
-        // ================= TMA warp: one box per lane =================
+        // ================= O-MMA warp: lane 0 issues O += P_j V_j =================
+        if ((tid & 31) == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(kRows, kD, true);
+            for (int j = 0; j < nb && ok; ++j) {
+                ok = mbar_wait(bar_p_full, j & 1) && mbar_wait(bar_v + (j % kStages) * 8, (j / kStages) & 1);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t vst = v_ring + (j % kStages) * kTileBytes;
+#pragma unroll
+                for (int ks = 0; ks < kBlock / 16; ++ks)  // P from the first columns of logit buffer j % 2
+                    umma_ts(tm + kColO, tm + kColS + (j & 1) * kBlock + ks * 8,
+                            umma_smem_desc(vst + ks * 2048, kHalfBytes, 1024), idesc, (j | ks) != 0);
+                umma_commit(bar_pv + (j & 1) * 8);
+            }
+            if (!ok) latch(p.status, kDevTimeout, b, blockIdx.x);
+        }
+    } else if (warp >= kRows / 32 + 2) {
+        // ================= two TMA warps (one streams K, the other V): one box per lane =================
         // A tile of 64 tokens is 4 pages x 2 halves = 8 boxes of 2 KB. Issued one after another by a single
         // thread they cost ~170 cycles each; here lane l issues box l of the tile in one warp instruction.
         // Page ids are fetched 32 at a time (one per lane), a group ahead of need.
@@ -212,20 +210,18 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             if (lane < 2 * kPagesPerBlock)
                 tma_load_2d(st + h * kHalfBytes + pg * (kPageSize * 128), map, h * 64, y, bar, policy);
         };
-        IdCache ck{-2, -1, -1}, cv{-2, -1, -1};
-        for (int j = 0; j < min(nb, kStages); ++j) {
-            issue_tile_loads(j, &tm_k, k_ring, bar_k, ck);
-            issue_tile_loads(j, &tm_v, v_ring, bar_v, cv);
-        }
-        // A tile is reloaded once the MMA that read it has completed; each ring slot has its own barrier,
-        // whose next phase cannot complete before this warp has reloaded the slot
+        // K and V have separate warps so that neither stream waits for the other's ring slot: a K tile is
+        // reloaded as soon as the S MMA that read it has completed, a V tile as soon as its O MMA has. The
+        // next phase of a slot's barrier cannot complete before the slot has been reloaded.
+        const bool is_k = warp == kRows / 32 + 2;
+        const CUtensorMap *map = is_k ? &tm_k : &tm_v;
+        const uint32_t ring = is_k ? k_ring : v_ring, bar_full = is_k ? bar_k : bar_v, bar_free = is_k ? bar_s : bar_pv;
+        IdCache cache{-2, -1, -1};
+        for (int j = 0; j < min(nb, kStages); ++j) issue_tile_loads(j, map, ring, bar_full, cache);
         for (int j = 0; j + kStages < nb && ok; ++j) {
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_k_free + (j % kStages) * 8, (j / kStages) & 1));
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_free + (j % kStages) * 8, (j / kStages) & 1));
             if (!ok) break;
-            issue_tile_loads(j + kStages, &tm_k, k_ring, bar_k, ck);
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_v_free + (j % kStages) * 8, (j / kStages) & 1));
-            if (!ok) break;
-            issue_tile_loads(j + kStages, &tm_v, v_ring, bar_v, cv);
+            issue_tile_loads(j + kStages, map, ring, bar_full, cache);
         }
         if (!ok && lane == 0) latch(p.status, kDevTimeout, b, blockIdx.x);
     } else {
@@ -245,16 +241,14 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 }
             };
             // ---- logits of block j: tensor memory -> registers
-            ok = mbar_wait(bar_s, j & 1);
+            const uint32_t buf = tm + lane_base + kColS + (j & 1) * kBlock;
+            ok = mbar_wait(bar_s + (j & 1) * 8, (j >> 1) & 1);
             lap(0);
             tc_fence_after_sync();
             uint32_t s[kBlock];
 #pragma unroll
-            for (int c = 0; c < kBlock / 32; ++c)
-                tmem_ld32(tm + lane_base + kColS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(s + c * 32));
+            for (int c = 0; c < kBlock / 32; ++c) tmem_ld32(buf + c * 32, *reinterpret_cast<uint32_t(*)[32]>(s + c * 32));
             tmem_wait_ld();
-            tc_fence_before_sync();
-            mbar_arrive(bar_s_read);
             lap(1);
             if (!ok) break;
 
@@ -304,12 +298,13 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             const float sum0 = acc0.x + acc0.y, sum1 = acc1.x + acc1.y;
             l_run = l_run * alpha + (sum0 + sum1);
             lap(2);
-            // the previous block's O += P V must have finished before P or O is touched
-            if (j > 0) {
-                ok = mbar_wait(bar_pv, (j - 1) & 1);
+            // rare: a running max moved by more than the slack. O must be rescaled, which needs the previous
+            // block's O += P V to have finished. (P_j itself goes to its own buffer and needs no wait.)
+            if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                ok = mbar_wait(bar_pv + ((j - 1) & 1) * 8, ((j - 1) >> 1) & 1);
                 tc_fence_after_sync();
                 lap(3);
-                if (__any_sync(0xffffffffu, alpha != 1.f)) {  // rare: rescale this warp's rows of O
+                {
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         uint32_t o[32];
@@ -322,8 +317,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 }
             }
 #pragma unroll
-            for (int c = 0; c < kBlock / 64; ++c)
-                tmem_st32(tm + lane_base + kColP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(pk + c * 32));
+            for (int c = 0; c < kBlock / 64; ++c) tmem_st32(buf + c * 32, *reinterpret_cast<uint32_t(*)[32]>(pk + c * 32));
             tmem_wait_st();
             // V rows past the context inside the last page may hold NaN; 0 * NaN is NaN, so clear them
             const int valid_rows = L - t0;
@@ -352,7 +346,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         }
 
         // ---- epilogue: O / l -> bf16 rows
-        if (ok) ok = mbar_wait(bar_pv, (nb - 1) & 1);
+        if (ok) ok = mbar_wait(bar_pv + ((nb - 1) & 1) * 8, ((nb - 1) >> 1) & 1);
         tc_fence_after_sync();
         const float inv = 1.f / l_run;
         __nv_bfloat16 *orow = p.out + (static_cast<size_t>(q0 + tile_start + tok) * p.Hq + kvh * G + head) * kD;
@@ -426,7 +420,7 @@ __global__ void advance_lens_kernel(const AppendTokensParams p) {
 
 }  // namespace
 
-size_t prefill_smem_bytes() { return kQBytes + 2 * kStages * kTileBytes + 1024 + (4 * kStages + 4) * 8 + 64; }
+size_t prefill_smem_bytes() { return kQBytes + 2 * kStages * kTileBytes + 1024 + (2 * kStages + 5) * 8 + 64; }
 
 cudaError_t prepare_prefill_attn() {
     return cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
