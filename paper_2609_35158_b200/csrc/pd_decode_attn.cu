@@ -324,18 +324,24 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
             if (lane == 0) latch_status(p.status, kDevBadPage, prod.b, pid);
             pid = 0;
         }
-        if (lane == 0) {
-            my_stage_range[p_stage] = p_rid;
+        {
+            // one TMA box per lane in a single warp instruction (lanes 0 .. 2*HALVES-1: K halves, then V
+            // halves); issued one after another by one lane the boxes cost that lane ~170 cycles each
             const int32_t y = (pid * p.Hkv + prod.kvh) * kPageSize;
             const uint32_t dst = ring + p_stage * STAGE_BYTES;
             const uint32_t bk = bar0 + p_stage * 16, bv = bk + 8;
-            mbar_arrive_expect_tx(bk, TILE_BYTES);
-#pragma unroll
-            for (int h = 0; h < HALVES; ++h) tma_load_2d(dst + h * HALF_BYTES, &tm_k, h * 64, y, bk, policy);
-            mbar_arrive_expect_tx(bv, TILE_BYTES);
-#pragma unroll
-            for (int h = 0; h < HALVES; ++h)
-                tma_load_2d(dst + TILE_BYTES + h * HALF_BYTES, &tm_v, h * 64, y, bv, policy);
+            if (lane == 0) {
+                my_stage_range[p_stage] = p_rid;
+                mbar_arrive_expect_tx(bk, TILE_BYTES);
+                mbar_arrive_expect_tx(bv, TILE_BYTES);
+            }
+            __syncwarp();
+            if (lane < 2 * HALVES) {
+                const bool is_v = lane >= HALVES;
+                const int h = is_v ? lane - HALVES : lane;
+                tma_load_2d(dst + (is_v ? TILE_BYTES : 0) + h * HALF_BYTES, is_v ? static_cast<const void *>(&tm_v) : &tm_k,
+                            h * 64, y, is_v ? bv : bk, policy);
+            }
         }
         advance(prod, cum, p.B, p.Hkv);
         --p_left;
