@@ -154,7 +154,7 @@ int pd_decode_step_host(pd_ctx *ctx, const void *q_host, const void *k_new_host,
  * pd_prefill_attn expects the cache to hold the new tokens already and
  * ctx_lens[b] = L_b to count them: query i of sequence b sits at position
  * L_b - q_len_b + i and out = softmax(sm_scale * q . K_{0..pos}^T) V_{0..pos}.
- * head_dim must be 128 (PD_ERR_UNSUPPORTED otherwise). The kernel runs on the
+ * The kernel runs on the
  * tcgen05 tensor cores with fp32 accumulation; P is rounded to bf16 before the
  * second product.
  */

@@ -420,7 +420,6 @@ int pd_prefill_attn(pd_ctx *ctx, const void *q, const int32_t *q_indptr, const v
                     const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse, int32_t batch,
                     int32_t max_q_len, float sm_scale, void *stream) {
     if (int rc = check_batch(ctx, batch)) return rc;
-    if (ctx->cfg.head_dim != 128) return fail(ctx, PD_ERR_UNSUPPORTED, "pd_prefill_attn: head_dim must be 128");
     if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(out) || q_indptr == nullptr ||
         page_table == nullptr || ctx_lens == nullptr)
         return fail(ctx, PD_ERR_INVALID_ARG, "pd_prefill_attn: null or misaligned pointer");
@@ -430,7 +429,7 @@ int pd_prefill_attn(pd_ctx *ctx, const void *q, const int32_t *q_indptr, const v
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
     if (!ctx->prefill_ready) {
-        const cudaError_t e = pd::prepare_prefill_attn();
+        const cudaError_t e = pd::prepare_prefill_attn(ctx->cfg.head_dim);
         if (e != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "prefill kernel attribute", e);
         ctx->prefill_ready = true;
     }
@@ -461,7 +460,8 @@ int pd_prefill_attn(pd_ctx *ctx, const void *q, const int32_t *q_indptr, const v
     p.trace = ctx->trace;                    // the worker-trace buffer doubles as [CTA][16] phase counters
     p.trace_ctas = ctx->trace_workers / 4;
     if (ctx->trace != nullptr) cudaMemsetAsync(ctx->trace, 0, static_cast<size_t>(ctx->trace_workers) * 32, static_cast<cudaStream_t>(stream));
-    const cudaError_t err = pd::launch_prefill_attn(ctx->tm_k, ctx->tm_v, p, max_q_len, static_cast<cudaStream_t>(stream));
+    const cudaError_t err = pd::launch_prefill_attn(ctx->cfg.head_dim, ctx->tm_k, ctx->tm_v, p, max_q_len,
+                                                    static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "prefill_attn launch", err);
     ctx->launches += 1;
     return PD_OK;

@@ -132,9 +132,9 @@ cudaError_t prepare_decode_attn(const AttnVariant &v, size_t *smem_bytes);  // o
 cudaError_t launch_decode_attn(const AttnVariant &v, const CUtensorMap &tm_k, const CUtensorMap &tm_v,
                                const AttnParams &p, int num_ctas, size_t smem_bytes, cudaStream_t stream);
 cudaError_t launch_lse_merge(int head_dim, const AttnParams &p, cudaStream_t stream);
-cudaError_t prepare_prefill_attn();  // opt-in shared memory, once
-cudaError_t launch_prefill_attn(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const PrefillParams &p, int max_q_len,
-                                cudaStream_t stream);
+cudaError_t prepare_prefill_attn(int head_dim);  // opt-in shared memory, once
+cudaError_t launch_prefill_attn(int head_dim, const CUtensorMap &tm_k, const CUtensorMap &tm_v, const PrefillParams &p,
+                                int max_q_len, cudaStream_t stream);
 cudaError_t launch_kv_append_tokens(const AppendTokensParams &p, int max_q_len, cudaStream_t stream);
 cudaError_t launch_kv_transfer(const TransferParams &p, bool scatter, int num_sms, cudaStream_t stream);
 

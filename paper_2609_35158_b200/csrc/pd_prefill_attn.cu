@@ -40,11 +40,8 @@ constexpr int kRows = 128;                    // query rows per CTA (MMA M), one
 constexpr int kThreads = kRows + 128;         // plus four service warps: S MMAs, O MMAs, K loads, V loads
 constexpr int kBlock = 64;                    // context tokens per step (MMA N of S, K of O)
 constexpr int kPagesPerBlock = kBlock / kPageSize;
-constexpr int kD = 128;
 constexpr int kQHalfBytes = kRows * 128;      // one 64-column half of the 128-row Q tile: 16 KB
-constexpr int kQBytes = 2 * kQHalfBytes;
 constexpr int kHalfBytes = kBlock * 128;      // one 64-column half of a K or V tile of kBlock tokens
-constexpr int kTileBytes = 2 * kHalfBytes;
 constexpr int kStages = 2;                    // K ring and V ring have two tiles each
 static_assert(kStages == 2, "ring slots and logit buffers share the index j % 2 and its barriers");
 // Two CTAs share an SM (96 KB of shared memory and 256 tensor-memory columns each): while one runs its
@@ -61,9 +58,13 @@ __device__ __forceinline__ void latch(int32_t *status, int code, int seq, int de
     }
 }
 
+template <int kD>
 __global__ void __launch_bounds__(kThreads, 2)
 prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                     const PrefillParams p) {
+    constexpr int kHalves = kD / 64;               // 64-column (128-byte) halves of a head row
+    constexpr int kQBytes = kHalves * kQHalfBytes;
+    constexpr int kTileBytes = kHalves * kHalfBytes;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_slot;
     const int tid = threadIdx.x, warp = tid >> 5;
@@ -116,7 +117,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         const uint4 *src = reinterpret_cast<const uint4 *>(
             p.q + (static_cast<size_t>(q0 + tile_start + tok) * p.Hq + kvh * G + head) * kD);
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
+        for (int c = 0; c < kD / 8; ++c) {
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
             if (row_valid) v = __ldg(src + c);
             const uint32_t a = q_s + (c >> 3) * kQHalfBytes + sw128_offset(tid, c & 7);
@@ -145,7 +146,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 tc_fence_after_sync();
                 const uint32_t kst = k_ring + (j % kStages) * kTileBytes;
 #pragma unroll
-                for (int h = 0; h < 2; ++h)
+                for (int h = 0; h < kHalves; ++h)
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
                         umma_ss(tm + kColS + (j & 1) * kBlock, umma_smem_desc(q_s + h * kQHalfBytes + ks * 32, 16, 1024),
@@ -173,7 +174,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         }
     } else if (warp >= kRows / 32 + 2) {
         // ================= two TMA warps (one streams K, the other V): one box per lane =================
-        // A tile of 64 tokens is 4 pages x 2 halves = 8 boxes of 2 KB. Issued one after another by a single
+        // A tile of 64 tokens is 4 pages x (D / 64) halves = 8 (or 4) boxes of 2 KB. Issued one after another by a single
         // thread they cost ~170 cycles each; here lane l issues box l of the tile in one warp instruction.
         // Page ids are fetched 32 at a time (one per lane), a group ahead of need.
         const int lane = tid & 31;
@@ -194,20 +195,20 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 c.grp = grp;
                 c.nval = load_group(grp + 1);
             }
-            const int pg = (lane >> 1) & (kPagesPerBlock - 1), h = lane & 1;
+            const int pg = (lane / kHalves) & (kPagesPerBlock - 1), h = lane % kHalves;
             const int lp = j * kPagesPerBlock + pg;
             int pid = __shfl_sync(0xffffffffu, c.val, lp & 31);
             int32_t y = oob_row;
             if (lp < n_pages) {
                 if (pid < 0 || pid >= p.num_pages) {
-                    if (lane < 2 * kPagesPerBlock && h == 0) latch(p.status, kDevBadPage, b, pid);
+                    if (lane < kHalves * kPagesPerBlock && h == 0) latch(p.status, kDevBadPage, b, pid);
                     pid = 0;
                 }
                 y = (pid * p.Hkv + kvh) * kPageSize;
             }
             if (lane == 0) mbar_arrive_expect_tx(bar, kTileBytes);
             __syncwarp();
-            if (lane < 2 * kPagesPerBlock)
+            if (lane < kHalves * kPagesPerBlock)
                 tma_load_2d(st + h * kHalfBytes + pg * (kPageSize * 128), map, h * 64, y, bar, policy);
         };
         // K and V have separate warps so that neither stream waits for the other's ring slot: a K tile is
@@ -306,7 +307,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 lap(3);
                 {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
+                    for (int c = 0; c < kD / 32; ++c) {
                         uint32_t o[32];
                         tmem_ld32(tm + lane_base + kColO + c * 32, o);
                         tmem_wait_ld();
@@ -325,8 +326,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 const uint32_t vst = v_ring + (j % kStages) * kTileBytes;
                 ok = ok && mbar_wait(bar_v + (j % kStages) * 8, (j / kStages) & 1);  // the tile must have landed
                 const int last = min(kBlock, (valid_rows + kPageSize - 1) / kPageSize * kPageSize);
-                for (int i = tid; i < (last - valid_rows) * 16; i += kRows) {
-                    const int r = valid_rows + (i >> 4), c = i & 15;
+                for (int i = tid; i < (last - valid_rows) * (kD / 8); i += kRows) {
+                    const int r = valid_rows + i / (kD / 8), c = i % (kD / 8);
                     st_shared_zero16(vst + (c >> 3) * kHalfBytes + r * 128 + (c & 7) * 16);
                 }
                 fence_proxy_async();
@@ -351,7 +352,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         const float inv = 1.f / l_run;
         __nv_bfloat16 *orow = p.out + (static_cast<size_t>(q0 + tile_start + tok) * p.Hq + kvh * G + head) * kD;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < kD / 32; ++c) {
             uint32_t o[32];
             tmem_ld32(tm + lane_base + kColO + c * 32, o);
             tmem_wait_ld();
@@ -420,19 +421,27 @@ __global__ void advance_lens_kernel(const AppendTokensParams p) {
 
 }  // namespace
 
-size_t prefill_smem_bytes() { return kQBytes + 2 * kStages * kTileBytes + 1024 + (2 * kStages + 5) * 8 + 64; }
-
-cudaError_t prepare_prefill_attn() {
-    return cudaFuncSetAttribute(prefill_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                static_cast<int>(prefill_smem_bytes()));
+size_t prefill_smem_bytes(int head_dim) {
+    const int halves = head_dim / 64;
+    return static_cast<size_t>(halves) * (kQHalfBytes + 2 * kStages * kHalfBytes) + 1024 + (2 * kStages + 5) * 8 + 64;
 }
 
-cudaError_t launch_prefill_attn(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const PrefillParams &p, int max_q_len,
-                                cudaStream_t stream) {
+cudaError_t prepare_prefill_attn(int head_dim) {
+    const int bytes = static_cast<int>(prefill_smem_bytes(head_dim));
+    if (head_dim == 128)
+        return cudaFuncSetAttribute(prefill_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    return cudaFuncSetAttribute(prefill_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
+cudaError_t launch_prefill_attn(int head_dim, const CUtensorMap &tm_k, const CUtensorMap &tm_v, const PrefillParams &p,
+                                int max_q_len, cudaStream_t stream) {
     if (p.B == 0 || max_q_len <= 0) return cudaSuccess;
     const int tok = kRows / p.G;
     const dim3 grid((max_q_len + tok - 1) / tok, p.Hkv, p.B);
-    return launch_pdl(prefill_attn_kernel, grid, dim3(kThreads), prefill_smem_bytes(), stream, p.pdl != 0, tm_k, tm_v, p);
+    const size_t smem = prefill_smem_bytes(head_dim);
+    if (head_dim == 128)
+        return launch_pdl(prefill_attn_kernel<128>, grid, dim3(kThreads), smem, stream, p.pdl != 0, tm_k, tm_v, p);
+    return launch_pdl(prefill_attn_kernel<64>, grid, dim3(kThreads), smem, stream, p.pdl != 0, tm_k, tm_v, p);
 }
 
 cudaError_t launch_kv_append_tokens(const AppendTokensParams &p, int max_q_len, cudaStream_t stream) {

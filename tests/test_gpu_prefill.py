@@ -24,9 +24,8 @@ def run_prefill(ctx, cache, q, ip, lens_dev, scale, max_q_len):
     return out, lse
 
 
-@pytest.mark.parametrize("Hq,Hkv", [(32, 8), (32, 4), (8, 8), (4, 2)])
-def test_prefill_small_ragged_poisoned(Hq, Hkv):
-    d = 128
+@pytest.mark.parametrize("Hq,Hkv,d", [(32, 8, 128), (32, 4, 128), (8, 8, 128), (4, 2, 128), (8, 2, 64), (16, 2, 64)])
+def test_prefill_small_ragged_poisoned(Hq, Hkv, d):
     lens = np.array([70, 33, 5, 40, 300, 129, 1000, 128], dtype=np.int32)
     q_lens = np.array([20, 33, 1, 0, 37, 129, 200, 16], dtype=np.int32)
     cache = wl.build_paged_cache(lens, Hkv, d, seed=100 + Hq, device=DEV, poison=True)
@@ -37,7 +36,7 @@ def test_prefill_small_ragged_poisoned(Hq, Hkv):
         out, lse = run_prefill(ctx, cache, q, torch.from_numpy(ip).to(DEV), cache.ctx_lens, scale, int(q_lens.max()))
     ref, ref_lse = oracle.prefill_attn(oracle.bf16_bits(q), ip, oracle.bf16_bits(cache.k_pages),
                                        oracle.bf16_bits(cache.v_pages), cache.page_table_host, lens, scale)
-    assert_parity(out, ref, f"prefill {Hq}/{Hkv}", scale_abs_by_magnitude=True)
+    assert_parity(out, ref, f"prefill {Hq}/{Hkv}/{d}", scale_abs_by_magnitude=True)
     np.testing.assert_allclose(lse.cpu().numpy(), ref_lse, rtol=3e-5, atol=3e-5)
 
 

@@ -56,7 +56,7 @@ def test_decode_random_case(seed):
 @pytest.mark.parametrize("seed", range(12))
 def test_prefill_random_case(seed):
     rng = np.random.default_rng(5000 + seed)
-    d = 128
+    d = int(rng.choice([64, 128]))
     g = int(rng.choice([1, 2, 4, 8]))
     Hkv = int(rng.choice([1, 2, 4]))
     Hq = g * Hkv
@@ -84,6 +84,6 @@ def test_prefill_random_case(seed):
         assert ctx.pd.pd_device_status(ctx.h)[0] == 0
     ref, ref_lse = oracle.prefill_attn(oracle.bf16_bits(q), ip, oracle.bf16_bits(cache.k_pages),
                                        oracle.bf16_bits(cache.v_pages), cache.page_table_host, lens, scale)
-    what = f"seed {seed}: {Hq}/{Hkv} q_lens={q_lens.tolist()} prefix={prefix.tolist()}"
+    what = f"seed {seed}: {Hq}/{Hkv} d={d} q_lens={q_lens.tolist()} prefix={prefix.tolist()}"
     assert_parity(out, ref, what, scale_abs_by_magnitude=True)
     np.testing.assert_allclose(lse.cpu().numpy(), ref_lse, rtol=3e-5, atol=3e-5, err_msg=what)
