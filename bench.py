@@ -183,9 +183,13 @@ def run_cuda(args):
     def device_step(i):
         nonlocal lens
         allocate_pages()
-        pd.pd_kv_append(ctx, kns[i % R], vns[i % R], cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens)
-        pd.pd_decode_attn(ctx, qs[i % R], cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, out,
-                          sm_scale=w.sm_scale)
+        if args.step == "fused":
+            pd.pd_decode_step(ctx, qs[i % R], kns[i % R], vns[i % R], cache.k_pages, cache.v_pages, cache.page_table,
+                              cache.ctx_lens, out, sm_scale=w.sm_scale)
+        else:
+            pd.pd_kv_append(ctx, kns[i % R], vns[i % R], cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens)
+            pd.pd_decode_attn(ctx, qs[i % R], cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, out,
+                              sm_scale=w.sm_scale)
         lens = lens + 1
         return int(lens.sum()) * bpt  # KV bytes this step's attention must read
 
@@ -710,6 +714,8 @@ def main():
     ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--step", default="fused", choices=["separate", "fused"],
+                    help="decode: pd_kv_append + pd_decode_attn (3 launches) or pd_decode_step (2 launches)")
     ap.add_argument("--op", default="decode", choices=["decode", "kv_transfer", "prefill", "fit_b"],
                     help="decode = the headline decode step; kv_transfer = page gather + scatter; "
                          "prefill = one append-prefill turn; fit_b = decode step time over batch size, fitted to A + b * B")

@@ -119,10 +119,28 @@ int pd_decode_attn(pd_ctx *ctx, const void *q, const void *k_pages, const void *
                    int32_t batch, float sm_scale, int32_t split_pages, void *stream);
 
 /*
+ * One decode step in two launches (Sec. 2.1: the new token joins the context,
+ * then attends over it): the result is that of pd_kv_append (advancing)
+ * followed by pd_decode_attn, but the append runs inside the split kernel.
+ * ctx_lens holds the lengths BEFORE the append on entry and the grown lengths
+ * after the kernels ran. The worker that reads a sequence's last page takes
+ * the new token's K/V rows from k_new / v_new instead of the pool (whatever
+ * the pool held in that slot is ignored) and stores them to the pool, bit for
+ * bit. Error behaviour as pd_kv_append: a sequence with no room in its table
+ * row or a bad page id at the new position is latched for pd_device_status,
+ * its pools and length stay as they were (its output is then unspecified).
+ * Shapes as pd_kv_append and pd_decode_attn; out rows of the step are
+ * attention over ctx_lens[b] + 1 tokens.
+ */
+int pd_decode_step(pd_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *k_pages,
+                   void *v_pages, const int32_t *page_table, int32_t *ctx_lens, void *out, float *lse,
+                   int32_t batch, float sm_scale, int32_t split_pages, void *stream);
+
+/*
  * One whole decode step for callers that hold the step's activations on the
  * HOST: copies q_host, k_new_host, v_new_host (host pointers, pinned or
- * pageable, same shapes as q/k_new/v_new) to device staging, runs pd_kv_append
- * (advancing ctx_lens) then pd_decode_attn over the grown contexts, copies the
+ * pageable, same shapes as q/k_new/v_new) to device staging, runs pd_decode_step
+ * (appending, advancing ctx_lens, attending over the grown contexts), copies the
  * result to out_host (host, [batch][num_q_heads][head_dim] bf16) and waits for
  * the stream, so out_host is valid on return. The cache itself (k_pages,
  * v_pages, page_table, ctx_lens) stays on the device.

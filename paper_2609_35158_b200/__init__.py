@@ -26,7 +26,7 @@ PD_APPEND_NO_ADVANCE = 1
 
 # every symbol include/pd.h declares
 EXPORTS = (
-    "pd_create", "pd_destroy", "pd_kv_append", "pd_decode_attn", "pd_decode_attn_static", "pd_decode_step_host",
+    "pd_create", "pd_destroy", "pd_kv_append", "pd_decode_attn", "pd_decode_attn_static", "pd_decode_step", "pd_decode_step_host",
     "pd_kv_gather", "pd_kv_scatter", "pd_kv_append_tokens", "pd_prefill_attn", "pd_device_status", "pd_read_worker_trace",
     "pd_makespan_coloc", "pd_makespan_disagg", "pd_feasible_disagg", "pd_decide", "pd_min_change_plan", "pd_toggle_gate",
     "pd_fit_decode_cost",
@@ -77,6 +77,7 @@ def _load() -> ctypes.CDLL:
     lib.pd_prefill_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp]
     lib.pd_kv_gather.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.pd_kv_scatter.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp]
+    lib.pd_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, vp]
     lib.pd_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, vp]
     lib.pd_device_status.argtypes = [vp, vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
     lib.pd_set_profile_events.argtypes = [vp, vp, vp]
@@ -204,6 +205,14 @@ def pd_decode_attn_static(cfg: pd_config, q, k_pages, v_pages, page_table, ctx_l
     _check(_lib.pd_decode_attn_static(ctypes.byref(cfg), _ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(page_table),
                                       _ptr(ctx_lens), _ptr(out), _ptr(lse), batch, sm_scale, _stream(stream)),
            "pd_decode_attn_static")
+
+
+def pd_decode_step(ctx, q, k_new, v_new, k_pages, v_pages, page_table, ctx_lens, out, lse=None, batch=None,
+                   sm_scale=1.0, split_pages=0, stream=None):
+    batch = q.shape[0] if batch is None else batch
+    _check(_lib.pd_decode_step(ctx, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pages), _ptr(v_pages), _ptr(page_table),
+                               _ptr(ctx_lens), _ptr(out), _ptr(lse), batch, sm_scale, split_pages, _stream(stream)),
+           "pd_decode_step", ctx)
 
 
 def pd_decode_step_host(ctx, q_host, k_new_host, v_new_host, k_pages, v_pages, page_table, ctx_lens, out_host,

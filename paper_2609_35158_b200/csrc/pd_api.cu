@@ -322,13 +322,23 @@ int pd_kv_scatter(pd_ctx *ctx, const void *packed, const int64_t *packed_page_of
                        const_cast<void *>(packed), batch, stream);
 }
 
-int pd_decode_attn(pd_ctx *ctx, const void *q, const void *k_pages, const void *v_pages, const int32_t *page_table,
-                   const int32_t *ctx_lens, void *out, float *lse, int32_t batch, float sm_scale, int32_t split_pages,
-                   void *stream) {
+}  // extern "C"
+
+namespace {
+
+// Split kernel + merge kernel. With k_new / v_new the split kernel also appends one token per sequence
+// (the pools and the lengths are then written) and attends over the grown contexts.
+int decode_attn_impl(pd_ctx *ctx, const char *who, const void *q, const void *k_new, const void *v_new, const void *k_pages,
+                     const void *v_pages, const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse,
+                     int32_t batch, float sm_scale, int32_t split_pages, void *stream) {
+    const bool fused = k_new != nullptr;
     if (int rc = check_batch(ctx, batch)) return rc;
     if (!aligned16(q) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(out) || page_table == nullptr ||
-        ctx_lens == nullptr)
-        return fail(ctx, PD_ERR_INVALID_ARG, "pd_decode_attn: null or misaligned pointer");
+        ctx_lens == nullptr || (fused && (!aligned16(k_new) || !aligned16(v_new)))) {
+        char msg[96];
+        std::snprintf(msg, sizeof msg, "%s: null or misaligned pointer", who);
+        return fail(ctx, PD_ERR_INVALID_ARG, msg);
+    }
     if (!(sm_scale > 0.f) || !(sm_scale < 3.0e38f)) return fail(ctx, PD_ERR_INVALID_ARG, "sm_scale must be finite and positive");
     if (split_pages < 0) return fail(ctx, PD_ERR_INVALID_ARG, "split_pages must be >= 0");
     if (batch == 0) return PD_OK;
@@ -369,6 +379,14 @@ int pd_decode_attn(pd_ctx *ctx, const void *q, const void *k_pages, const void *
     p.pdl = hooked ? 0 : ctx->pdl;  // timing events must bracket the split kernel alone: no overlap with neighbours
     p.merge_rows = ctx->merge_rows;
     p.trace = ctx->trace;
+    if (fused) {
+        p.k_new = static_cast<const __nv_bfloat16 *>(k_new);
+        p.v_new = static_cast<const __nv_bfloat16 *>(v_new);
+        p.k_pool_w = static_cast<__nv_bfloat16 *>(const_cast<void *>(k_pages));
+        p.v_pool_w = static_cast<__nv_bfloat16 *>(const_cast<void *>(v_pages));
+        p.ctx_lens_w = const_cast<int32_t *>(ctx_lens);
+        p.fused = 1;
+    }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (hooked) cudaEventRecord(ctx->ev_before, s);
     cudaError_t err = pd::launch_decode_attn(ctx->variant, ctx->tm_k, ctx->tm_v, p, ctx->num_ctas, ctx->smem_bytes, s);
@@ -382,6 +400,26 @@ int pd_decode_attn(pd_ctx *ctx, const void *q, const void *k_pages, const void *
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "lse_merge launch", err);
     ctx->launches += 2;
     return PD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int pd_decode_attn(pd_ctx *ctx, const void *q, const void *k_pages, const void *v_pages, const int32_t *page_table,
+                   const int32_t *ctx_lens, void *out, float *lse, int32_t batch, float sm_scale, int32_t split_pages,
+                   void *stream) {
+    return decode_attn_impl(ctx, "pd_decode_attn", q, nullptr, nullptr, k_pages, v_pages, page_table, ctx_lens, out, lse,
+                            batch, sm_scale, split_pages, stream);
+}
+
+int pd_decode_step(pd_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *k_pages, void *v_pages,
+                   const int32_t *page_table, int32_t *ctx_lens, void *out, float *lse, int32_t batch, float sm_scale,
+                   int32_t split_pages, void *stream) {
+    if (ctx == nullptr) return PD_ERR_INVALID_ARG;
+    if (k_new == nullptr || v_new == nullptr) return fail(ctx, PD_ERR_INVALID_ARG, "pd_decode_step: null k_new / v_new");
+    return decode_attn_impl(ctx, "pd_decode_step", q, k_new, v_new, k_pages, v_pages, page_table, ctx_lens, out, lse, batch,
+                            sm_scale, split_pages, stream);
 }
 
 int pd_kv_append_tokens(pd_ctx *ctx, const void *k_new, const void *v_new, const int32_t *q_indptr, void *k_pages,
@@ -483,10 +521,8 @@ int pd_decode_step_host(pd_ctx *ctx, const void *q_host, const void *k_new_host,
     if (err == cudaSuccess) err = cudaMemcpyAsync(ctx->stage_k, k_new_host, nkv, cudaMemcpyHostToDevice, s);
     if (err == cudaSuccess) err = cudaMemcpyAsync(ctx->stage_v, v_new_host, nkv, cudaMemcpyHostToDevice, s);
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "host-to-device copy", err);
-    if (int rc = pd_kv_append(ctx, ctx->stage_k, ctx->stage_v, k_pages, v_pages, page_table, ctx_lens, batch, 0, stream))
-        return rc;
-    if (int rc = pd_decode_attn(ctx, ctx->stage_q, k_pages, v_pages, page_table, ctx_lens, ctx->stage_out, nullptr, batch,
-                                sm_scale, split_pages, stream))
+    if (int rc = pd_decode_step(ctx, ctx->stage_q, ctx->stage_k, ctx->stage_v, k_pages, v_pages, page_table, ctx_lens,
+                                ctx->stage_out, nullptr, batch, sm_scale, split_pages, stream))
         return rc;
     err = cudaMemcpyAsync(out_host, ctx->stage_out, nq, cudaMemcpyDeviceToHost, s);
     if (err == cudaSuccess) err = cudaStreamSynchronize(s);

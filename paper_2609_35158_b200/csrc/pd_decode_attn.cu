@@ -91,8 +91,8 @@ __device__ void scan_pages(const AttnParams &p, int32_t *cum, int32_t *warp_sums
     const int begin = min(p.B, tid * items), end = min(p.B, begin + items);
     int sum = 0;
     for (int i = begin; i < end; ++i) {
-        const int L = __ldg(p.ctx_lens + i);
-        if (L < 0 || L > p.MP * kPageSize) latch_status(p.status, kDevBadLength, i, L);
+        const int L = __ldg(p.ctx_lens + i) + p.fused;
+        if (L < p.fused || L > p.MP * kPageSize) latch_status(p.status, kDevBadLength, i, L - p.fused);
         sum += (clamp_len(L, p.MP) + kPageSize - 1) / kPageSize;
     }
     int incl = sum;
@@ -108,7 +108,7 @@ __device__ void scan_pages(const AttnParams &p, int32_t *cum, int32_t *warp_sums
     int run = base + incl - sum;
     for (int i = begin; i < end; ++i) {
         cum[i] = run;
-        run += (clamp_len(__ldg(p.ctx_lens + i), p.MP) + kPageSize - 1) / kPageSize;
+        run += (clamp_len(__ldg(p.ctx_lens + i) + p.fused, p.MP) + kPageSize - 1) / kPageSize;
     }
     if (tid == THREADS - 1) cum[p.B] = run;
     __syncthreads();
@@ -228,7 +228,8 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + WARPS * STAGES * STAGE_BYTES);
     Plan *plan_s = reinterpret_cast<Plan *>(bars + WARPS * STAGES * 2);
     int32_t *stage_range = reinterpret_cast<int32_t *>(plan_s + 1);  // [WARPS][STAGES] range id of the page in a stage
-    int32_t *warp_sums = stage_range + WARPS * STAGES;
+    int32_t *stage_pid = stage_range + WARPS * STAGES;  // [WARPS][STAGES] physical page in a stage, -1 if it was clamped
+    int32_t *warp_sums = stage_pid + WARPS * STAGES;
     int32_t *cum = warp_sums + 32;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -275,6 +276,7 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     const uint32_t ring = ring0 + warp * STAGES * STAGE_BYTES;
     const uint32_t bar0 = smem_u32(bars + warp * STAGES * 2);
     int32_t *my_stage_range = stage_range + warp * STAGES;
+    int32_t *my_stage_pid = stage_pid + warp * STAGES;
     const uint64_t policy = l2_policy_evict_first();
     const int quad_row = lane >> 2;        // B-fragment column of this lane: the query head whose Q it holds
     const int quad_col = (lane & 3) * 2;   // accumulator columns of this lane: heads quad_col and quad_col + 1
@@ -320,9 +322,11 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
             p_rid = rid;
         }
         int pid = page_id(pt, p, prod.b, prod.page, lane);
+        bool pid_ok = true;
         if (pid < 0 || pid >= p.num_pages) {
             if (lane == 0) latch_status(p.status, kDevBadPage, prod.b, pid);
             pid = 0;
+            pid_ok = false;
         }
         {
             // one TMA box per lane in a single warp instruction (lanes 0 .. 2*HALVES-1: K halves, then V
@@ -332,6 +336,7 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
             const uint32_t bk = bar0 + p_stage * 16, bv = bk + 8;
             if (lane == 0) {
                 my_stage_range[p_stage] = p_rid;
+                my_stage_pid[p_stage] = pid_ok ? pid : -1;
                 mbar_arrive_expect_tx(bk, TILE_BYTES);
                 mbar_arrive_expect_tx(bv, TILE_BYTES);
             }
@@ -362,7 +367,7 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     cons.b = 0; cons.kvh = 0; cons.page = 0; cons.np = 1;
     int c_rid = -1, c_left = 0;
     uint32_t stage = 0, parity = 0;  // ring position of the next page to consume
-    bool alive = true, seg_open = false;
+    bool alive = true, seg_open = false, seg_append = false;
     int seg_page0 = 0, L = 0;
     uint32_t qb[KSTEPS][2];     // Q^T as the B operand: head quad_row, d = 16 kk + quad_col (+1), and +8
     float O[MTILES][4];          // O^T: rows d = 16 j + quad_row (+8), columns heads quad_col, quad_col + 1
@@ -378,7 +383,9 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         if (!seg_open) {  // first page of a segment: its queries, a fresh running state
             seg_open = true;
             seg_page0 = cons.page;
-            L = clamp_len(__ldg(p.ctx_lens + cons.b), p.MP);
+            const int L_raw = __ldg(p.ctx_lens + cons.b) + p.fused;
+            L = clamp_len(L_raw, p.MP);
+            seg_append = p.fused != 0 && L == L_raw && L > 0;  // never patch a row of a length that was clamped
             const __nv_bfloat16 *qrow = p.q + (static_cast<size_t>(cons.b) * p.Hq + cons.kvh * G + quad_row) * D;
 #pragma unroll
             for (int kk = 0; kk < KSTEPS; ++kk) {
@@ -401,10 +408,37 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         const uint32_t bk = bar0 + stage * 16, bv = bk + 8;
         const int valid = L - cons.page * kPageSize;  // tokens of this page inside the context
 
+        // fused append: the page that receives the new token is the last one of the pair. Its K and V rows
+        // come from k_new / v_new: they are patched into the tile in shared memory (the pool still holds
+        // whatever was in that slot) and written to the pool, which is the append itself.
+        const bool appending = seg_append && cons.page == cons.np - 1;
+        const int new_slot = (L - 1) & (kPageSize - 1);
+        uint4 new_row = make_uint4(0u, 0u, 0u, 0u);
+        constexpr int ROW_CHUNKS = D / 8;  // 16-byte chunks of one K (or V) row: lanes [0, ROW_CHUNKS) K, the next ones V
+        if (appending && lane < 2 * ROW_CHUNKS) {
+            const bool is_v = lane >= ROW_CHUNKS;
+            const int c = is_v ? lane - ROW_CHUNKS : lane;
+            const __nv_bfloat16 *src = (is_v ? p.v_new : p.k_new) + (static_cast<size_t>(cons.b) * p.Hkv + cons.kvh) * D + c * 8;
+            new_row = __ldg(reinterpret_cast<const uint4 *>(src));
+            const int pid = my_stage_pid[stage];
+            if (pid >= 0) {
+                __nv_bfloat16 *dst = (is_v ? p.v_pool_w : p.k_pool_w) +
+                                     ((static_cast<size_t>(pid) * p.Hkv + cons.kvh) * kPageSize + new_slot) * D + c * 8;
+                *reinterpret_cast<uint4 *>(dst) = new_row;
+            }
+        }
         if (!__all_sync(0xffffffffu, mbar_wait(bk, parity))) { alive = false; break; }
         if (p.trace != nullptr) {
             t_last = global_timer_ns();
             if (t_first == 0ull) t_first = t_last;
+        }
+        if (appending) {
+            if (lane < ROW_CHUNKS) {
+                const uint32_t a = kbase + (lane >> 3) * HALF_BYTES + new_slot * 128 + (((lane & 7) ^ (new_slot & 7)) << 4);
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(new_row.x), "r"(new_row.y),
+                             "r"(new_row.z), "r"(new_row.w) : "memory");
+            }
+            __syncwarp();
         }
 
         // S^T = K Q^T for the 16 tokens of the page (two accumulators shorten the dependent chain)
@@ -459,6 +493,15 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         }
 
         if (!__all_sync(0xffffffffu, mbar_wait(bv, parity))) { alive = false; break; }
+        if (appending) {
+            if (lane >= ROW_CHUNKS && lane < 2 * ROW_CHUNKS) {
+                const int c = lane - ROW_CHUNKS;
+                const uint32_t a = vbase + (c >> 3) * HALF_BYTES + new_slot * 128 + (((c & 7) ^ (new_slot & 7)) << 4);
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(new_row.x), "r"(new_row.y),
+                             "r"(new_row.z), "r"(new_row.w) : "memory");
+            }
+            __syncwarp();
+        }
         if (valid < kPageSize) {
             // V rows past the context may hold NaN; 0 * NaN is NaN, so clear them first
             for (int row = valid; row < kPageSize; ++row)
@@ -476,7 +519,7 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
             if (HILO) mma_bf16_16816(O[j], a0, a1, a2, a3, pl0, pl1);
         }
         __syncwarp();  // every lane has read this stage
-        if (valid < kPageSize) fence_proxy_async();  // generic-proxy stores before the next TMA write
+        if (valid < kPageSize || appending) fence_proxy_async();  // generic-proxy stores before the next TMA write
         --inflight;
         issue_next();  // refills the stage just freed (p_stage == stage here)
         if (++stage == STAGES) { stage = 0; parity ^= 1u; }
@@ -528,6 +571,7 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         advance(cons, cum, p.B, p.Hkv);
     }
 
+    bool last_worker = false;
     if (lane == 0) {
         if (!alive) latch_status(p.status, kDevTimeout, -1, worker);
         if (p.trace != nullptr) {
@@ -538,6 +582,16 @@ decode_attn_split_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         if (atomicAdd(p.status + kSchedDone, 1) == n_workers - 1) {
             p.status[kSchedNext] = 0;
             p.status[kSchedDone] = 0;
+            last_worker = true;
+        }
+    }
+    // fused append: the last worker to finish (every CTA has long read the old lengths) advances them
+    if (p.fused != 0 && __shfl_sync(0xffffffffu, static_cast<int>(last_worker), 0)) {
+        for (int i = lane; i < p.B; i += 32) {
+            const int Lold = p.ctx_lens_w[i];
+            if (Lold < 0 || Lold + 1 > p.MP * kPageSize) continue;  // latched as a bad length by the scan
+            const int pid = __ldg(p.page_table + static_cast<size_t>(i) * p.MP + Lold / kPageSize);
+            if (pid >= 0 && pid < p.num_pages) p.ctx_lens_w[i] = Lold + 1;  // a bad page id was latched by its reader
         }
     }
 }
@@ -668,7 +722,7 @@ template <int D, int WARPS, int STAGES, bool HILO>
 size_t smem_bytes_for() {
     // ring + 1 KB alignment slack + barriers + plan + stage tags + warp sums + prefix sums
     return static_cast<size_t>(WARPS) * STAGES * (2 * kPageSize * D * 2) + 1024 + WARPS * STAGES * 2 * 8 +
-           sizeof(Plan) + WARPS * STAGES * 4 + 32 * 4 + (kMaxBatch + 1) * 4;
+           sizeof(Plan) + 2 * WARPS * STAGES * 4 + 32 * 4 + (kMaxBatch + 1) * 4;
 }
 
 template <typename F>

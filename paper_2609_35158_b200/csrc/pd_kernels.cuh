@@ -46,6 +46,13 @@ struct AttnParams {
     int32_t halving_levels;     // automatic plan: number of levels whose ranges halve the remaining fair share
     int32_t tail_pages;         // automatic plan: pages per range of the last level
     int32_t pdl;                // launch with programmatic stream serialization
+    // fused one-token append (all null / 0 for plain attention): ctx_lens holds the lengths BEFORE the
+    // append; the kernel attends over ctx_lens + 1 tokens, takes the new token's K/V rows from k_new / v_new,
+    // writes them into the pools and finally adds 1 to every length
+    const __nv_bfloat16 *k_new, *v_new;  // [B][Hkv][D]
+    __nv_bfloat16 *k_pool_w, *v_pool_w;  // the pools, writable
+    int32_t *ctx_lens_w;
+    int32_t fused;
     int32_t merge_rows;         // rows per CTA of the merge kernel, 0 = chosen from the row count
     unsigned long long *trace;  // optional [workers][4] ns timestamps: kernel entry, first data, last data, exit
 };
