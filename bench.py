@@ -652,6 +652,57 @@ def run_fit_b(args):
     }), flush=True)
 
 
+# ------------------------------------------------------------------------------------------ pool toggle
+
+def run_pool_toggle(args):
+    """Wall time to release and to restore the physical memory of a KV pool of the multi-turn workload's size
+    (the KV-cache share of T_toggle in Eq. 7). Host driver calls, so the clock is the host's."""
+    import time
+
+    import torch
+
+    import paper_2609_35158_b200 as pd
+    import workloads as wl
+
+    torch.cuda.set_device(0)
+    w = wl.WORKLOADS[4]
+    lens = wl.context_lengths(4).astype(np.int64) + 128
+    pages = int(np.ceil(1.0625 * ((lens + 15) // 16).sum()))
+    cap = 2 * pages * w.num_kv_heads * 16 * w.head_dim * 2
+    reps = max(3, min(args.steps, 10))
+    rows = []
+    for chunk in (64 << 20, 256 << 20, 1 << 30):
+        pool = pd.pd_pool_create(0, cap, chunk)
+        rel, res, touch = [], [], []
+        for _ in range(reps):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            pd.pd_pool_resize(pool, pd.pd_pool_capacity(pool))
+            t1 = time.perf_counter()
+            whole = pd.pool_tensor(pool, 0, (pd.pd_pool_capacity(pool),), torch.uint8)
+            whole.zero_()  # first touch of the restored memory
+            torch.cuda.synchronize()
+            t2 = time.perf_counter()
+            del whole
+            pd.pd_pool_resize(pool, 0)
+            t3 = time.perf_counter()
+            res.append(t1 - t0)
+            touch.append(t2 - t1)
+            rel.append(t3 - t2)
+        rows.append({"chunk_mib": pd.pd_pool_chunk_bytes(pool) >> 20, "capacity_gb": round(pd.pd_pool_capacity(pool) / 1e9, 2),
+                     "restore_ms": round(1e3 * float(np.median(res)), 2), "first_write_ms": round(1e3 * float(np.median(touch)), 2),
+                     "release_ms": round(1e3 * float(np.median(rel)), 2)})
+        pd.pd_pool_destroy(pool)
+    best = min(rows, key=lambda r: r["restore_ms"] + r["release_ms"])
+    t_toggle = (best["restore_ms"] + best["release_ms"]) * 1e-3
+    print(json.dumps({
+        "metric": "KV pool release + restore wall time (KV share of T_toggle, Eq. 7)", "value": round(t_toggle * 1e3, 2),
+        "unit": "ms", "higher_is_better": False, "repetitions": reps, "by_chunk": rows,
+        "example_gate": {"assumed": "R/B = 0.25, T_ded = 60 s, T_full = 40 s",
+                         "borrow": bool(pd.pd_toggle_gate(16, 64, 60.0, 40.0, t_toggle))},
+    }), flush=True)
+
+
 # ------------------------------------------------------------------------------------------ reference arm
 
 def run_reference(args):
@@ -716,9 +767,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--step", default="fused", choices=["separate", "fused"],
                     help="decode: pd_kv_append + pd_decode_attn (3 launches) or pd_decode_step (2 launches)")
-    ap.add_argument("--op", default="decode", choices=["decode", "kv_transfer", "prefill", "fit_b"],
+    ap.add_argument("--op", default="decode", choices=["decode", "kv_transfer", "prefill", "fit_b", "pool_toggle"],
                     help="decode = the headline decode step; kv_transfer = page gather + scatter; "
-                         "prefill = one append-prefill turn; fit_b = decode step time over batch size, fitted to A + b * B")
+                         "prefill = one append-prefill turn; fit_b = decode step time over batch size, fitted to A + b * B; "
+                         "pool_toggle = release and restore of a KV pool's physical memory")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
@@ -730,6 +782,8 @@ def main():
         run_prefill(args)
     elif args.op == "fit_b":
         run_fit_b(args)
+    elif args.op == "pool_toggle":
+        run_pool_toggle(args)
     else:
         run_cuda(args)
 

@@ -355,6 +355,36 @@ int32_t pd_toggle_gate(double R, double B, double T_ded, double T_full, double T
 /* Least-squares line step_seconds = A + b * concurrency over n >= 2 measurements. */
 int pd_fit_decode_cost(const double *concurrency, const double *step_seconds, int32_t n, double *A, double *b);
 
+/* ---- Elastic KV pool on CUDA virtual memory management (Sec. 4.6: the intra-scale toggle keeps the
+ * rollout process and swaps device state; Sec. 5: the KV cache is released when training begins and
+ * restored when the GPU is available again). A pool is a device address range of `capacity` bytes whose
+ * first `resident` bytes are backed by physical memory, in chunks. Resizing changes the backing only:
+ * the base address, and with it page ids, pointers and tensor maps derived from it, stay valid across
+ * release and restore. Contents of a chunk are lost when it is released; a restored chunk holds
+ * unspecified bytes. The non-resident part of the range must not be accessed (the caller's page
+ * allocator must hand out only pages below resident_bytes). The wall time of pd_pool_resize(pool, 0)
+ * plus pd_pool_resize(pool, capacity) is the KV-cache share of T_toggle in Eq. 7.
+ * Host calls, synchronous; not thread-safe per pool. */
+typedef struct pd_pool pd_pool; /* opaque */
+
+/* Reserves the address range on `device`; nothing is resident yet. chunk_bytes = 0 picks 256 MiB; it is
+ * rounded up to the device's allocation granularity and capacity up to a whole number of chunks.
+ * PD_ERR_UNSUPPORTED if the driver lacks the virtual-memory calls. */
+int pd_pool_create(int32_t device, uint64_t capacity_bytes, uint64_t chunk_bytes, pd_pool **out);
+/* Makes ceil(resident_bytes / chunk) chunks resident, releasing or backing chunks at the end of the
+ * resident prefix. Before chunks are released the call waits for `stream_to_drain` (a cudaStream_t as
+ * void*; NULL = the whole device), so no kernel still touches them. PD_ERR_WORKSPACE when the device has
+ * no memory for a chunk (the chunks backed so far stay resident), PD_ERR_INVALID_ARG above capacity. */
+int pd_pool_resize(pd_pool *pool, uint64_t resident_bytes, void *stream_to_drain);
+/* Device pointer to the start of the range (256-byte aligned at least), fixed for the pool's lifetime. */
+void *pd_pool_base(const pd_pool *pool);
+uint64_t pd_pool_capacity(const pd_pool *pool);
+uint64_t pd_pool_chunk_bytes(const pd_pool *pool);
+uint64_t pd_pool_resident_bytes(const pd_pool *pool);
+const char *pd_pool_last_error(const pd_pool *pool);
+/* Synchronises the device, releases every chunk and the address range. NULL is accepted. */
+int pd_pool_destroy(pd_pool *pool);
+
 const char *pd_status_string(int status);
 
 /* Text of the most recent failure recorded by this context (CUDA error string

@@ -30,6 +30,8 @@ EXPORTS = (
     "pd_kv_gather", "pd_kv_scatter", "pd_kv_append_tokens", "pd_prefill_attn", "pd_device_status", "pd_read_worker_trace",
     "pd_makespan_coloc", "pd_makespan_disagg", "pd_feasible_disagg", "pd_decide", "pd_min_change_plan", "pd_toggle_gate",
     "pd_fit_decode_cost",
+    "pd_pool_create", "pd_pool_resize", "pd_pool_base", "pd_pool_capacity", "pd_pool_chunk_bytes", "pd_pool_resident_bytes",
+    "pd_pool_last_error", "pd_pool_destroy",
     "pd_set_profile_events", "pd_workspace_bytes", "pd_launch_count", "pd_last_plan", "pd_status_string", "pd_last_error", "pd_version",
 )
 
@@ -102,8 +104,21 @@ def _load() -> ctypes.CDLL:
     lib.pd_last_error.argtypes = [vp]
     lib.pd_last_error.restype = ctypes.c_char_p
     lib.pd_version.argtypes = []
+    u64 = ctypes.c_uint64
+    lib.pd_pool_create.argtypes = [i32, u64, u64, ctypes.POINTER(vp)]
+    lib.pd_pool_resize.argtypes = [vp, u64, vp]
+    lib.pd_pool_destroy.argtypes = [vp]
+    lib.pd_pool_base.argtypes = [vp]
+    lib.pd_pool_base.restype = vp
+    for name in ("pd_pool_capacity", "pd_pool_chunk_bytes", "pd_pool_resident_bytes"):
+        getattr(lib, name).argtypes = [vp]
+        getattr(lib, name).restype = u64
+    lib.pd_pool_last_error.argtypes = [vp]
+    lib.pd_pool_last_error.restype = ctypes.c_char_p
+    own_restype = ("pd_status_string", "pd_last_error", "pd_makespan_coloc", "pd_makespan_disagg", "pd_pool_base",
+                   "pd_pool_capacity", "pd_pool_chunk_bytes", "pd_pool_resident_bytes", "pd_pool_last_error")
     for name in EXPORTS:
-        if name not in ("pd_status_string", "pd_last_error", "pd_makespan_coloc", "pd_makespan_disagg"):
+        if name not in own_restype:
             getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -224,6 +239,67 @@ def pd_decode_step_host(ctx, q_host, k_new_host, v_new_host, k_pages, v_pages, p
     _check(_lib.pd_decode_step_host(ctx, _ptr(q_host), _ptr(k_new_host), _ptr(v_new_host), _ptr(k_pages),
                                     _ptr(v_pages), _ptr(page_table), _ptr(ctx_lens), _ptr(out_host), batch,
                                     sm_scale, split_pages, _stream(stream)), "pd_decode_step_host", ctx)
+
+
+def pd_pool_create(device: int, capacity_bytes: int, chunk_bytes: int = 0):
+    """Elastic KV pool: a fixed device address range backed chunk by chunk; returns the opaque handle."""
+    h = ctypes.c_void_p()
+    _check(_lib.pd_pool_create(device, capacity_bytes, chunk_bytes, ctypes.byref(h)), "pd_pool_create")
+    return h
+
+
+def _check_pool(rc, where, pool):
+    if rc != PD_OK:
+        raise PdError(rc, where, (_lib.pd_pool_last_error(pool) or b"").decode())
+
+
+def pd_pool_resize(pool, resident_bytes: int, stream_to_drain=None):
+    s = None if stream_to_drain is None else _stream(stream_to_drain)
+    _check_pool(_lib.pd_pool_resize(pool, resident_bytes, s), "pd_pool_resize", pool)
+
+
+def pd_pool_base(pool) -> int:
+    return _lib.pd_pool_base(pool) or 0
+
+
+def pd_pool_capacity(pool) -> int:
+    return _lib.pd_pool_capacity(pool)
+
+
+def pd_pool_chunk_bytes(pool) -> int:
+    return _lib.pd_pool_chunk_bytes(pool)
+
+
+def pd_pool_resident_bytes(pool) -> int:
+    return _lib.pd_pool_resident_bytes(pool)
+
+
+def pd_pool_last_error(pool) -> str:
+    return (_lib.pd_pool_last_error(pool) or b"").decode()
+
+
+def pd_pool_destroy(pool):
+    _check(_lib.pd_pool_destroy(pool), "pd_pool_destroy")
+
+
+class _DeviceRange:
+    """Exposes raw device bytes through the CUDA array interface so torch can alias them."""
+
+    def __init__(self, ptr: int, nbytes: int):
+        self.__cuda_array_interface__ = {"shape": (nbytes,), "typestr": "|u1", "data": (ptr, False), "version": 2}
+
+
+def pool_tensor(pool, offset_bytes: int, shape, dtype, device: int = 0):
+    """A torch tensor aliasing ``shape`` elements of ``dtype`` at ``offset_bytes`` of the pool's range
+    (no copy, no ownership). Only the resident prefix may be touched."""
+    n = 1
+    for s in shape:
+        n *= int(s)
+    nbytes = n * torch.empty((), dtype=dtype).element_size()
+    if offset_bytes < 0 or offset_bytes + nbytes > pd_pool_resident_bytes(pool):
+        raise ValueError("the requested range is not resident")
+    raw = torch.as_tensor(_DeviceRange(pd_pool_base(pool) + offset_bytes, nbytes), device=f"cuda:{device}")
+    return raw.view(dtype).view(*shape)
 
 
 def pd_device_status(ctx, stream=None):

@@ -56,6 +56,21 @@ def test_create_rejects_bad_geometry_before_touching_the_device():
         assert e.value.code == pd.PD_ERR_CUDA
 
 
+def test_pool_calls_reject_bad_arguments_without_a_device():
+    import paper_2609_35158_b200 as pd
+
+    for args in ((0, 0, 0), (-1, 1 << 20, 0)):
+        with pytest.raises(pd.PdError) as e:
+            pd.pd_pool_create(*args)
+        assert e.value.code == pd.PD_ERR_INVALID_ARG
+    assert pd.pd_pool_base(None) == 0 and pd.pd_pool_capacity(None) == 0 and pd.pd_pool_resident_bytes(None) == 0
+    pd.pd_pool_destroy(None)
+    if not torch.cuda.is_available():
+        with pytest.raises(pd.PdError) as e:
+            pd.pd_pool_create(0, 1 << 20)
+        assert e.value.code == pd.PD_ERR_CUDA
+
+
 def test_product_path_does_not_import_the_oracle():
     for rel in ("paper_2609_35158_b200/__init__.py", "paper_2609_35158_b200/build.py"):
         src = open(os.path.join(ROOT, rel)).read()
