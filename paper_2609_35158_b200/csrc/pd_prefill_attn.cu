@@ -96,12 +96,15 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     // O += P_j V_j has completed and V tile j % 2 and logit buffer j % 2 are free again (commit after the O MMA)
     const uint32_t bar_s = smem_u32(bars + 2 * kStages);
     const uint32_t bar_pv = smem_u32(bars + 2 * kStages + 2);
-    const uint32_t bar_p_full = smem_u32(bars + 2 * kStages + 4);  // all 128 rows wrote P_j
+    // [2]: every softmax warp wrote its rows of P_j (barrier j % 2). One barrier per parity: a softmax warp may
+    // run a whole block ahead of another, and its arrival for block j + 1 must not count towards block j.
+    const uint32_t bar_p_full = smem_u32(bars + 2 * kStages + 4);
 
     // ---- set-up: barriers, tensor memory, the Q tile
     if (tid == 0) {
         for (int i = 0; i < 2 * kStages + 4; ++i) mbar_init(smem_u32(bars + i), 1);
-        mbar_init(bar_p_full, kRows);
+        mbar_init(bar_p_full, kRows / 32);  // one arrival per softmax warp
+        mbar_init(bar_p_full + 8, kRows / 32);
         mbar_init_fence();
         prefetch_tensormap(&tm_k);
         prefetch_tensormap(&tm_v);
@@ -160,7 +163,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         if ((tid & 31) == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(kRows, kD, true);
             for (int j = 0; j < nb && ok; ++j) {
-                ok = mbar_wait(bar_p_full, j & 1) && mbar_wait(bar_v + (j % kStages) * 8, (j / kStages) & 1);
+                ok = mbar_wait(bar_p_full + (j & 1) * 8, (j >> 1) & 1) && mbar_wait(bar_v + (j % kStages) * 8, (j / kStages) & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t vst = v_ring + (j % kStages) * kTileBytes;
@@ -333,7 +336,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 fence_proxy_async();
             }
             tc_fence_before_sync();
-            mbar_arrive(bar_p_full);
+            __syncwarp();
+            if ((tid & 31) == 0) mbar_arrive(bar_p_full + (j & 1) * 8);
             lap(4);
         }
         if (tracing && tid == 0) {
@@ -423,7 +427,7 @@ __global__ void advance_lens_kernel(const AppendTokensParams p) {
 
 size_t prefill_smem_bytes(int head_dim) {
     const int halves = head_dim / 64;
-    return static_cast<size_t>(halves) * (kQHalfBytes + 2 * kStages * kHalfBytes) + 1024 + (2 * kStages + 5) * 8 + 64;
+    return static_cast<size_t>(halves) * (kQHalfBytes + 2 * kStages * kHalfBytes) + 1024 + (2 * kStages + 6) * 8 + 64;
 }
 
 cudaError_t prepare_prefill_attn(int head_dim) {
