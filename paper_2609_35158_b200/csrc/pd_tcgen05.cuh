@@ -45,7 +45,8 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr, uint32_t 
 
 // ---- instruction descriptor for kind::f16 with bf16 inputs and fp32 accumulation
 // Bits: [4,6) D format (1 = fp32); [7,10) A format (1 = bf16); [10,13) B format; 15 A major (0 = K);
-// 16 B major (1 = MN); [17,23) N >> 3; [24,29) M >> 4.
+// 16 B major (1 = MN); [17,23) N >> 3; [24,29) M >> 4. A and B must have the same format: an fp16 A
+// with a bf16 B is rejected by the hardware as an illegal instruction.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n, bool b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(b_mn_major) << 16) |
            (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
