@@ -18,17 +18,18 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "pd_oracle.c")
+_SRC_FP8 = os.path.join(_HERE, "pd_oracle_fp8.c")
 _LIB = os.path.join(_HERE, "libpd_oracle.so")
 _lib = None
 
 
 def build(force: bool = False) -> str:
-    """Compile ``pd_oracle.c`` into ``libpd_oracle.so`` (gcc, no fast-math)."""
-    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    """Compile ``pd_oracle.c`` and ``pd_oracle_fp8.c`` into ``libpd_oracle.so`` (gcc, no fast-math)."""
+    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_FP8))
     if force or stale:
         tmp = f"{_LIB}.{os.getpid()}.tmp"
         subprocess.run(
-            ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-pthread", _SRC, "-o", tmp, "-lm"],
+            ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-pthread", _SRC, _SRC_FP8, "-o", tmp, "-lm"],
             check=True,
         )
         os.replace(tmp, _LIB)
@@ -55,6 +56,16 @@ def _load():
         lib.pd_oracle_kv_gather.restype = i
         lib.pd_oracle_kv_scatter.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, ctypes.c_int64]
         lib.pd_oracle_kv_scatter.restype = i
+        lib.pd_oracle_e4m3_to_f64.argtypes = [ctypes.c_uint8]
+        lib.pd_oracle_e4m3_to_f64.restype = ctypes.c_double
+        lib.pd_oracle_f32_to_e4m3.argtypes = [ctypes.c_float]
+        lib.pd_oracle_f32_to_e4m3.restype = ctypes.c_uint8
+        lib.pd_oracle_fp8_quantize_pages.argtypes = [p, p, p, ctypes.c_int64, i, i, i, p, p, p]
+        lib.pd_oracle_fp8_quantize_pages.restype = i
+        lib.pd_oracle_fp8_kv_append.argtypes = [p, p, p, p, p, p, p, i, i, i, i, i, ctypes.c_int64, i]
+        lib.pd_oracle_fp8_kv_append.restype = i
+        lib.pd_oracle_fp8_decode_attn.argtypes = [p, p, p, p, p, p, i, i, i, i, i, i, ctypes.c_float, i, p, p]
+        lib.pd_oracle_fp8_decode_attn.restype = i
         _lib = lib
     return _lib
 
@@ -238,3 +249,84 @@ def kv_append_tokens(k_new, v_new, q_indptr, k_pages, v_pages, page_table, ctx_l
     return lib.pd_oracle_kv_append_tokens(k_new.ctypes.data, v_new.ctypes.data, ip.ctypes.data, k_pages.ctypes.data,
                                           v_pages.ctypes.data, page_table.ctypes.data, ctx_lens.ctypes.data,
                                           len(ip) - 1, Hkv, d, P, page_table.shape[1], NP)
+
+
+# ---------------------------------------------------------------- FP8 (e4m3) pages, see pd_oracle_fp8.c
+
+def e4m3_to_f64(codes) -> np.ndarray:
+    """Exact values of OCP FP8 E4M3 codes (uint8 array)."""
+    lib = _load()
+    codes = np.asarray(codes, dtype=np.uint8)
+    table = np.array([lib.pd_oracle_e4m3_to_f64(c) for c in range(256)], dtype=np.float64)
+    return table[codes]
+
+
+def f32_to_e4m3(x) -> np.ndarray:
+    """fp32 -> e4m3 codes, round to nearest even, saturating at +-448 (element by element through the C routine)."""
+    lib = _load()
+    x = np.asarray(x, dtype=np.float32)
+    flat = np.array([lib.pd_oracle_f32_to_e4m3(ctypes.c_float(v)) for v in x.ravel()], dtype=np.uint8)
+    return flat.reshape(x.shape)
+
+
+def fp8_quantize_pages(k_pages, v_pages, tokens_in_page):
+    """bf16 pools (uint16 bits) -> (k8, v8 uint8 pools, scales fp32 [NP, Hkv, 4]) with one amax scale per tile."""
+    lib = _load()
+    k_pages = _c(k_pages, np.uint16)
+    v_pages = _c(v_pages, np.uint16)
+    NP, Hkv, P, d = k_pages.shape
+    tip = _c(tokens_in_page, np.int32)
+    assert tip.shape == (NP,)
+    k8 = np.empty(k_pages.shape, dtype=np.uint8)
+    v8 = np.empty(k_pages.shape, dtype=np.uint8)
+    scales = np.empty((NP, Hkv, 4), dtype=np.float32)
+    rc = lib.pd_oracle_fp8_quantize_pages(k_pages.ctypes.data, v_pages.ctypes.data, tip.ctypes.data, NP, Hkv, P, d,
+                                          k8.ctypes.data, v8.ctypes.data, scales.ctypes.data)
+    if rc != 0:
+        raise RuntimeError(f"pd_oracle_fp8_quantize_pages failed ({rc})")
+    return k8, v8, scales
+
+
+def fp8_kv_append(k_new, v_new, k8, v8, scales, page_table, ctx_lens, *, advance: bool = True) -> int:
+    """One-token append into FP8 pools, in place (k8, v8, scales, ctx_lens are modified)."""
+    lib = _load()
+    k_new = _c(k_new, np.uint16)
+    v_new = _c(v_new, np.uint16)
+    for a, dt in ((k8, np.uint8), (v8, np.uint8), (scales, np.float32), (ctx_lens, np.int32)):
+        assert a.dtype == dt and a.flags.c_contiguous
+    page_table = _c(page_table, np.int32)
+    B, Hkv, d = k_new.shape
+    NP, Hkv2, P, d2 = k8.shape
+    assert (Hkv2, d2) == (Hkv, d)
+    return lib.pd_oracle_fp8_kv_append(k_new.ctypes.data, v_new.ctypes.data, k8.ctypes.data, v8.ctypes.data,
+                                       scales.ctypes.data, page_table.ctypes.data, ctx_lens.ctypes.data, B, Hkv, d, P,
+                                       page_table.shape[1], NP, int(advance))
+
+
+def fp8_decode_attn(q, k8, v8, scales, page_table, ctx_lens, sm_scale, *, nthreads: int | None = None):
+    """Attention over FP8 pages with per-(page, KV head) scales. Returns (out fp64 [B, Hq, d], lse fp64 [B, Hq])."""
+    lib = _load()
+    q = _c(q, np.uint16)
+    k8 = _c(k8, np.uint8)
+    v8 = _c(v8, np.uint8)
+    scales = _c(scales, np.float32)
+    page_table = _c(page_table, np.int32)
+    ctx_lens = _c(ctx_lens, np.int32)
+    B, Hq, d = q.shape
+    NP, Hkv, P, d2 = k8.shape
+    assert d2 == d and v8.shape == k8.shape and scales.shape == (NP, Hkv, 4)
+    MP = page_table.shape[1]
+    for b in range(B):
+        n = (int(ctx_lens[b]) + P - 1) // P
+        if n:
+            used = page_table[b, :n]
+            assert used.min() >= 0 and used.max() < NP, "page id out of range"
+    out = np.empty((B, Hq, d), dtype=np.float64)
+    lse = np.empty((B, Hq), dtype=np.float64)
+    rc = lib.pd_oracle_fp8_decode_attn(q.ctypes.data, k8.ctypes.data, v8.ctypes.data, scales.ctypes.data,
+                                       page_table.ctypes.data, ctx_lens.ctypes.data, B, Hq, Hkv, d, P, MP,
+                                       ctypes.c_float(np.float32(sm_scale)), int(nthreads or os.cpu_count() or 1),
+                                       out.ctypes.data, lse.ctypes.data)
+    if rc != 0:
+        raise RuntimeError(f"pd_oracle_fp8_decode_attn failed ({rc})")
+    return out, lse
