@@ -355,6 +355,42 @@ int32_t pd_toggle_gate(double R, double B, double T_ded, double T_full, double T
 /* Least-squares line step_seconds = A + b * concurrency over n >= 2 measurements. */
 int pd_fit_decode_cost(const double *concurrency, const double *step_seconds, int32_t n, double *A, double *b);
 
+/* ---- FP8 KV pages. The paper has no counterpart (its decode cost b is the KV-cache HBM read per
+ * concurrent sequence, Eq. 1; one byte per cached value halves it); the format is this library's:
+ *   k8, v8     [num_pages][num_kv_heads][16][head_dim] bytes, OCP FP8 E4M3 (bias 7, no infinities,
+ *              0x7f / 0xff = NaN, largest finite value 448), device, 16-byte aligned
+ *   kv_scales  [num_pages][num_kv_heads][4] fp32 = {k_scale, v_scale, 0, 0}, device, 16-byte aligned
+ * and K_t = k_scale * e4m3(byte), V_t = v_scale * e4m3(byte). head_dim must be 128 for attention.
+ */
+
+/*
+ * Quantises every (page, KV head) tile of the bf16 pools: amax over the first tokens_in_page[page]
+ * slots (device int32 [num_pages], 0..16; NaN ignored), scale = amax / 448 in fp32 (1 if amax = 0),
+ * code = e4m3(x / scale) with IEEE fp32 division, round to nearest even, saturating; slots past
+ * tokens_in_page are written as 0. Covers all cfg.num_pages pages.
+ */
+int pd_kv_quantize_pages(pd_ctx *ctx, const void *k_pages, const void *v_pages, const int32_t *tokens_in_page,
+                         void *k8, void *v8, float *kv_scales, void *stream);
+
+/*
+ * One-token append into FP8 pools; positions, skipping and error reporting as pd_kv_append. A token
+ * that opens a page (slot 0) sets that page's k_scale and v_scale from its own rows,
+ * scale = (amax * 2) / 448 (1 if amax = 0): a factor two of headroom for the 15 tokens that follow.
+ * Any other token is quantised with the page's stored scales and saturates at +-448.
+ */
+int pd_kv_append_fp8(pd_ctx *ctx, const void *k_new, const void *v_new, void *k8, void *v8, float *kv_scales,
+                     const int32_t *page_table, int32_t *ctx_lens, int32_t batch, uint32_t call_flags,
+                     void *stream);
+
+/*
+ * pd_decode_attn over FP8 pools: same outputs, plan, split_pages meaning, error behaviour and
+ * bit-reproducibility. q is bf16 with |q| below the fp16 range (65504): the products run in fp16 with
+ * fp32 accumulation, scales are applied in fp32.
+ */
+int pd_decode_attn_fp8(pd_ctx *ctx, const void *q, const void *k8, const void *v8, const float *kv_scales,
+                       const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse,
+                       int32_t batch, float sm_scale, int32_t split_pages, void *stream);
+
 /* ---- Elastic KV pool on CUDA virtual memory management (Sec. 4.6: the intra-scale toggle keeps the
  * rollout process and swaps device state; Sec. 5: the KV cache is released when training begins and
  * restored when the GPU is available again). A pool is a device address range of `capacity` bytes whose

@@ -61,8 +61,13 @@ struct pd_ctx {
     const void *map_k_ptr = nullptr, *map_v_ptr = nullptr;
     alignas(64) CUtensorMap tm_k{};
     alignas(64) CUtensorMap tm_v{};
+    // the same for FP8 pools
+    const void *map_k8_ptr = nullptr, *map_v8_ptr = nullptr;
+    alignas(64) CUtensorMap tm_k8{};
+    alignas(64) CUtensorMap tm_v8{};
     cudaEvent_t ev_before = nullptr, ev_after = nullptr;  // optional timing hook around the split kernel
     bool prefill_ready = false;
+    bool fp8_ready = false;
     int64_t launches = 0;
     char last_error[256] = {0};
 };
@@ -94,6 +99,24 @@ int encode_pool_map(pd_ctx *ctx, const void *pool, CUtensorMap *out) {
     const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(c.page_size)};
     const cuuint32_t elem_strides[2] = {1, 1};
     const CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box,
+                                   elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        std::snprintf(ctx->last_error, sizeof ctx->last_error, "cuTensorMapEncodeTiled failed (%d)", static_cast<int>(r));
+        return PD_ERR_CUDA;
+    }
+    return PD_OK;
+}
+
+// The same view of an FP8 pool: columns = head_dim bytes, one box = 16 rows x 128 B.
+int encode_pool_map_fp8(pd_ctx *ctx, const void *pool, CUtensorMap *out) {
+    const pd_config &c = ctx->cfg;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c.head_dim),
+                                static_cast<cuuint64_t>(c.num_pages) * c.num_kv_heads * c.page_size};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c.head_dim)};
+    const cuuint32_t box[2] = {128, static_cast<cuuint32_t>(c.page_size)};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    const CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(pool), dims, strides, box,
                                    elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -420,6 +443,132 @@ int pd_decode_step(pd_ctx *ctx, const void *q, const void *k_new, const void *v_
     if (k_new == nullptr || v_new == nullptr) return fail(ctx, PD_ERR_INVALID_ARG, "pd_decode_step: null k_new / v_new");
     return decode_attn_impl(ctx, "pd_decode_step", q, k_new, v_new, k_pages, v_pages, page_table, ctx_lens, out, lse, batch,
                             sm_scale, split_pages, stream);
+}
+
+int pd_kv_quantize_pages(pd_ctx *ctx, const void *k_pages, const void *v_pages, const int32_t *tokens_in_page, void *k8,
+                         void *v8, float *kv_scales, void *stream) {
+    if (ctx == nullptr) return PD_ERR_INVALID_ARG;
+    if (!aligned16(k_pages) || !aligned16(v_pages) || !aligned16(k8) || !aligned16(v8) || !aligned16(kv_scales) ||
+        tokens_in_page == nullptr)
+        return fail(ctx, PD_ERR_INVALID_ARG, "pd_kv_quantize_pages: null or misaligned pointer");
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
+    pd::QuantizeParams p{};
+    p.k_pages = static_cast<const __nv_bfloat16 *>(k_pages);
+    p.v_pages = static_cast<const __nv_bfloat16 *>(v_pages);
+    p.tokens_in_page = tokens_in_page;
+    p.k8 = static_cast<uint8_t *>(k8);
+    p.v8 = static_cast<uint8_t *>(v8);
+    p.scales = kv_scales;
+    p.num_pages = ctx->cfg.num_pages;
+    p.Hkv = ctx->cfg.num_kv_heads;
+    p.D = ctx->cfg.head_dim;
+    p.pdl = ctx->pdl;
+    const cudaError_t err = pd::launch_kv_quantize_pages(p, static_cast<cudaStream_t>(stream));
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "kv_quantize_pages launch", err);
+    ctx->launches += 1;
+    return PD_OK;
+}
+
+int pd_kv_append_fp8(pd_ctx *ctx, const void *k_new, const void *v_new, void *k8, void *v8, float *kv_scales,
+                     const int32_t *page_table, int32_t *ctx_lens, int32_t batch, uint32_t call_flags, void *stream) {
+    if (int rc = check_batch(ctx, batch)) return rc;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k8) || !aligned16(v8) || !aligned16(kv_scales) ||
+        page_table == nullptr || ctx_lens == nullptr)
+        return fail(ctx, PD_ERR_INVALID_ARG, "pd_kv_append_fp8: null or misaligned pointer");
+    if (batch == 0) return PD_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
+    pd::AppendFp8Params p{};
+    p.k_new = static_cast<const __nv_bfloat16 *>(k_new);
+    p.v_new = static_cast<const __nv_bfloat16 *>(v_new);
+    p.k8 = static_cast<uint8_t *>(k8);
+    p.v8 = static_cast<uint8_t *>(v8);
+    p.scales = kv_scales;
+    p.page_table = page_table;
+    p.ctx_lens = ctx_lens;
+    p.status = ctx->status;
+    p.B = batch;
+    p.Hkv = ctx->cfg.num_kv_heads;
+    p.D = ctx->cfg.head_dim;
+    p.MP = ctx->cfg.max_pages_per_seq;
+    p.num_pages = static_cast<int32_t>(ctx->cfg.num_pages);
+    p.advance = (call_flags & PD_APPEND_NO_ADVANCE) ? 0 : 1;
+    p.pdl = ctx->pdl;
+    const cudaError_t err = pd::launch_kv_append_fp8(p, static_cast<cudaStream_t>(stream));
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "kv_append_fp8 launch", err);
+    ctx->launches += 1;
+    return PD_OK;
+}
+
+int pd_decode_attn_fp8(pd_ctx *ctx, const void *q, const void *k8, const void *v8, const float *kv_scales,
+                       const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse, int32_t batch,
+                       float sm_scale, int32_t split_pages, void *stream) {
+    if (int rc = check_batch(ctx, batch)) return rc;
+    if (ctx->cfg.head_dim != 128) return fail(ctx, PD_ERR_UNSUPPORTED, "pd_decode_attn_fp8: head_dim must be 128");
+    if (!aligned16(q) || !aligned16(k8) || !aligned16(v8) || !aligned16(kv_scales) || !aligned16(out) ||
+        page_table == nullptr || ctx_lens == nullptr)
+        return fail(ctx, PD_ERR_INVALID_ARG, "pd_decode_attn_fp8: null or misaligned pointer");
+    if (!(sm_scale > 0.f) || !(sm_scale < 3.0e38f)) return fail(ctx, PD_ERR_INVALID_ARG, "sm_scale must be finite and positive");
+    if (split_pages < 0) return fail(ctx, PD_ERR_INVALID_ARG, "split_pages must be >= 0");
+    if (batch == 0) return PD_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
+    if (ctx->variant.warps != pd::decode_attn_fp8_warps())
+        return fail(ctx, PD_ERR_UNSUPPORTED, "pd_decode_attn_fp8: the workspace was sized for another worker count");
+    if (!ctx->fp8_ready) {
+        const cudaError_t e = pd::prepare_decode_attn_fp8();
+        if (e != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "fp8 decode kernel attribute", e);
+        ctx->fp8_ready = true;
+    }
+    if (ctx->map_k8_ptr != k8) {
+        if (int rc = encode_pool_map_fp8(ctx, k8, &ctx->tm_k8)) return rc;
+        ctx->map_k8_ptr = k8;
+    }
+    if (ctx->map_v8_ptr != v8) {
+        if (int rc = encode_pool_map_fp8(ctx, v8, &ctx->tm_v8)) return rc;
+        ctx->map_v8_ptr = v8;
+    }
+    pd::AttnParams p{};
+    p.q = static_cast<const __nv_bfloat16 *>(q);
+    p.kv_scales = kv_scales;
+    p.page_table = page_table;
+    p.ctx_lens = ctx_lens;
+    p.out = static_cast<__nv_bfloat16 *>(out);
+    p.lse = lse;
+    p.part_o = ctx->part_o;
+    p.part_ml = ctx->part_ml;
+    p.cum_pages = ctx->cum_pages;
+    p.plan = ctx->plan;
+    p.status = ctx->status;
+    p.B = batch;
+    p.Hq = ctx->cfg.num_q_heads;
+    p.Hkv = ctx->cfg.num_kv_heads;
+    p.G = ctx->group;
+    p.MP = ctx->cfg.max_pages_per_seq;
+    p.num_pages = static_cast<int32_t>(ctx->cfg.num_pages);
+    p.scale_log2 = sm_scale * 1.4426950408889634f;
+    p.split_pages = split_pages;
+    p.max_ranges = ctx->max_ranges;
+    p.min_pages_auto = ctx->min_pages_auto;
+    p.halving_levels = ctx->halving_levels;
+    p.tail_pages = ctx->tail_pages;
+    const bool hooked = ctx->ev_before != nullptr;
+    p.pdl = hooked ? 0 : ctx->pdl;
+    p.merge_rows = ctx->merge_rows;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (hooked) cudaEventRecord(ctx->ev_before, s);
+    cudaError_t err = pd::launch_decode_attn_fp8(ctx->tm_k8, ctx->tm_v8, p, ctx->num_ctas, s);
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "decode_attn_split_fp8 launch", err);
+    if (hooked) {
+        cudaEventRecord(ctx->ev_after, s);
+        ctx->ev_before = nullptr;
+        ctx->ev_after = nullptr;
+    }
+    err = pd::launch_lse_merge(ctx->cfg.head_dim, p, s);
+    if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "lse_merge launch", err);
+    ctx->launches += 2;
+    return PD_OK;
 }
 
 int pd_kv_append_tokens(pd_ctx *ctx, const void *k_new, const void *v_new, const int32_t *q_indptr, void *k_pages,

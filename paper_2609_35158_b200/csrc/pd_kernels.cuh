@@ -53,6 +53,8 @@ struct AttnParams {
     __nv_bfloat16 *k_pool_w, *v_pool_w;  // the pools, writable
     int32_t *ctx_lens_w;
     int32_t fused;
+    // FP8 pages (null for bf16 pools): {k_scale, v_scale, 0, 0} fp32 per (page, KV head)
+    const float *kv_scales;
     int32_t merge_rows;         // rows per CTA of the merge kernel, 0 = chosen from the row count
     unsigned long long *trace;  // optional [workers][4] ns timestamps: kernel entry, first data, last data, exit
 };
@@ -110,6 +112,27 @@ struct AppendTokensParams {
 };
 
 // Shape of one compiled variant of the split kernel.
+// Whole-page FP8 quantisation: bf16 pools -> e4m3 pools + scale records.
+struct QuantizeParams {
+    const __nv_bfloat16 *k_pages, *v_pages;  // [num_pages][Hkv][16][D]
+    const int32_t *tokens_in_page;           // [num_pages] leading slots that hold tokens
+    uint8_t *k8, *v8;                        // [num_pages][Hkv][16][D]
+    float *scales;                           // [num_pages][Hkv][4]
+    int64_t num_pages;
+    int32_t Hkv, D, pdl;
+};
+
+// One-token append into FP8 pools.
+struct AppendFp8Params {
+    const __nv_bfloat16 *k_new, *v_new;  // [B][Hkv][D]
+    uint8_t *k8, *v8;
+    float *scales;
+    const int32_t *page_table;
+    int32_t *ctx_lens;
+    int32_t *status;
+    int32_t B, Hkv, D, MP, num_pages, advance, pdl;
+};
+
 struct AttnVariant {
     int head_dim, warps, stages, hilo;
 };
@@ -139,6 +162,14 @@ cudaError_t prepare_decode_attn(const AttnVariant &v, size_t *smem_bytes);  // o
 cudaError_t launch_decode_attn(const AttnVariant &v, const CUtensorMap &tm_k, const CUtensorMap &tm_v,
                                const AttnParams &p, int num_ctas, size_t smem_bytes, cudaStream_t stream);
 cudaError_t launch_lse_merge(int head_dim, const AttnParams &p, cudaStream_t stream);
+// FP8 pages (head_dim 128): the split kernel writes the same partials and plan, so launch_lse_merge follows it
+cudaError_t prepare_decode_attn_fp8();
+size_t decode_attn_fp8_smem_bytes();
+int decode_attn_fp8_warps();
+cudaError_t launch_decode_attn_fp8(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, int num_ctas,
+                                   cudaStream_t stream);
+cudaError_t launch_kv_quantize_pages(const QuantizeParams &p, cudaStream_t stream);
+cudaError_t launch_kv_append_fp8(const AppendFp8Params &p, cudaStream_t stream);
 cudaError_t prepare_prefill_attn(int head_dim);  // opt-in shared memory, once
 cudaError_t launch_prefill_attn(int head_dim, const CUtensorMap &tm_k, const CUtensorMap &tm_v, const PrefillParams &p,
                                 int max_q_len, cudaStream_t stream);

@@ -16,7 +16,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def header_functions():
     text = open(os.path.join(ROOT, "include", "pd.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(pd_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(pd_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_library_builds_and_exports_every_declared_symbol():

@@ -1,0 +1,234 @@
+"""GPU parity of the FP8 (e4m3) KV path through the C ABI: whole-page quantiser and one-token append are
+bit-exact against the oracle; attention over FP8 pages is within the decode tolerances (max abs 1e-2 scaled
+by magnitude, per-row relative L2 5e-3) of the fp64 oracle evaluated on the SAME quantised cache."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wl
+from pd_testlib import Ctx, assert_parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+P = wl.PAGE_SIZE
+
+
+def tokens_in_page(cache, lens):
+    tip = np.zeros(cache.k_pages.shape[0], dtype=np.int32)
+    for b, L in enumerate(lens):
+        for i in range((int(L) + P - 1) // P):
+            tip[cache.page_table_host[b, i]] = min(P, int(L) - i * P)
+    return tip
+
+
+def quantized_on_host(cache, lens, poison_codes=True):
+    """The oracle's quantisation of a bf16 cache; unused slots and pages get NaN codes and NaN scales."""
+    tip = tokens_in_page(cache, lens)
+    k8, v8, sc = oracle.fp8_quantize_pages(oracle.bf16_bits(cache.k_pages), oracle.bf16_bits(cache.v_pages), tip)
+    if poison_codes:
+        for page, n in enumerate(tip):
+            k8[page, :, n:] = 0x7F
+            v8[page, :, n:] = 0xFF
+            if n == 0:
+                sc[page, :, :2] = np.nan
+    return k8, v8, sc, tip
+
+
+def to_dev(*arrays):
+    return [torch.from_numpy(np.ascontiguousarray(a)).to(DEV) for a in arrays]
+
+
+@pytest.mark.parametrize("Hkv,d", [(8, 128), (2, 64)])
+def test_quantize_pages_bit_exact(Hkv, d):
+    import paper_2609_35158_b200 as pd
+
+    lens = np.array([0, 1, 15, 16, 17, 100, 333], dtype=np.int32)
+    cache = wl.build_paged_cache(lens, Hkv, d, seed=80, device=DEV, poison=True)  # NaN in every slot without a token
+    cache.k_pages[cache.page_table_host[5, 0], 0, :, :] = 0  # an all-zero tile: scale 1
+    cache.v_pages.mul_(0.03)
+    tip = tokens_in_page(cache, lens)
+    want_k, want_v, want_sc = oracle.fp8_quantize_pages(oracle.bf16_bits(cache.k_pages), oracle.bf16_bits(cache.v_pages), tip)
+    NP = cache.k_pages.shape[0]
+    k8 = torch.full((NP, Hkv, P, d), 0x55, dtype=torch.uint8, device=DEV)
+    v8 = torch.full_like(k8, 0x55)
+    sc = torch.full((NP, Hkv, 4), -1.0, dtype=torch.float32, device=DEV)
+    with Ctx(Hkv, Hkv, d, len(lens), cache.page_table.shape[1], NP) as ctx:
+        pd.pd_kv_quantize_pages(ctx.h, cache.k_pages, cache.v_pages, torch.from_numpy(tip).to(DEV), k8, v8, sc)
+        torch.cuda.synchronize()
+    assert np.array_equal(sc.cpu().numpy().view(np.uint32), want_sc.view(np.uint32))
+    assert np.array_equal(k8.cpu().numpy(), want_k)
+    assert np.array_equal(v8.cpu().numpy(), want_v)
+    assert want_sc[cache.page_table_host[5, 0], 0, 0] == 1.0
+
+
+GEOMS = [(32, 8), (32, 4), (8, 8), (4, 2), (16, 2)]
+
+
+@pytest.mark.parametrize("Hq,Hkv", GEOMS)
+@pytest.mark.parametrize("split_pages", [0, 1, 3, 100000])
+def test_fp8_attention_small_ragged_poisoned(Hq, Hkv, split_pages):
+    import paper_2609_35158_b200 as pd
+
+    d = 128
+    lens = np.array([1, 15, 16, 17, 31, 33, 64, 300, 1000, 0, 2500], dtype=np.int32)
+    cache = wl.build_paged_cache(lens, Hkv, d, seed=81, device=DEV, poison=True)
+    cache.v_pages.mul_(0.02)  # small values: a v_scale folded into fp16 probabilities would flush them
+    k8, v8, sc, _ = quantized_on_host(cache, lens)
+    q = wl.random_bf16((len(lens), Hq, d), 82, DEV)
+    scale = d ** -0.5
+    ref, ref_lse = oracle.fp8_decode_attn(oracle.bf16_bits(q), k8, v8, sc, cache.page_table_host, lens, scale)
+    k8d, v8d, scd = to_dev(k8, v8, sc)
+    out = torch.full((len(lens), Hq, d), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((len(lens), Hq), float("nan"), dtype=torch.float32, device=DEV)
+    with Ctx(Hq, Hkv, d, len(lens), cache.page_table.shape[1], cache.k_pages.shape[0]) as ctx:
+        pd.pd_decode_attn_fp8(ctx.h, q, k8d, v8d, scd, cache.page_table, cache.ctx_lens, out, lse, sm_scale=scale,
+                              split_pages=split_pages)
+        torch.cuda.synchronize()
+        assert pd.pd_device_status(ctx.h)[0] == 0
+        again = torch.empty_like(out)
+        pd.pd_decode_attn_fp8(ctx.h, q, k8d, v8d, scd, cache.page_table, cache.ctx_lens, again, sm_scale=scale,
+                              split_pages=split_pages)
+        torch.cuda.synchronize()
+    assert torch.equal(out.view(torch.int16), again.view(torch.int16))  # bit-reproducible
+    # outputs here are ~0.02 in magnitude: compare relative to the output scale
+    live = lens > 0
+    assert_parity((out[torch.from_numpy(live).to(DEV)].float() * 50).to(torch.bfloat16), ref[live] * 50,
+                  f"{Hq}/{Hkv} split {split_pages}", scale_abs_by_magnitude=True)
+    got_lse = lse.cpu().numpy()
+    assert np.all(np.isneginf(got_lse[~live])) and np.all(out[torch.from_numpy(~live).to(DEV)].float().cpu().numpy() == 0)
+    np.testing.assert_allclose(got_lse[live], ref_lse[live], rtol=3e-5, atol=3e-5)
+
+
+def test_fp8_attention_closed_form_and_dominant_key():
+    import paper_2609_35158_b200 as pd
+
+    Hq, Hkv, d, NP = 4, 1, 128, 3
+    # two tokens: q.k = (1, 0) after scaling, V = +1 / -1 everywhere -> every output is tanh(1/2)
+    k8 = np.zeros((NP, Hkv, P, d), dtype=np.uint8)
+    v8 = np.zeros_like(k8)
+    sc = np.zeros((NP, Hkv, 4), dtype=np.float32)
+    k8[1, 0, 0, 0] = 0x38       # 1.0
+    v8[1, 0, 0, :] = 0x40       # 2.0 * v_scale 0.5 = +1
+    v8[1, 0, 1, :] = 0xC0       # -1
+    sc[1, 0, 0], sc[1, 0, 1] = 2.0, 0.5   # K_0 = (2, 0, ...)
+    q = torch.zeros((1, Hq, d), dtype=torch.bfloat16, device=DEV)
+    q[:, :, 0] = 4.0            # scale 0.125: logits (1, 0)
+    table = torch.tensor([[1, 2]], dtype=torch.int32, device=DEV)
+    lens = torch.tensor([2], dtype=torch.int32, device=DEV)
+    out = torch.empty_like(q)
+    lse = torch.empty((1, Hq), dtype=torch.float32, device=DEV)
+    k8d, v8d, scd = to_dev(k8, v8, sc)
+    with Ctx(Hq, Hkv, d, 1, 2, NP) as ctx:
+        pd.pd_decode_attn_fp8(ctx.h, q, k8d, v8d, scd, table, lens, out, lse, sm_scale=0.125)
+        torch.cuda.synchronize()
+        assert pd.pd_device_status(ctx.h)[0] == 0
+    assert np.allclose(out.float().cpu().numpy(), np.tanh(0.5), atol=2e-3)
+    assert np.allclose(lse.cpu().numpy(), np.log(1 + np.e), atol=1e-5)
+
+
+def test_fp8_append_bit_exact_then_attend():
+    import paper_2609_35158_b200 as pd
+
+    Hq, Hkv, d = 32, 8, 128
+    lens0 = np.array([0, 5, 15, 16, 31, 32, 100], dtype=np.int32)
+    steps = 20
+    cache = wl.build_paged_cache(lens0, Hkv, d, seed=83, device=DEV, reserve_tokens=steps)
+    k8, v8, sc, _ = quantized_on_host(cache, lens0, poison_codes=False)
+    lens = lens0.copy()
+    k8d, v8d, scd = to_dev(k8, v8, sc)
+    B = len(lens0)
+    with Ctx(Hq, Hkv, d, B, cache.page_table.shape[1], cache.k_pages.shape[0]) as ctx:
+        for t in range(steps):
+            kn = wl.random_bf16((B, Hkv, d), 900 + 2 * t, DEV) * (1.0 + 0.2 * t)  # growing: later tokens meet the stored scale
+            vn = wl.random_bf16((B, Hkv, d), 901 + 2 * t, DEV)
+            n = oracle.fp8_kv_append(oracle.bf16_bits(kn), oracle.bf16_bits(vn), k8, v8, sc, cache.page_table_host, lens)
+            assert n == B
+            pd.pd_kv_append_fp8(ctx.h, kn, vn, k8d, v8d, scd, cache.page_table, cache.ctx_lens)
+        torch.cuda.synchronize()
+        assert pd.pd_device_status(ctx.h)[0] == 0
+        assert np.array_equal(cache.ctx_lens.cpu().numpy(), lens)
+        assert np.array_equal(scd.cpu().numpy().view(np.uint32), sc.view(np.uint32))
+        assert np.array_equal(k8d.cpu().numpy(), k8) and np.array_equal(v8d.cpu().numpy(), v8)
+        assert (np.abs(oracle.e4m3_to_f64(k8)) == 448.0).any()  # the growing keys saturated somewhere
+        q = wl.random_bf16((B, Hq, d), 84, DEV)
+        out = torch.empty((B, Hq, d), dtype=torch.bfloat16, device=DEV)
+        pd.pd_decode_attn_fp8(ctx.h, q, k8d, v8d, scd, cache.page_table, cache.ctx_lens, out, sm_scale=d ** -0.5)
+        torch.cuda.synchronize()
+        assert pd.pd_device_status(ctx.h)[0] == 0
+    ref, _ = oracle.fp8_decode_attn(oracle.bf16_bits(q), k8, v8, sc, cache.page_table_host, lens, d ** -0.5)
+    assert_parity(out, ref, "after 20 FP8 appends", scale_abs_by_magnitude=True)
+
+
+def test_fp8_append_errors_are_reported_and_skipped():
+    import paper_2609_35158_b200 as pd
+
+    lens = np.array([16, 5], dtype=np.int32)
+    cache = wl.build_paged_cache(lens, 2, 128, seed=85, device=DEV, poison=True)  # next page of sequence 0 is -1
+    NP = cache.k_pages.shape[0]
+    k8 = torch.zeros((NP, 2, P, 128), dtype=torch.uint8, device=DEV)
+    v8 = torch.zeros_like(k8)
+    sc = torch.ones((NP, 2, 4), dtype=torch.float32, device=DEV)
+    kn = wl.random_bf16((2, 2, 128), 86, DEV)
+    with Ctx(2, 2, 128, 2, cache.page_table.shape[1], NP) as ctx:
+        pd.pd_kv_append_fp8(ctx.h, kn, kn, k8, v8, sc, cache.page_table, cache.ctx_lens)
+        code, seq, _ = pd.pd_device_status(ctx.h)
+        assert code == pd.PD_ERR_DEVICE_FAULT and seq == 0
+        assert cache.ctx_lens.cpu().tolist() == [16, 6]
+        touched = (k8 != 0).nonzero()
+        assert len(touched) and bool((touched[:, 0] == int(cache.page_table_host[1, 0])).all()) and bool((touched[:, 2] == 5).all())
+
+
+def test_fp8_attention_needs_head_dim_128():
+    import paper_2609_35158_b200 as pd
+
+    with Ctx(8, 2, 64, 1, 1, 4) as ctx:
+        x = torch.zeros(4096, dtype=torch.uint8, device=DEV)
+        q = torch.zeros((1, 8, 64), dtype=torch.bfloat16, device=DEV)
+        i = torch.zeros(4, dtype=torch.int32, device=DEV)
+        with pytest.raises(pd.PdError) as e:
+            pd.pd_decode_attn_fp8(ctx.h, q, x, x, x.view(torch.float32), i, i, q)
+        assert e.value.code == pd.PD_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("config", [1, 3])
+def test_fp8_full_size_config_sampled_sequences(config):
+    import paper_2609_35158_b200 as pd
+
+    w = wl.WORKLOADS[config]
+    lens = wl.context_lengths(config)
+    cache = wl.build_paged_cache(lens, w.num_kv_heads, w.head_dim, seed=config, device=DEV)
+    NP = cache.k_pages.shape[0]
+    B = len(lens)
+    k8d = torch.empty((NP, w.num_kv_heads, P, w.head_dim), dtype=torch.uint8, device=DEV)
+    v8d = torch.empty_like(k8d)
+    scd = torch.empty((NP, w.num_kv_heads, 4), dtype=torch.float32, device=DEV)
+    tip = tokens_in_page(cache, lens)
+    q = wl.random_bf16((B, w.num_q_heads, w.head_dim), 87, DEV)
+    out = torch.empty_like(q)
+    with Ctx(w.num_q_heads, w.num_kv_heads, w.head_dim, B, cache.page_table.shape[1], NP) as ctx:
+        # the GPU quantiser prepares the cache (it is bit-identical to the oracle's, checked on the sample below)
+        pd.pd_kv_quantize_pages(ctx.h, cache.k_pages, cache.v_pages, torch.from_numpy(tip).to(DEV), k8d, v8d, scd)
+        pd.pd_decode_attn_fp8(ctx.h, q, k8d, v8d, scd, cache.page_table, cache.ctx_lens, out, sm_scale=w.sm_scale)
+        torch.cuda.synchronize()
+        assert pd.pd_device_status(ctx.h)[0] == 0
+    sample = sorted({int(np.argmin(lens)), int(np.argmax(lens)), 0, B - 1})
+    # oracle inputs come from the oracle: quantise the sampled sequences' pages on the host
+    pages = np.concatenate([cache.page_table_host[b, :(int(lens[b]) + P - 1) // P] for b in sample])
+    idx = torch.from_numpy(pages.astype(np.int64)).to(DEV)
+    kb = oracle.bf16_bits(cache.k_pages.index_select(0, idx))
+    vb = oracle.bf16_bits(cache.v_pages.index_select(0, idx))
+    k8, v8, sc = oracle.fp8_quantize_pages(kb, vb, tip[pages])
+    assert np.array_equal(k8d.index_select(0, idx).cpu().numpy(), k8)
+    assert np.array_equal(scd.index_select(0, idx).cpu().numpy().view(np.uint32), sc.view(np.uint32))
+    table = np.full((len(sample), cache.page_table.shape[1]), -1, dtype=np.int32)
+    cur = 0
+    for i, b in enumerate(sample):
+        n = (int(lens[b]) + P - 1) // P
+        table[i, :n] = np.arange(cur, cur + n)
+        cur += n
+    qs = oracle.bf16_bits(q[torch.tensor(sample, device=DEV)])
+    ref, _ = oracle.fp8_decode_attn(qs, k8, v8, sc, table, lens[sample], w.sm_scale)
+    # long contexts average unit-variance values to outputs of ~0.02: compare at that scale
+    assert_parity((out[torch.tensor(sample, device=DEV)].float() * 32).to(torch.bfloat16), ref * 32,
+                  f"config {config}", scale_abs_by_magnitude=True)
