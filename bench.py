@@ -652,6 +652,123 @@ def run_fit_b(args):
     }), flush=True)
 
 
+# ------------------------------------------------------------------------------------------ FP8 pages
+
+def run_decode_fp8(args):
+    """The decode step over FP8 (e4m3) KV pages: pd_kv_append_fp8 + pd_decode_attn_fp8, device-resident inputs.
+    Bytes per cached token: one byte per K and V value plus the 16-byte scale record of each (page, KV head)."""
+    import torch
+
+    import oracle
+    import paper_2609_35158_b200 as pd
+    import workloads as wl
+
+    torch.cuda.set_device(0)
+    dev = "cuda:0"
+    cfg_id = args.config
+    w = wl.WORKLOADS[cfg_id]
+    assert w.head_dim == 128, "FP8 attention is built for head_dim 128"
+    K, W = args.steps, args.warmup
+    lens0 = wl.context_lengths(cfg_id)
+    B = w.batch
+    cache = wl.build_paged_cache(lens0, w.num_kv_heads, w.head_dim, seed=cfg_id, device=dev, reserve_tokens=W + K + 2)
+    NP, P = cache.num_pages, w.page_size
+    ctx = pd.pd_create(w.num_q_heads, w.num_kv_heads, w.head_dim, P, B, cache.page_table.shape[1], NP, 0)
+    tip = np.zeros(NP, dtype=np.int32)
+    for b, L in enumerate(lens0):
+        n = (int(L) + P - 1) // P
+        tip[cache.page_table_host[b, :n]] = P
+        if L % P:
+            tip[cache.page_table_host[b, n - 1]] = L % P
+    k8 = torch.empty((NP, w.num_kv_heads, P, w.head_dim), dtype=torch.uint8, device=dev)
+    v8 = torch.empty_like(k8)
+    sc = torch.empty((NP, w.num_kv_heads, 4), dtype=torch.float32, device=dev)
+    pd.pd_kv_quantize_pages(ctx, cache.k_pages, cache.v_pages, torch.from_numpy(tip).to(dev), k8, v8, sc)
+    torch.cuda.synchronize()
+    del cache.k_pages, cache.v_pages
+    R = 4
+    qs = [wl.random_bf16((B, w.num_q_heads, w.head_dim), 10 + i, dev) for i in range(R)]
+    kns = [wl.random_bf16((B, w.num_kv_heads, w.head_dim), 20 + i, dev) for i in range(R)]
+    vns = [wl.random_bf16((B, w.num_kv_heads, w.head_dim), 30 + i, dev) for i in range(R)]
+    out = torch.empty((B, w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=dev)
+    lens = lens0.astype(np.int64).copy()
+    per_token = 2 * w.num_kv_heads * w.head_dim          # one byte per K and per V value
+    per_page = w.num_kv_heads * 16                        # scale records
+
+    def step(i):
+        nonlocal lens
+        pd.pd_kv_append_fp8(ctx, kns[i % R], vns[i % R], k8, v8, sc, cache.page_table, cache.ctx_lens)
+        pd.pd_decode_attn_fp8(ctx, qs[i % R], k8, v8, sc, cache.page_table, cache.ctx_lens, out, sm_scale=w.sm_scale)
+        lens = lens + 1
+        return int(lens.sum()) * per_token + int(((lens + P - 1) // P).sum()) * per_page
+
+    for i in range(W):
+        step(i)
+    torch.cuda.synchronize()
+    assert pd.pd_device_status(ctx)[0] == 0
+    hooked = [i for i in range(K) if i % 16 == min(8, K - 1)]
+    befores = {i: torch.cuda.Event(enable_timing=True) for i in hooked}
+    afters = {i: torch.cuda.Event(enable_timing=True) for i in hooked}
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(0)
+    torch.cuda.synchronize()
+    sampler.start()
+    t0.record()
+    total = hooked_bytes = 0
+    for i in range(K):
+        if i in befores:
+            pd.pd_set_profile_events(ctx, befores[i], afters[i])
+        nb = step(W + i)
+        total += nb
+        if i in befores:
+            hooked_bytes += nb
+    t1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    assert pd.pd_device_status(ctx)[0] == 0
+    ms = t0.elapsed_time(t1)
+    split_ms = float(np.mean([befores[i].elapsed_time(afters[i]) for i in hooked]))
+    per_launch = hooked_bytes / len(hooked)
+    peak, peak_kind = measured_hbm_peak()
+    achieved = per_launch / (split_ms * 1e-3) / 1e9
+
+    # parity on the spot: the oracle on one short and one long sequence of the final cache
+    sample = [int(np.argmin(lens)), int(np.argmax(lens))]
+    pages = np.concatenate([cache.page_table_host[b, :(int(lens[b]) + P - 1) // P] for b in sample])
+    idx = torch.from_numpy(pages.astype(np.int64)).to(dev)
+    table = np.full((2, cache.page_table.shape[1]), -1, dtype=np.int32)
+    cur = 0
+    for i, b in enumerate(sample):
+        n = (int(lens[b]) + P - 1) // P
+        table[i, :n] = np.arange(cur, cur + n)
+        cur += n
+    tc = time.perf_counter()
+    ref, _ = oracle.fp8_decode_attn(oracle.bf16_bits(qs[(W + K - 1) % R][torch.tensor(sample, device=dev)]),
+                                    k8.index_select(0, idx).cpu().numpy(), v8.index_select(0, idx).cpu().numpy(),
+                                    sc.index_select(0, idx).cpu().numpy(), table, lens[sample].astype(np.int32), w.sm_scale)
+    oracle_s = time.perf_counter() - tc
+    got = out[torch.tensor(sample, device=dev)].float().cpu().numpy().astype(np.float64)
+    rel = float((np.linalg.norm(got - ref, axis=-1) / np.linalg.norm(ref, axis=-1)).max())
+    oracle_bytes = float(lens[sample].sum()) * per_token
+    value = total / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "FP8-page decode-attn achieved HBM GB/s and seq-steps/s per layer", "value": round(value, 2), "unit": "GB/s",
+        "n_gpus": 1, "steps": K, "warmup": W, "ms_per_step": round(ms / K, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "e4m3 pages, fp16 products, fp32 accumulation", "data": "synthetic",
+        "config": {**workload_config(w, lens, cfg_id), "bytes_per_cached_token": per_token + per_page / P,
+                   "l2": f"KV read per step {total / K / 1e9:.2f} GB >> 126 MB L2; activations rotate over {R} buffers"},
+        "seq_steps_per_s": round(B * K / (ms * 1e-3), 1), "pct_of_measured_hbm_peak": round(100 * value / peak, 2),
+        "clocks": clocks, "gpu_launches": 3 * K,
+        "roofline": {"bound": "hbm", "kernel": "decode_attn_split_fp8_kernel", "achieved": round(achieved, 2), "peak": peak,
+                     "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "algorithmic_bytes_per_launch": int(per_launch), "avg_launch_ms": round(split_ms, 5)},
+        "parity_check": {"sequences": sample, "max_row_rel_l2": round(rel, 6)},
+        "cpu_baseline": {"value": round(oracle_bytes / oracle_s / 1e9, 4), "unit": "GB/s", "cores": os.cpu_count(), "kind": "oracle",
+                         "sample": f"FP8 oracle on sequences {sample} ({int(lens[sample].sum())} cached tokens), {oracle_s:.1f} s"},
+    }), flush=True)
+    pd.pd_destroy(ctx)
+
+
 # ------------------------------------------------------------------------------------------ pool toggle
 
 def run_pool_toggle(args):
@@ -767,10 +884,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--step", default="fused", choices=["separate", "fused"],
                     help="decode: pd_kv_append + pd_decode_attn (3 launches) or pd_decode_step (2 launches)")
-    ap.add_argument("--op", default="decode", choices=["decode", "kv_transfer", "prefill", "fit_b", "pool_toggle"],
+    ap.add_argument("--op", default="decode", choices=["decode", "decode_fp8", "kv_transfer", "prefill", "fit_b", "pool_toggle"],
                     help="decode = the headline decode step; kv_transfer = page gather + scatter; "
                          "prefill = one append-prefill turn; fit_b = decode step time over batch size, fitted to A + b * B; "
-                         "pool_toggle = release and restore of a KV pool's physical memory")
+                         "pool_toggle = release and restore of a KV pool's physical memory; "
+                         "decode_fp8 = the decode step over FP8 (e4m3) KV pages")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
@@ -782,6 +900,8 @@ def main():
         run_prefill(args)
     elif args.op == "fit_b":
         run_fit_b(args)
+    elif args.op == "decode_fp8":
+        run_decode_fp8(args)
     elif args.op == "pool_toggle":
         run_pool_toggle(args)
     else:

@@ -514,8 +514,6 @@ int pd_decode_attn_fp8(pd_ctx *ctx, const void *q, const void *k8, const void *v
     if (batch == 0) return PD_OK;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
-    if (ctx->variant.warps != pd::decode_attn_fp8_warps())
-        return fail(ctx, PD_ERR_UNSUPPORTED, "pd_decode_attn_fp8: the workspace was sized for another worker count");
     if (!ctx->fp8_ready) {
         const cudaError_t e = pd::prepare_decode_attn_fp8();
         if (e != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "fp8 decode kernel attribute", e);

@@ -9,7 +9,8 @@
 // The kernel is the bf16 split kernel's skeleton (same plan of ranges, same warp-private TMA rings, same
 // partial format, same merge kernel) with a different inner product:
 //   * a tile is one 16 x 128 B TMA box (128-byte swizzle); the page's scale record rides along as a
-//     16-byte bulk copy on the K barrier; six stages per warp keep as many bytes in flight as bf16 did;
+//     16-byte bulk copy on the K barrier; sixteen worker warps with three stages each keep as many bytes
+//     in flight per SM as the bf16 kernel does;
 //   * ldmatrix on the byte tile (viewed as b16) hands every lane four consecutive d of a token; two
 //     cvt.rn.f16x2.e4m3x2 make them fp16 pairs, exactly, and Q is converted to fp16 once per segment with
 //     the matching d order, so S^T = K8 Q^T runs on mma.sync fp16 (tokens as M, as in the bf16 kernel);
@@ -25,6 +26,8 @@
 
 #include <cuda_fp16.h>
 #include <cuda_fp8.h>
+
+#include <cstdlib>
 
 namespace pd {
 
@@ -366,7 +369,6 @@ constexpr size_t fp8_smem_bytes() {
            sizeof(Plan) + WARPS * STAGES * 4 + 32 * 4 + (kMaxBatch + 1) * 4;
 }
 
-constexpr int kFp8Warps = 8, kFp8Stages = 6;
 
 // ---- whole-page quantiser: one CTA per (page, KV head), K then V
 __device__ __forceinline__ float block_amax(float v, float *red) {
@@ -462,19 +464,40 @@ __global__ void __launch_bounds__(256) kv_append_fp8_kernel(const AppendFp8Param
 
 }  // namespace
 
-size_t decode_attn_fp8_smem_bytes() { return fp8_smem_bytes<kFp8Warps, kFp8Stages>(); }
-int decode_attn_fp8_warps() { return kFp8Warps; }
+namespace {
+// Worker warps per CTA x stages per warp: the bytes in flight per SM stay at 192 KB. The conversions make a
+// page cost ~380 instructions in half the time a bf16 page has, and with two warps per scheduler the
+// dependent chains (convert, MMA, softmax) left the issue slots idle: measured 4.4 TB/s with 8 warps x 6
+// stages, 5.5 with 12 x 4, 6.3 with 16 x 3 (128 registers, no spills), which is the default.
+int fp8_shape() {
+    static const int v = [] {
+        const char *e = std::getenv("PD_TUNE_FP8_WARPS");
+        const int w = e != nullptr ? std::atoi(e) : 16;
+        return (w == 8 || w == 12) ? w : 16;
+    }();
+    return v;
+}
+template <typename F>
+cudaError_t with_fp8_kernel(F &&f) {
+    switch (fp8_shape()) {
+        case 8: return f(decode_attn_split_fp8_kernel<8, 6>, fp8_smem_bytes<8, 6>(), 8);
+        case 12: return f(decode_attn_split_fp8_kernel<12, 4>, fp8_smem_bytes<12, 4>(), 12);
+        default: return f(decode_attn_split_fp8_kernel<16, 3>, fp8_smem_bytes<16, 3>(), 16);
+    }
+}
+}  // namespace
 
 cudaError_t prepare_decode_attn_fp8() {
-    return cudaFuncSetAttribute(decode_attn_split_fp8_kernel<kFp8Warps, kFp8Stages>,
-                                cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                static_cast<int>(fp8_smem_bytes<kFp8Warps, kFp8Stages>()));
+    return with_fp8_kernel([](auto *k, size_t bytes, int) {
+        return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+    });
 }
 
 cudaError_t launch_decode_attn_fp8(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, int num_ctas,
                                    cudaStream_t stream) {
-    return launch_pdl(decode_attn_split_fp8_kernel<kFp8Warps, kFp8Stages>, dim3(num_ctas), dim3(kFp8Warps * 32),
-                      fp8_smem_bytes<kFp8Warps, kFp8Stages>(), stream, p.pdl != 0, tm_k, tm_v, p);
+    return with_fp8_kernel([&](auto *k, size_t bytes, int warps) {
+        return launch_pdl(k, dim3(num_ctas), dim3(warps * 32), bytes, stream, p.pdl != 0, tm_k, tm_v, p);
+    });
 }
 
 cudaError_t launch_kv_quantize_pages(const QuantizeParams &p, cudaStream_t stream) {

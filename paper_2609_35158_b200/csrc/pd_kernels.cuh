@@ -164,8 +164,6 @@ cudaError_t launch_decode_attn(const AttnVariant &v, const CUtensorMap &tm_k, co
 cudaError_t launch_lse_merge(int head_dim, const AttnParams &p, cudaStream_t stream);
 // FP8 pages (head_dim 128): the split kernel writes the same partials and plan, so launch_lse_merge follows it
 cudaError_t prepare_decode_attn_fp8();
-size_t decode_attn_fp8_smem_bytes();
-int decode_attn_fp8_warps();
 cudaError_t launch_decode_attn_fp8(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, int num_ctas,
                                    cudaStream_t stream);
 cudaError_t launch_kv_quantize_pages(const QuantizeParams &p, cudaStream_t stream);
