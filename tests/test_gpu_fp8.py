@@ -232,3 +232,53 @@ def test_fp8_full_size_config_sampled_sequences(config):
     # long contexts average unit-variance values to outputs of ~0.02: compare at that scale
     assert_parity((out[torch.tensor(sample, device=DEV)].float() * 32).to(torch.bfloat16), ref * 32,
                   f"config {config}", scale_abs_by_magnitude=True)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_fp8_random_case(seed):
+    import math
+
+    import paper_2609_35158_b200 as pd
+
+    rng = np.random.default_rng(4000 + seed)
+    d = 128
+    g = int(rng.choice([1, 2, 4, 8]))
+    Hkv = int(rng.choice([1, 2, 4, 8]))
+    Hq = g * Hkv
+    B = int(rng.integers(1, 13))
+    kind = seed % 4
+    if kind == 0:
+        lens = rng.integers(0, 48, size=B)
+    elif kind == 1:
+        lens = rng.integers(1, 700, size=B)
+    elif kind == 2:
+        lens = np.where(rng.random(B) < 0.3, rng.integers(2000, 6000, size=B), rng.integers(1, 64, size=B))
+    else:
+        lens = 16 * rng.integers(1, 40, size=B) + rng.choice([-1, 0, 1], size=B)
+    lens = np.maximum(lens, 0).astype(np.int32)
+    split = int(rng.choice([0, 0, 1, 2, 5, 13, 64, 100000]))
+    cache = wl.build_paged_cache(lens, Hkv, d, seed=4100 + seed, device=DEV, poison=True,
+                                 max_pages_per_seq=int(max(1, (lens.max() + 15) // 16 + rng.integers(0, 5))))
+    cache.k_pages.mul_(float(rng.choice([0.25, 1.0, 6.0])))
+    cache.v_pages.mul_(float(rng.choice([0.01, 1.0, 30.0])))
+    k8, v8, sc, _ = quantized_on_host(cache, lens)
+    q = wl.random_bf16((B, Hq, d), 4200 + seed, DEV)
+    scale = float(rng.choice([1.0 / math.sqrt(d), 0.05]))
+    ref, ref_lse = oracle.fp8_decode_attn(oracle.bf16_bits(q), k8, v8, sc, cache.page_table_host, lens, scale)
+    k8d, v8d, scd = to_dev(k8, v8, sc)
+    out = torch.full((B, Hq, d), float("nan"), dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device=DEV)
+    with Ctx(Hq, Hkv, d, B + int(rng.integers(0, 4)), cache.page_table.shape[1], cache.k_pages.shape[0]) as ctx:
+        pd.pd_decode_attn_fp8(ctx.h, q, k8d, v8d, scd, cache.page_table, cache.ctx_lens, out, lse, sm_scale=scale,
+                              split_pages=split)
+        torch.cuda.synchronize()
+        assert pd.pd_device_status(ctx.h)[0] == 0
+    what = f"seed {seed}: B={B} {Hq}/{Hkv} split={split} lens={lens.tolist()}"
+    live = lens > 0
+    if live.any():
+        # compare at unit output scale: divide by the RMS of the reference rows
+        rms = float(np.sqrt(np.mean(ref[live] ** 2))) or 1.0
+        assert_parity((out[torch.from_numpy(live).to(DEV)].float() / rms).to(torch.bfloat16), ref[live] / rms, what,
+                      scale_abs_by_magnitude=True)
+        np.testing.assert_allclose(lse.cpu().numpy()[live], ref_lse[live], rtol=3e-5, atol=3e-5, err_msg=what)
+    assert np.all(np.isneginf(lse.cpu().numpy()[~live]))
