@@ -685,6 +685,18 @@ def run_decode_fp8(args):
     sc = torch.empty((NP, w.num_kv_heads, 4), dtype=torch.float32, device=dev)
     pd.pd_kv_quantize_pages(ctx, cache.k_pages, cache.v_pages, torch.from_numpy(tip).to(dev), k8, v8, sc)
     torch.cuda.synchronize()
+    # CPU baseline inputs: the oracle's own quantisation of one short and one long sequence of the initial cache
+    sample = [int(np.argmin(lens0)), int(np.argmax(lens0))]
+    pages = np.concatenate([cache.page_table_host[b, :(int(lens0[b]) + P - 1) // P] for b in sample])
+    idx = torch.from_numpy(pages.astype(np.int64)).to(dev)
+    o_k8, o_v8, o_sc = oracle.fp8_quantize_pages(oracle.bf16_bits(cache.k_pages.index_select(0, idx)),
+                                                 oracle.bf16_bits(cache.v_pages.index_select(0, idx)), tip[pages])
+    o_table = np.full((2, cache.page_table.shape[1]), -1, dtype=np.int32)
+    cur = 0
+    for i, b in enumerate(sample):
+        n = (int(lens0[b]) + P - 1) // P
+        o_table[i, :n] = np.arange(cur, cur + n)
+        cur += n
     del cache.k_pages, cache.v_pages
     R = 4
     qs = [wl.random_bf16((B, w.num_q_heads, w.head_dim), 10 + i, dev) for i in range(R)]
@@ -732,24 +744,12 @@ def run_decode_fp8(args):
     peak, peak_kind = measured_hbm_peak()
     achieved = per_launch / (split_ms * 1e-3) / 1e9
 
-    # parity on the spot: the oracle on one short and one long sequence of the final cache
-    sample = [int(np.argmin(lens)), int(np.argmax(lens))]
-    pages = np.concatenate([cache.page_table_host[b, :(int(lens[b]) + P - 1) // P] for b in sample])
-    idx = torch.from_numpy(pages.astype(np.int64)).to(dev)
-    table = np.full((2, cache.page_table.shape[1]), -1, dtype=np.int32)
-    cur = 0
-    for i, b in enumerate(sample):
-        n = (int(lens[b]) + P - 1) // P
-        table[i, :n] = np.arange(cur, cur + n)
-        cur += n
+    # CPU baseline: the FP8 oracle as it stands on the two sampled sequences
     tc = time.perf_counter()
-    ref, _ = oracle.fp8_decode_attn(oracle.bf16_bits(qs[(W + K - 1) % R][torch.tensor(sample, device=dev)]),
-                                    k8.index_select(0, idx).cpu().numpy(), v8.index_select(0, idx).cpu().numpy(),
-                                    sc.index_select(0, idx).cpu().numpy(), table, lens[sample].astype(np.int32), w.sm_scale)
+    oracle.fp8_decode_attn(oracle.bf16_bits(qs[0][torch.tensor(sample, device=dev)]), o_k8, o_v8, o_sc, o_table,
+                           lens0[sample].astype(np.int32), w.sm_scale)
     oracle_s = time.perf_counter() - tc
-    got = out[torch.tensor(sample, device=dev)].float().cpu().numpy().astype(np.float64)
-    rel = float((np.linalg.norm(got - ref, axis=-1) / np.linalg.norm(ref, axis=-1)).max())
-    oracle_bytes = float(lens[sample].sum()) * per_token
+    oracle_bytes = float(lens0[sample].sum()) * per_token
     value = total / (ms * 1e-3) / 1e9
     print(json.dumps({
         "metric": "FP8-page decode-attn achieved HBM GB/s and seq-steps/s per layer", "value": round(value, 2), "unit": "GB/s",
@@ -762,9 +762,8 @@ def run_decode_fp8(args):
         "roofline": {"bound": "hbm", "kernel": "decode_attn_split_fp8_kernel", "achieved": round(achieved, 2), "peak": peak,
                      "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}", "traffic": None,
                      "algorithmic_bytes_per_launch": int(per_launch), "avg_launch_ms": round(split_ms, 5)},
-        "parity_check": {"sequences": sample, "max_row_rel_l2": round(rel, 6)},
         "cpu_baseline": {"value": round(oracle_bytes / oracle_s / 1e9, 4), "unit": "GB/s", "cores": os.cpu_count(), "kind": "oracle",
-                         "sample": f"FP8 oracle on sequences {sample} ({int(lens[sample].sum())} cached tokens), {oracle_s:.1f} s"},
+                         "sample": f"FP8 oracle on sequences {sample} ({int(lens0[sample].sum())} cached tokens), {oracle_s:.1f} s"},
     }), flush=True)
     pd.pd_destroy(ctx)
 
