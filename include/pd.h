@@ -143,7 +143,8 @@ int pd_decode_step(pd_ctx *ctx, const void *q, const void *k_new, const void *v_
  * (appending, advancing ctx_lens, attending over the grown contexts), copies the
  * result to out_host (host, [batch][num_q_heads][head_dim] bf16) and waits for
  * the stream, so out_host is valid on return. The cache itself (k_pages,
- * v_pages, page_table, ctx_lens) stays on the device.
+ * v_pages, page_table, ctx_lens) stays on the device. If k_new_host starts where
+ * q_host ends and v_new_host where k_new_host ends, the three travel in one copy.
  */
 int pd_decode_step_host(pd_ctx *ctx, const void *q_host, const void *k_new_host, const void *v_new_host,
                         void *k_pages, void *v_pages, const int32_t *page_table, int32_t *ctx_lens,

@@ -238,10 +238,10 @@ int pd_create(const pd_config *cfg, pd_ctx **out) {
     ctx->cum_pages = reinterpret_cast<int32_t *>(w); w += b_cum;
     ctx->plan = reinterpret_cast<int32_t *>(w); w += b_plan;
     ctx->status = reinterpret_cast<int32_t *>(w); w += b_status;
-    ctx->stage_q = reinterpret_cast<__nv_bfloat16 *>(w); w += b_q;
-    ctx->stage_out = reinterpret_cast<__nv_bfloat16 *>(w); w += b_q;
+    ctx->stage_q = reinterpret_cast<__nv_bfloat16 *>(w); w += b_q;  // q, k_new, v_new are adjacent: one copy can fill them
     ctx->stage_k = reinterpret_cast<__nv_bfloat16 *>(w); w += b_kv;
     ctx->stage_v = reinterpret_cast<__nv_bfloat16 *>(w); w += b_kv;
+    ctx->stage_out = reinterpret_cast<__nv_bfloat16 *>(w); w += b_q;
     if (b_trace != 0) {
         ctx->trace = reinterpret_cast<unsigned long long *>(w);
         ctx->trace_workers = n_workers;
@@ -664,11 +664,30 @@ int pd_decode_step_host(pd_ctx *ctx, const void *q_host, const void *k_new_host,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t nq = static_cast<size_t>(batch) * ctx->cfg.num_q_heads * ctx->cfg.head_dim * 2;
     const size_t nkv = static_cast<size_t>(batch) * ctx->cfg.num_kv_heads * ctx->cfg.head_dim * 2;
-    cudaError_t err = cudaMemcpyAsync(ctx->stage_q, q_host, nq, cudaMemcpyHostToDevice, s);
-    if (err == cudaSuccess) err = cudaMemcpyAsync(ctx->stage_k, k_new_host, nkv, cudaMemcpyHostToDevice, s);
-    if (err == cudaSuccess) err = cudaMemcpyAsync(ctx->stage_v, v_new_host, nkv, cudaMemcpyHostToDevice, s);
+    // Host buffers that follow one another in memory (q, then k_new, then v_new) travel in one copy. Adjacent
+    // addresses can still belong to separately pinned allocations, which a single copy may not span: if the
+    // runtime refuses it, nothing was enqueued and the three buffers are copied one by one.
+    const char *qh = static_cast<const char *>(q_host);
+    bool adjacent = static_cast<const char *>(k_new_host) == qh + nq && static_cast<const char *>(v_new_host) == qh + nq + nkv;
+    __nv_bfloat16 *dq = ctx->stage_q, *dk = ctx->stage_k, *dv = ctx->stage_v;
+    cudaError_t err = cudaSuccess;
+    if (adjacent) {
+        err = cudaMemcpyAsync(dq, q_host, nq + 2 * nkv, cudaMemcpyHostToDevice, s);
+        if (err == cudaSuccess) {
+            dk = reinterpret_cast<__nv_bfloat16 *>(reinterpret_cast<char *>(dq) + nq);
+            dv = reinterpret_cast<__nv_bfloat16 *>(reinterpret_cast<char *>(dq) + nq + nkv);
+        } else {
+            (void)cudaGetLastError();
+            adjacent = false;
+        }
+    }
+    if (!adjacent) {
+        err = cudaMemcpyAsync(dq, q_host, nq, cudaMemcpyHostToDevice, s);
+        if (err == cudaSuccess) err = cudaMemcpyAsync(dk, k_new_host, nkv, cudaMemcpyHostToDevice, s);
+        if (err == cudaSuccess) err = cudaMemcpyAsync(dv, v_new_host, nkv, cudaMemcpyHostToDevice, s);
+    }
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "host-to-device copy", err);
-    if (int rc = pd_decode_step(ctx, ctx->stage_q, ctx->stage_k, ctx->stage_v, k_pages, v_pages, page_table, ctx_lens,
+    if (int rc = pd_decode_step(ctx, dq, dk, dv, k_pages, v_pages, page_table, ctx_lens,
                                 ctx->stage_out, nullptr, batch, sm_scale, split_pages, stream))
         return rc;
     err = cudaMemcpyAsync(out_host, ctx->stage_out, nq, cudaMemcpyDeviceToHost, s);

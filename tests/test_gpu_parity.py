@@ -256,6 +256,16 @@ def test_host_step_equals_append_plus_attention():
         assert torch.equal(out_host, out_dev.cpu())
         assert torch.equal(caches[0].k_pages, caches[1].k_pages)
         assert c.ctx_lens.cpu().tolist() == (lens + 1).tolist()
+        # host buffers that follow one another (q, k_new, v_new in one slab) take the single-copy path
+        slab = torch.empty(q.numel() + kn.numel() + vn.numel(), dtype=torch.bfloat16).pin_memory()
+        a, b2 = q.numel(), q.numel() + kn.numel()
+        slab[:a].copy_(q.reshape(-1)); slab[a:b2].copy_(kn.reshape(-1)); slab[b2:].copy_(vn.reshape(-1))
+        c2 = wl.build_paged_cache(lens, w.num_kv_heads, w.head_dim, seed=0, device=DEV, reserve_tokens=4)
+        out_slab = torch.empty_like(out_host).pin_memory()
+        ctx.pd.pd_decode_step_host(ctx.h, slab[:a].view(q.shape), slab[a:b2].view(kn.shape), slab[b2:].view(vn.shape),
+                                   c2.k_pages, c2.v_pages, c2.page_table, c2.ctx_lens, out_slab, sm_scale=w.sm_scale)
+        assert torch.equal(out_slab, out_host)
+        assert torch.equal(c2.k_pages, caches[0].k_pages) and torch.equal(c2.v_pages, caches[0].v_pages)
 
 
 def test_bad_page_id_is_reported_not_fatal():
