@@ -128,3 +128,21 @@ def test_error_metric_helper():
     got[0, 0, 1] = 0.5
     m, r = error_metrics(got, ref)
     assert m == 0.5 and abs(r - 0.5) < 1e-12
+
+
+def test_reference_arm_prints_the_contract_line():
+    """bench.py --impl reference times the oracle on the host cores and prints one JSON line with the keys the
+    driver reads (runs on the smallest configuration here)."""
+    import json
+
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "0",
+                          "--steps", "2", "--warmup", "1"], capture_output=True, text=True, timeout=600, cwd=ROOT)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    r = json.loads(lines[0])
+    assert r["impl"] == "reference" and r["n_gpus"] == 1 and r["steps"] == 2 and r["warmup"] == 1
+    assert r["unit"] == "GB/s" and r["higher_is_better"] is True and r["value"] > 0 and r["gpu_launches"] == 0
+    assert r["cpu_baseline"]["kind"] == "oracle" and r["cpu_baseline"]["value"] == r["value"] and r["cpu_baseline"]["cores"] >= 1
+    assert r["e2e"] == {"value": r["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    assert "workload" in r["config"] and r["data"] == "synthetic"
