@@ -392,6 +392,19 @@ int pd_decode_attn_fp8(pd_ctx *ctx, const void *q, const void *k8, const void *v
                        const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse,
                        int32_t batch, float sm_scale, int32_t split_pages, void *stream);
 
+/*
+ * pd_kv_gather / pd_kv_scatter for FP8 pools: a packed page is the K block, the V block (num_kv_heads *
+ * 16 * head_dim bytes each) and the page's num_kv_heads scale records (16 bytes each), so the scales
+ * travel with their page. K = 2 * num_kv_heads * head_dim + num_kv_heads bytes per token per layer.
+ * Everything else as the bf16 calls.
+ */
+int pd_kv_gather_fp8(pd_ctx *ctx, const void *k8, const void *v8, const float *kv_scales, const int32_t *page_table,
+                     const int32_t *page_begin, const int32_t *page_end, const int64_t *packed_page_offset,
+                     void *packed, int32_t batch, void *stream);
+int pd_kv_scatter_fp8(pd_ctx *ctx, const void *packed, const int64_t *packed_page_offset, void *k8, void *v8,
+                      float *kv_scales, const int32_t *page_table, const int32_t *page_begin,
+                      const int32_t *page_end, int32_t batch, void *stream);
+
 /* ---- Elastic KV pool on CUDA virtual memory management (Sec. 4.6: the intra-scale toggle keeps the
  * rollout process and swaps device state; Sec. 5: the KV cache is released when training begins and
  * restored when the GPU is available again). A pool is a device address range of `capacity` bytes whose

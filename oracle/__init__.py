@@ -330,3 +330,35 @@ def fp8_decode_attn(q, k8, v8, scales, page_table, ctx_lens, sm_scale, *, nthrea
     if rc != 0:
         raise RuntimeError(f"pd_oracle_fp8_decode_attn failed ({rc})")
     return out, lse
+
+
+def fp8_kv_gather(k8, v8, scales, page_table, page_begin, page_end, dst_page_offset, total_pages: int) -> np.ndarray:
+    """Packs logical pages [page_begin[b], page_end[b]) of every sequence: packed page i is the K block, the V
+    block and the Hkv scale records (as bytes) of one pool page. Returns uint8 [total_pages, 2*Hkv*P*d + Hkv*16]."""
+    k8 = _c(k8, np.uint8)
+    v8 = _c(v8, np.uint8)
+    scales = _c(scales, np.float32)
+    NP, Hkv, P, d = k8.shape
+    block = Hkv * P * d
+    packed = np.zeros((total_pages, 2 * block + Hkv * 16), dtype=np.uint8)
+    for b in range(len(page_begin)):
+        for i, lp in enumerate(range(int(page_begin[b]), int(page_end[b]))):
+            page = int(page_table[b, lp])
+            row = packed[int(dst_page_offset[b]) + i]
+            row[:block] = k8[page].reshape(-1)
+            row[block:2 * block] = v8[page].reshape(-1)
+            row[2 * block:] = scales[page].reshape(-1).view(np.uint8)
+    return packed
+
+
+def fp8_kv_scatter(packed, src_page_offset, k8, v8, scales, page_table, page_begin, page_end) -> None:
+    """The inverse of ``fp8_kv_gather``, in place on k8, v8 and scales."""
+    NP, Hkv, P, d = k8.shape
+    block = Hkv * P * d
+    for b in range(len(page_begin)):
+        for i, lp in enumerate(range(int(page_begin[b]), int(page_end[b]))):
+            page = int(page_table[b, lp])
+            row = packed[int(src_page_offset[b]) + i]
+            k8[page] = row[:block].reshape(Hkv, P, d)
+            v8[page] = row[block:2 * block].reshape(Hkv, P, d)
+            scales[page] = row[2 * block:].view(np.float32).reshape(Hkv, 4)

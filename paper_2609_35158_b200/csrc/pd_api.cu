@@ -298,12 +298,13 @@ int pd_kv_append(pd_ctx *ctx, const void *k_new, const void *v_new, void *k_page
 
 namespace {
 
-int kv_transfer(pd_ctx *ctx, bool scatter, void *k_pages, void *v_pages, const int32_t *page_table,
+int kv_transfer(pd_ctx *ctx, bool scatter, void *k_pages, void *v_pages, float *kv_scales, const int32_t *page_table,
                 const int32_t *page_begin, const int32_t *page_end, const int64_t *packed_page_offset, void *packed,
                 int32_t batch, void *stream) {
     if (int rc = check_batch(ctx, batch)) return rc;
     if (!aligned16(k_pages) || !aligned16(v_pages) || !aligned16(packed) || page_table == nullptr ||
-        page_begin == nullptr || page_end == nullptr || packed_page_offset == nullptr)
+        page_begin == nullptr || page_end == nullptr || packed_page_offset == nullptr ||
+        (kv_scales != nullptr && !aligned16(kv_scales)))
         return fail(ctx, PD_ERR_INVALID_ARG, "KV transfer: null or misaligned pointer");
     if (batch == 0) return PD_OK;
     DeviceGuard guard(ctx->cfg.device);
@@ -323,6 +324,8 @@ int kv_transfer(pd_ctx *ctx, bool scatter, void *k_pages, void *v_pages, const i
     p.MP = ctx->cfg.max_pages_per_seq;
     p.num_pages = static_cast<int32_t>(ctx->cfg.num_pages);
     p.pdl = ctx->pdl;
+    p.elem_bytes = kv_scales != nullptr ? 1 : 2;
+    p.scales = kv_scales;
     const cudaError_t err = pd::launch_kv_transfer(p, scatter, ctx->num_sms, static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, scatter ? "kv_scatter launch" : "kv_gather launch", err);
     ctx->launches += 1;
@@ -334,14 +337,30 @@ int kv_transfer(pd_ctx *ctx, bool scatter, void *k_pages, void *v_pages, const i
 int pd_kv_gather(pd_ctx *ctx, const void *k_pages, const void *v_pages, const int32_t *page_table,
                  const int32_t *page_begin, const int32_t *page_end, const int64_t *packed_page_offset, void *packed,
                  int32_t batch, void *stream) {
-    return kv_transfer(ctx, false, const_cast<void *>(k_pages), const_cast<void *>(v_pages), page_table, page_begin,
+    return kv_transfer(ctx, false, const_cast<void *>(k_pages), const_cast<void *>(v_pages), nullptr, page_table, page_begin,
                        page_end, packed_page_offset, packed, batch, stream);
+}
+
+int pd_kv_gather_fp8(pd_ctx *ctx, const void *k8, const void *v8, const float *kv_scales, const int32_t *page_table,
+                     const int32_t *page_begin, const int32_t *page_end, const int64_t *packed_page_offset, void *packed,
+                     int32_t batch, void *stream) {
+    if (ctx != nullptr && kv_scales == nullptr) return fail(ctx, PD_ERR_INVALID_ARG, "pd_kv_gather_fp8: null kv_scales");
+    return kv_transfer(ctx, false, const_cast<void *>(k8), const_cast<void *>(v8), const_cast<float *>(kv_scales), page_table,
+                       page_begin, page_end, packed_page_offset, packed, batch, stream);
+}
+
+int pd_kv_scatter_fp8(pd_ctx *ctx, const void *packed, const int64_t *packed_page_offset, void *k8, void *v8,
+                      float *kv_scales, const int32_t *page_table, const int32_t *page_begin, const int32_t *page_end,
+                      int32_t batch, void *stream) {
+    if (ctx != nullptr && kv_scales == nullptr) return fail(ctx, PD_ERR_INVALID_ARG, "pd_kv_scatter_fp8: null kv_scales");
+    return kv_transfer(ctx, true, k8, v8, kv_scales, page_table, page_begin, page_end, packed_page_offset,
+                       const_cast<void *>(packed), batch, stream);
 }
 
 int pd_kv_scatter(pd_ctx *ctx, const void *packed, const int64_t *packed_page_offset, void *k_pages, void *v_pages,
                   const int32_t *page_table, const int32_t *page_begin, const int32_t *page_end, int32_t batch,
                   void *stream) {
-    return kv_transfer(ctx, true, k_pages, v_pages, page_table, page_begin, page_end, packed_page_offset,
+    return kv_transfer(ctx, true, k_pages, v_pages, nullptr, page_table, page_begin, page_end, packed_page_offset,
                        const_cast<void *>(packed), batch, stream);
 }
 

@@ -81,6 +81,10 @@ struct TransferParams {
     int32_t B, Hkv, D, MP;
     int32_t num_pages;
     int32_t pdl;
+    // FP8 pools: elem_bytes = 1 and the scale records [NP][Hkv][4] fp32 travel with their page (a packed page is
+    // then K block, V block, Hkv records); bf16 pools: elem_bytes = 2, scales = null
+    int32_t elem_bytes;
+    float *scales;
 };
 
 struct PrefillParams {

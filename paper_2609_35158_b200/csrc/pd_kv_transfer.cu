@@ -78,9 +78,11 @@ __global__ void __launch_bounds__(32) kv_transfer_bulk_kernel(const TransferPara
     mbar_init_fence();
     const int pb = p.page_begin[b], pe = p.page_end[b];
     const long long base = p.packed_page_offset[b];
-    const uint32_t block_bytes = static_cast<uint32_t>(p.Hkv) * kPageSize * p.D * 2;  // K (or V) block of a page
+    const uint32_t block_bytes = static_cast<uint32_t>(p.Hkv) * kPageSize * p.D * p.elem_bytes;  // K (or V) block of a page
+    const uint32_t scale_bytes = p.scales != nullptr ? static_cast<uint32_t>(p.Hkv) * 16u : 0u;  // the page's scale records
     const uint32_t chunks_per_block = (block_bytes + kBulkChunk - 1) / kBulkChunk;
-    const uint32_t chunks_per_page = 2 * chunks_per_block;
+    const uint32_t chunks_per_page = 2 * chunks_per_block + (scale_bytes ? 1u : 0u);
+    const size_t packed_page_bytes = 2 * static_cast<size_t>(block_bytes) + scale_bytes;
     // this CTA's pages: pb + blockIdx.x, + gridDim.x, ...
     const int first = pb + blockIdx.x;
     const long long n_pages = first < pe ? (pe - first + gridDim.x - 1) / gridDim.x : 0;
@@ -92,9 +94,7 @@ __global__ void __launch_bounds__(32) kv_transfer_bulk_kernel(const TransferPara
     auto locate = [&](long long i, uint8_t *&pool, uint8_t *&packed, uint32_t &bytes) {
         const int lp = first + static_cast<int>(i / chunks_per_page) * gridDim.x;
         const uint32_t c = static_cast<uint32_t>(i % chunks_per_page);
-        const uint32_t which = c / chunks_per_block, off = (c % chunks_per_block) * kBulkChunk;
         const int page = (lp >= 0 && lp < p.MP) ? p.page_table[static_cast<size_t>(b) * p.MP + lp] : -1;
-        bytes = min(static_cast<uint32_t>(kBulkChunk), block_bytes - off);
         if (page < 0 || page >= p.num_pages) {
             if (c == 0 && atomicCAS(p.status, kDevOk, kDevBadPage) == kDevOk) {
                 p.status[1] = b;
@@ -103,9 +103,17 @@ __global__ void __launch_bounds__(32) kv_transfer_bulk_kernel(const TransferPara
             bytes = 0;
             return;
         }
+        uint8_t *packed_page = reinterpret_cast<uint8_t *>(p.packed) + (static_cast<size_t>(base) + (lp - pb)) * packed_page_bytes;
+        if (c == 2 * chunks_per_block) {  // the scale records
+            bytes = scale_bytes;
+            pool = reinterpret_cast<uint8_t *>(p.scales) + static_cast<size_t>(page) * scale_bytes;
+            packed = packed_page + 2 * static_cast<size_t>(block_bytes);
+            return;
+        }
+        const uint32_t which = c / chunks_per_block, off = (c % chunks_per_block) * kBulkChunk;
+        bytes = min(static_cast<uint32_t>(kBulkChunk), block_bytes - off);
         pool = reinterpret_cast<uint8_t *>(which ? p.v_pages : p.k_pages) + static_cast<size_t>(page) * block_bytes + off;
-        packed = reinterpret_cast<uint8_t *>(p.packed) +
-                 (static_cast<size_t>(base) + (lp - pb)) * 2 * block_bytes + static_cast<size_t>(which) * block_bytes + off;
+        packed = packed_page + static_cast<size_t>(which) * block_bytes + off;
     };
 
     for (long long i = 0; i < n + kBulkAhead && ok; ++i) {
@@ -149,11 +157,11 @@ cudaError_t launch_kv_transfer(const TransferParams &p, bool scatter, int num_sm
         const char *e = std::getenv("PD_TUNE_TRANSFER_BULK");
         return e != nullptr ? std::atoi(e) : 128;
     }();
-    if (use_bulk > 0) {
+    if (use_bulk > 0 || p.elem_bytes != 2) {  // FP8 pools always take the bulk kernel
         // CTAs per sequence: `use_bulk` per SM over the batch. Many short-lived CTAs of a page or two each
         // measured 6.7 TB/s against 6.0 TB/s for two long-lived CTAs per SM: SMs that get more bandwidth simply
         // take more CTAs.
-        int per_seq = (use_bulk * num_sms + p.B - 1) / p.B;
+        int per_seq = ((use_bulk > 0 ? use_bulk : 128) * num_sms + p.B - 1) / p.B;
         per_seq = per_seq < 1 ? 1 : (per_seq > p.MP ? p.MP : per_seq);
         const dim3 grid(per_seq, p.B);
         const size_t smem = static_cast<size_t>(kBulkStages) * kBulkChunk;

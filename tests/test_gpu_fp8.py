@@ -282,3 +282,53 @@ def test_fp8_random_case(seed):
                       scale_abs_by_magnitude=True)
         np.testing.assert_allclose(lse.cpu().numpy()[live], ref_lse[live], rtol=3e-5, atol=3e-5, err_msg=what)
     assert np.all(np.isneginf(lse.cpu().numpy()[~live]))
+
+
+def test_fp8_gather_scatter_bit_exact_and_attention_on_the_moved_cache():
+    import paper_2609_35158_b200 as pd
+
+    Hq, Hkv, d = 32, 8, 128
+    lens = np.array([40, 1000, 17, 333, 2048], dtype=np.int32)
+    B = len(lens)
+    src = wl.build_paged_cache(lens, Hkv, d, seed=90, device=DEV)
+    dst = wl.build_paged_cache(lens, Hkv, d, seed=91, device=DEV)  # other page ids, other contents
+    k8, v8, sc, _ = quantized_on_host(src, lens, poison_codes=False)
+    n_pages = (lens + P - 1) // P
+    pb = np.zeros(B, dtype=np.int32)
+    pb[1] = 3  # move only the pages from logical page 3 on for sequence 1 (as after a prefix hit)
+    pe = n_pages.astype(np.int32)
+    counts = pe - pb
+    off = np.concatenate([[0], np.cumsum(counts)[:-1]]).astype(np.int64)
+    total = int(counts.sum())
+    want = oracle.fp8_kv_gather(k8, v8, sc, src.page_table_host, pb, pe, off, total)
+    k8d, v8d, scd = to_dev(k8, v8, sc)
+    d_pb, d_pe, d_off = to_dev(pb, pe, off)
+    packed = torch.full((total, want.shape[1]), 0xAA, dtype=torch.uint8, device=DEV)
+    NPd = dst.k_pages.shape[0]
+    dk = torch.zeros((NPd, Hkv, P, d), dtype=torch.uint8, device=DEV)
+    dv = torch.zeros_like(dk)
+    ds = torch.zeros((NPd, Hkv, 4), dtype=torch.float32, device=DEV)
+    q = wl.random_bf16((B, Hq, d), 92, DEV)
+    with Ctx(Hq, Hkv, d, B, src.page_table.shape[1], src.k_pages.shape[0]) as cs, \
+            Ctx(Hq, Hkv, d, B, dst.page_table.shape[1], NPd) as cd:
+        pd.pd_kv_gather_fp8(cs.h, k8d, v8d, scd, src.page_table, d_pb, d_pe, d_off, packed)
+        torch.cuda.synchronize()
+        assert np.array_equal(packed.cpu().numpy(), want)
+        # the receiver already holds the first three pages of sequence 1 (the shared prefix)
+        want_k, want_v, want_s = dk.cpu().numpy(), dv.cpu().numpy(), ds.cpu().numpy()
+        for lp in range(3):
+            s_page, t_page = src.page_table_host[1, lp], dst.page_table_host[1, lp]
+            want_k[t_page], want_v[t_page], want_s[t_page] = k8[s_page], v8[s_page], sc[s_page]
+        dk.copy_(torch.from_numpy(want_k)); dv.copy_(torch.from_numpy(want_v)); ds.copy_(torch.from_numpy(want_s))
+        oracle.fp8_kv_scatter(want, off, want_k, want_v, want_s, dst.page_table_host, pb, pe)
+        pd.pd_kv_scatter_fp8(cd.h, packed, d_off, dk, dv, ds, dst.page_table, d_pb, d_pe)
+        torch.cuda.synchronize()
+        assert pd.pd_device_status(cs.h)[0] == 0 and pd.pd_device_status(cd.h)[0] == 0
+        assert np.array_equal(dk.cpu().numpy(), want_k) and np.array_equal(dv.cpu().numpy(), want_v)
+        assert np.array_equal(ds.cpu().numpy().view(np.uint32), want_s.view(np.uint32))
+        out_s = torch.empty((B, Hq, d), dtype=torch.bfloat16, device=DEV)
+        out_d = torch.empty_like(out_s)
+        pd.pd_decode_attn_fp8(cs.h, q, k8d, v8d, scd, src.page_table, src.ctx_lens, out_s, sm_scale=d ** -0.5, split_pages=7)
+        pd.pd_decode_attn_fp8(cd.h, q, dk, dv, ds, dst.page_table, dst.ctx_lens, out_d, sm_scale=d ** -0.5, split_pages=7)
+        torch.cuda.synchronize()
+        assert torch.equal(out_s.view(torch.int16), out_d.view(torch.int16))

@@ -207,3 +207,34 @@ def test_fp8_append_against_separate_index_arithmetic():
     # the stored-scale path really saturated somewhere, and a fresh page keeps a factor two of headroom
     assert (np.abs(oracle.e4m3_to_f64(v8[3, :, 5])) == 448.0).any()
     assert np.abs(oracle.e4m3_to_f64(k8[0, :, 0])).max() == 224.0
+
+
+# ---------------------------------------------------------------- page gather / scatter
+
+def test_fp8_gather_layout_and_scatter_round_trip():
+    rng = np.random.default_rng(40)
+    NP, Hkv, d = 11, 2, 64
+    k8 = rng.integers(0, 256, size=(NP, Hkv, P, d)).astype(np.uint8)
+    v8 = rng.integers(0, 256, size=(NP, Hkv, P, d)).astype(np.uint8)
+    sc = rng.uniform(0.01, 2.0, size=(NP, Hkv, 4)).astype(np.float32)
+    table = np.array([[3, 7, 1, -1], [10, 0, 5, 2]], dtype=np.int32)
+    pb, pe = np.array([1, 0]), np.array([3, 4])
+    off = np.array([4, 0])  # sequence 1's pages first, then sequence 0's
+    packed = oracle.fp8_kv_gather(k8, v8, sc, table, pb, pe, off, 6)
+    block = Hkv * P * d
+    assert packed.shape == (6, 2 * block + Hkv * 16)
+    # packed page 4 is logical page 1 of sequence 0 = pool page 7; packed page 2 is pool page 5
+    for row, page in ((4, 7), (5, 1), (0, 10), (1, 0), (2, 5), (3, 2)):
+        assert packed[row, :block].tobytes() == k8[page].tobytes()
+        assert packed[row, block:2 * block].tobytes() == v8[page].tobytes()
+        assert packed[row, 2 * block:].tobytes() == sc[page].tobytes()
+    # scatter into a differently numbered destination and read the same logical pages back
+    dst_table = np.array([[9, 8, 7, 6], [5, 4, 3, 2]], dtype=np.int32)
+    dk, dv, ds = np.zeros_like(k8), np.zeros_like(v8), np.zeros_like(sc)
+    oracle.fp8_kv_scatter(packed, off, dk, dv, ds, dst_table, pb, pe)
+    for b in range(2):
+        for lp in range(pb[b], pe[b]):
+            s, t = table[b, lp], dst_table[b, lp]
+            assert np.array_equal(dk[t], k8[s]) and np.array_equal(dv[t], v8[s]) and np.array_equal(ds[t], sc[s])
+    untouched = sorted(set(range(NP)) - {8, 7, 5, 4, 3, 2})
+    assert not dk[untouched].any() and not ds[untouched].any()
