@@ -354,11 +354,12 @@ def test_full_size_configs_all_rows(config):
     print(f"config {config}: max_abs {max_abs:.2e} rel_l2 {rel:.2e} plan {plan}")
 
 
-def test_config4_multiturn_loop_with_page_allocation():
+@pytest.mark.parametrize("fused", [False, True])
+def test_config4_multiturn_loop_with_page_allocation(fused):
     """Config 4 at full batch: 128 steps of (allocate, append, attend) with the host free list in the
-    loop. Every append is checked on the slot it must fill; attention is checked against the oracle on
-    steps 0, 1, 63, 126 and 127 for a sample of sequences that holds the shortest, the longest and
-    several that open a new page during the loop."""
+    loop, as two calls and as the fused step the benchmark times. Every append is checked on the slot it
+    must fill; attention is checked against the oracle on steps 0, 1, 63, 126 and 127 for a sample of
+    sequences that holds the shortest, the longest and several that open a new page during the loop."""
     w = wl.WORKLOADS[4]
     lens0 = wl.context_lengths(4)
     B, steps = w.batch, 128
@@ -380,10 +381,14 @@ def test_config4_multiturn_loop_with_page_allocation():
             q = wl.random_bf16((B, w.num_q_heads, w.head_dim), 4000 + step, DEV)
             kn = wl.random_bf16((B, w.num_kv_heads, w.head_dim), 5000 + step, DEV)
             vn = wl.random_bf16((B, w.num_kv_heads, w.head_dim), 6000 + step, DEV)
-            ctx.pd.pd_kv_append(ctx.h, kn, vn, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens)
             out = torch.empty((B, w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=DEV)
-            ctx.pd.pd_decode_attn(ctx.h, q, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, out,
-                                  sm_scale=w.sm_scale)
+            if fused:
+                ctx.pd.pd_decode_step(ctx.h, q, kn, vn, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens,
+                                      out, sm_scale=w.sm_scale)
+            else:
+                ctx.pd.pd_kv_append(ctx.h, kn, vn, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens)
+                ctx.pd.pd_decode_attn(ctx.h, q, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, out,
+                                      sm_scale=w.sm_scale)
             # append: the slot of every sequence holds exactly the new rows
             pos = torch.from_numpy(lens.astype(np.int64)).to(DEV)
             page = cache.page_table[ar, pos // 16].long()
