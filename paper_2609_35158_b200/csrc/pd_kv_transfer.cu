@@ -165,12 +165,12 @@ cudaError_t launch_kv_transfer(const TransferParams &p, bool scatter, int num_sm
         per_seq = per_seq < 1 ? 1 : (per_seq > p.MP ? p.MP : per_seq);
         const dim3 grid(per_seq, p.B);
         const size_t smem = static_cast<size_t>(kBulkStages) * kBulkChunk;
-        static bool attr_set = false;
-        if (!attr_set) {
-            cudaFuncSetAttribute(kv_transfer_bulk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-            cudaFuncSetAttribute(kv_transfer_bulk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-            attr_set = true;
-        }
+        // the opt-in is per device and costs a microsecond: set it on every launch rather than track devices
+        const cudaError_t e = scatter ? cudaFuncSetAttribute(kv_transfer_bulk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                             static_cast<int>(smem))
+                                      : cudaFuncSetAttribute(kv_transfer_bulk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                             static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
         if (scatter) return launch_pdl(kv_transfer_bulk_kernel<true>, grid, dim3(32), smem, stream, p.pdl != 0, p);
         return launch_pdl(kv_transfer_bulk_kernel<false>, grid, dim3(32), smem, stream, p.pdl != 0, p);
     }
