@@ -663,6 +663,7 @@ int pd_prefill_attn(pd_ctx *ctx, const void *q, const int32_t *q_indptr, const v
     p.pdl = ctx->pdl;
     p.trace = ctx->trace;                    // the worker-trace buffer doubles as [CTA][16] phase counters
     p.trace_ctas = ctx->trace_workers / 4;
+    p.reverse_tiles = env_int("PD_TUNE_PREFILL_REVERSE", 1);
     if (ctx->trace != nullptr) cudaMemsetAsync(ctx->trace, 0, static_cast<size_t>(ctx->trace_workers) * 32, static_cast<cudaStream_t>(stream));
     const cudaError_t err = pd::launch_prefill_attn(ctx->cfg.head_dim, ctx->tm_k, ctx->tm_v, p, max_q_len,
                                                     static_cast<cudaStream_t>(stream));

@@ -101,6 +101,7 @@ struct PrefillParams {
     int32_t pdl;
     unsigned long long *trace;  // optional [trace_ctas][8] SM-clock cycles per phase of row thread 0
     int32_t trace_ctas;
+    int32_t reverse_tiles;      // schedule a sequence's last query tiles (the longest contexts) first
 };
 
 struct AppendTokensParams {

@@ -74,7 +74,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     grid_dependency_wait();
     launch_dependents();
     const int q0 = p.q_indptr[b], q_len = p.q_indptr[b + 1] - q0;
-    const int tile_start = blockIdx.x * TOK;
+    // tiles are scheduled in index order: start a sequence's last tiles (the longest contexts) first
+    const int tile_start = static_cast<int>(p.reverse_tiles ? gridDim.x - 1 - blockIdx.x : blockIdx.x) * TOK;
     if (tile_start >= q_len) return;  // before any allocation
     const int L = min(max(p.ctx_lens[b], 0), p.MP * kPageSize);
     if (L < q_len) {  // the cache must already hold the new tokens
