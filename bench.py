@@ -895,6 +895,17 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
+    if args.impl == "cuda":
+        # the built library is not tracked: compile it if this checkout has none yet (rank 0 first under torchrun)
+        import __graft_entry__ as entry
+
+        if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+            entry.ensure_built()
+        else:
+            for _ in range(600):
+                if os.path.exists(os.path.join(ROOT, "paper_2609_35158_b200", "libpd.so")):
+                    break
+                time.sleep(0.5)
     if args.impl == "reference":
         run_reference(args)
     elif args.op == "kv_transfer":

@@ -67,7 +67,7 @@ def _load() -> ctypes.CDLL:
     path = _build.LIB
     if not os.path.exists(path):
         raise ImportError(
-            f"{path} is missing: build it with `python -m paper_2609_35158_b200.build` "
+            f"{path} is missing: build it with `python paper_2609_35158_b200/build.py` "
             "(nvcc, sm_100a). This package has no fallback path.")
     lib = ctypes.CDLL(path)
     vp, i32, u32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_int64, ctypes.c_float
