@@ -588,7 +588,7 @@ def run_prefill(args):
         "e2e": {"value": round(flops / (e2e_ms * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
                 "h2d_bytes_per_step": int((hq.numel() + hk.numel() + hv.numel()) * 2), "d2h_bytes_per_step": int(hout.numel() * 2),
                 "ms_per_step": round(e2e_ms, 5)},
-        "gpu_launches": 3 * K,
+        "gpu_launches": 4 * K,  # append (2 kernels), sequence ordering, attention
         "roofline": {"bound": "tensor", "kernel": "prefill_attn_kernel", "achieved": round(achieved, 2), "peak": peak,
                      "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}", "traffic": None,
                      "avg_launch_ms": round(attn_ms, 5)},

@@ -664,11 +664,12 @@ int pd_prefill_attn(pd_ctx *ctx, const void *q, const int32_t *q_indptr, const v
     p.trace = ctx->trace;                    // the worker-trace buffer doubles as [CTA][16] phase counters
     p.trace_ctas = ctx->trace_workers / 4;
     p.reverse_tiles = env_int("PD_TUNE_PREFILL_REVERSE", 1);
+    p.order = env_int("PD_TUNE_PREFILL_ORDER", 1) ? ctx->cum_pages : nullptr;  // the decode kernels' prefix-sum buffer is free here
     if (ctx->trace != nullptr) cudaMemsetAsync(ctx->trace, 0, static_cast<size_t>(ctx->trace_workers) * 32, static_cast<cudaStream_t>(stream));
     const cudaError_t err = pd::launch_prefill_attn(ctx->cfg.head_dim, ctx->tm_k, ctx->tm_v, p, max_q_len,
                                                     static_cast<cudaStream_t>(stream));
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "prefill_attn launch", err);
-    ctx->launches += 1;
+    ctx->launches += p.order != nullptr ? 2 : 1;
     return PD_OK;
 }
 

@@ -102,6 +102,7 @@ struct PrefillParams {
     unsigned long long *trace;  // optional [trace_ctas][8] SM-clock cycles per phase of row thread 0
     int32_t trace_ctas;
     int32_t reverse_tiles;      // schedule a sequence's last query tiles (the longest contexts) first
+    int32_t *order;             // [B] sequences by decreasing work, written by a small kernel before the attention (null = index order)
 };
 
 struct AppendTokensParams {

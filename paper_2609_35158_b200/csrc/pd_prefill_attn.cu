@@ -68,11 +68,12 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint32_t tmem_slot;
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int b = blockIdx.z, kvh = blockIdx.y;
+    const int kvh = blockIdx.y;
     const int G = p.G, TOK = kRows / G;
 
     grid_dependency_wait();
     launch_dependents();
+    const int b = p.order != nullptr ? p.order[blockIdx.z] : static_cast<int>(blockIdx.z);  // heaviest sequences first
     const int q0 = p.q_indptr[b], q_len = p.q_indptr[b + 1] - q0;
     // tiles are scheduled in index order: start a sequence's last tiles (the longest contexts) first
     const int tile_start = static_cast<int>(p.reverse_tiles ? gridDim.x - 1 - blockIdx.x : blockIdx.x) * TOK;
@@ -382,6 +383,28 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
     if (warp == 0) tmem_dealloc(tm, kTmemCols);
 }
 
+// Sequences ranked by the attention work of their turn, q_len * (context seen on average), heaviest first:
+// CTAs start in block-index order, so the long sequences no longer end up as the tail of the grid.
+// One thread per sequence counts the sequences that precede it (B <= 4096: at most 16 M comparisons).
+__global__ void __launch_bounds__(256) prefill_order_kernel(const PrefillParams p) {
+    grid_dependency_wait();
+    launch_dependents();
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= p.B) return;
+    auto work = [&](int i) {
+        const long long n = p.q_indptr[i + 1] - p.q_indptr[i];
+        const long long L = p.ctx_lens[i];
+        return n * (2 * L - n);  // twice the number of (query, key) pairs under the causal mask, up to O(n)
+    };
+    const long long mine = work(b);
+    int rank = 0;
+    for (int i = 0; i < p.B; ++i) {
+        const long long w = work(i);
+        rank += (w > mine || (w == mine && i < b)) ? 1 : 0;
+    }
+    p.order[rank] = b;
+}
+
 // Multi-token append: CTA (x, b) copies tokens x, x + gridDim.x, ... of sequence b. Lengths are read
 // here and advanced by a separate tiny kernel, so no CTA sees a half-updated length.
 __global__ void __launch_bounds__(256) kv_append_tokens_kernel(const AppendTokensParams p) {
@@ -444,6 +467,10 @@ cudaError_t launch_prefill_attn(int head_dim, const CUtensorMap &tm_k, const CUt
     const int tok = kRows / p.G;
     const dim3 grid((max_q_len + tok - 1) / tok, p.Hkv, p.B);
     const size_t smem = prefill_smem_bytes(head_dim);
+    if (p.order != nullptr) {
+        const cudaError_t e = launch_pdl(prefill_order_kernel, dim3((p.B + 255) / 256), dim3(256), 0, stream, p.pdl != 0, p);
+        if (e != cudaSuccess) return e;
+    }
     if (head_dim == 128)
         return launch_pdl(prefill_attn_kernel<128>, grid, dim3(kThreads), smem, stream, p.pdl != 0, tm_k, tm_v, p);
     return launch_pdl(prefill_attn_kernel<64>, grid, dim3(kThreads), smem, stream, p.pdl != 0, tm_k, tm_v, p);
