@@ -17,11 +17,13 @@
 //   tcgen05  S = Q K^T into tensor memory (8 MMAs of 128x64x16, one thread)
 //   threads  one thread per row: load its 64 logits from tensor memory, mask,
 //            running max with a slack of 8 log2 units, exp2, row sum, P as bf16
-//            back into tensor memory; a rare correction pass rescales O
-//   tcgen05  O += P V (P from tensor memory, 4 MMAs of 128x128x16)
+//            back into tensor memory (head_dim 64: a high and a low bf16 part);
+//            a rare correction pass rescales O
+//   tcgen05  O += P V (P from tensor memory, 4 MMAs of 128x128x16; head_dim 64:
+//            4 + 4 of 128x64x16 for the two parts of P)
 // Four service warps issue the S MMAs, the O MMAs, the TMA loads of K and those
-// of V (one box per lane), so the row threads never run issue code or meet at a CTA barrier: they hand over through mbarriers (logits
-// read, probabilities written). The S MMA of block j+1 is issued as soon as
+// of V (one box per lane), so the row threads never run issue code or meet at a
+// CTA barrier: they hand over through mbarriers (logits read, probabilities written). The S MMA of block j+1 is issued as soon as
 // every row holds block j's logits in registers, and two CTAs share each SM (96 KB of shared memory, 256
 // tensor-memory columns each), so one CTA's softmax overlaps the other's MMAs. All waits are
 // bounded; a wait that runs out latches PD_ERR_TIMEOUT and the CTA unwinds and
@@ -50,6 +52,11 @@ constexpr int kTmemCols = 256;
 // Tensor-memory columns: two logit buffers of kBlock columns (block j uses buffer j % 2; its probabilities
 // overwrite the first kBlock / 2 columns of the same buffer once the logits are in registers), then the output.
 constexpr int kColS = 0, kColO = 128;
+// head_dim 64 only: the output takes 64 columns, which leaves room for the low halves of the probabilities
+// (two buffers of kBlock / 2 columns). There P = P_hi + P_lo (two bf16, ~16 significant bits) and the O product
+// is issued twice, as in the decode kernel: a 64-element output row does not average the 2^-9 rounding of a
+// single bf16 P away when a handful of tokens carry the row.
+constexpr int kColPlo = 192;
 
 __device__ __forceinline__ void latch(int32_t *status, int code, int seq, int detail) {
     if (atomicCAS(status, kDevOk, code) == kDevOk) {
@@ -173,6 +180,12 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 for (int ks = 0; ks < kBlock / 16; ++ks)  // P from the first columns of logit buffer j % 2
                     umma_ts(tm + kColO, tm + kColS + (j & 1) * kBlock + ks * 8,
                             umma_smem_desc(vst + ks * 2048, kHalfBytes, 1024), idesc, (j | ks) != 0);
+                if constexpr (kD == 64) {  // the low halves of P
+#pragma unroll
+                    for (int ks = 0; ks < kBlock / 16; ++ks)
+                        umma_ts(tm + kColO, tm + kColPlo + (j & 1) * (kBlock / 2) + ks * 8,
+                                umma_smem_desc(vst + ks * 2048, kHalfBytes, 1024), idesc, true);
+                }
                 umma_commit(bar_pv + (j & 1) * 8);
             }
             if (!ok) latch(p.status, kDevTimeout, b, blockIdx.x);
@@ -286,20 +299,47 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 alpha = fast_exp2(m_run - m_new);
                 m_run = m_new;
             }
-            uint32_t pk[kBlock / 2];
             // packed fp32x2 arithmetic: one FMA and one add per pair of logits
             const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-m_run, -m_run);
             float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+            uint32_t pk[kBlock / 2];
+            if constexpr (kD == 64) {
+                // P_hi over the first columns of the logit buffer (all logits are in registers), P_lo to its own
+                // buffer, sixteen logits at a time
+                const uint32_t plo = tm + lane_base + kColPlo + (j & 1) * (kBlock / 2);
 #pragma unroll
-            for (int c = 0; c < kBlock; c += 4) {
-                const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, nm2);
-                const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), sc2, nm2);
-                const float2 e0 = make_float2(fast_exp2(x0.x), fast_exp2(x0.y));
-                const float2 e1 = make_float2(fast_exp2(x1.x), fast_exp2(x1.y));
-                acc0 = __fadd2_rn(acc0, e0);
-                acc1 = __fadd2_rn(acc1, e1);
-                pk[c >> 1] = pack_bf16x2(e0.x, e0.y);
-                pk[(c >> 1) + 1] = pack_bf16x2(e1.x, e1.y);
+                for (int c0 = 0; c0 < kBlock; c0 += 16) {
+                    uint32_t hi[8], lo[8];
+#pragma unroll
+                    for (int c = c0; c < c0 + 16; c += 4) {
+                        const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, nm2);
+                        const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), sc2, nm2);
+                        const float2 e0 = make_float2(fast_exp2(x0.x), fast_exp2(x0.y));
+                        const float2 e1 = make_float2(fast_exp2(x1.x), fast_exp2(x1.y));
+                        acc0 = __fadd2_rn(acc0, e0);
+                        acc1 = __fadd2_rn(acc1, e1);
+                        const __nv_bfloat162 h0 = __floats2bfloat162_rn(e0.x, e0.y), h1 = __floats2bfloat162_rn(e1.x, e1.y);
+                        const int i = (c - c0) >> 1;
+                        hi[i] = *reinterpret_cast<const uint32_t *>(&h0);
+                        hi[i + 1] = *reinterpret_cast<const uint32_t *>(&h1);
+                        lo[i] = pack_bf16x2(e0.x - __low2float(h0), e0.y - __high2float(h0));
+                        lo[i + 1] = pack_bf16x2(e1.x - __low2float(h1), e1.y - __high2float(h1));
+                    }
+                    tmem_st8(buf + (c0 >> 1), hi);
+                    tmem_st8(plo + (c0 >> 1), lo);
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < kBlock; c += 4) {
+                    const float2 x0 = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, nm2);
+                    const float2 x1 = __ffma2_rn(make_float2(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), sc2, nm2);
+                    const float2 e0 = make_float2(fast_exp2(x0.x), fast_exp2(x0.y));
+                    const float2 e1 = make_float2(fast_exp2(x1.x), fast_exp2(x1.y));
+                    acc0 = __fadd2_rn(acc0, e0);
+                    acc1 = __fadd2_rn(acc1, e1);
+                    pk[c >> 1] = pack_bf16x2(e0.x, e0.y);
+                    pk[(c >> 1) + 1] = pack_bf16x2(e1.x, e1.y);
+                }
             }
             const float sum0 = acc0.x + acc0.y, sum1 = acc1.x + acc1.y;
             l_run = l_run * alpha + (sum0 + sum1);
@@ -323,7 +363,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 }
             }
 #pragma unroll
-            for (int c = 0; c < kBlock / 64; ++c) tmem_st32(buf + c * 32, *reinterpret_cast<uint32_t(*)[32]>(pk + c * 32));
+            if constexpr (kD != 64)
+                for (int c = 0; c < kBlock / 64; ++c) tmem_st32(buf + c * 32, *reinterpret_cast<uint32_t(*)[32]>(pk + c * 32));
             tmem_wait_st();
             // V rows past the context inside the last page may hold NaN; 0 * NaN is NaN, so clear them
             const int valid_rows = L - t0;

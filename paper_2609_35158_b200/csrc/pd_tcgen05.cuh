@@ -101,6 +101,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         : "memory");
 }
 
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+        : "memory");
+}
+
 // Byte offset of the 16-byte chunk `chunk` (0..7) of row `row` inside a block of 128-byte rows laid out
 // with the 128-byte swizzle (the block base must be 1024-byte aligned).
 __device__ __forceinline__ uint32_t sw128_offset(uint32_t row, uint32_t chunk) {
