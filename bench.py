@@ -659,7 +659,8 @@ def run_fit_b(args):
 # ------------------------------------------------------------------------------------------ FP8 pages
 
 def run_decode_fp8(args):
-    """The decode step over FP8 (e4m3) KV pages: pd_kv_append_fp8 + pd_decode_attn_fp8, device-resident inputs.
+    """The decode step over FP8 (e4m3) KV pages: pd_decode_step_fp8 (or, with --step separate, pd_kv_append_fp8 +
+    pd_decode_attn_fp8), device-resident inputs.
     Bytes per cached token: one byte per K and V value plus the 16-byte scale record of each (page, KV head)."""
     import torch
 
@@ -713,8 +714,12 @@ def run_decode_fp8(args):
 
     def step(i):
         nonlocal lens
-        pd.pd_kv_append_fp8(ctx, kns[i % R], vns[i % R], k8, v8, sc, cache.page_table, cache.ctx_lens)
-        pd.pd_decode_attn_fp8(ctx, qs[i % R], k8, v8, sc, cache.page_table, cache.ctx_lens, out, sm_scale=w.sm_scale)
+        if args.step == "fused":
+            pd.pd_decode_step_fp8(ctx, qs[i % R], kns[i % R], vns[i % R], k8, v8, sc, cache.page_table, cache.ctx_lens, out,
+                                  sm_scale=w.sm_scale)
+        else:
+            pd.pd_kv_append_fp8(ctx, kns[i % R], vns[i % R], k8, v8, sc, cache.page_table, cache.ctx_lens)
+            pd.pd_decode_attn_fp8(ctx, qs[i % R], k8, v8, sc, cache.page_table, cache.ctx_lens, out, sm_scale=w.sm_scale)
         lens = lens + 1
         return int(lens.sum()) * per_token + int(((lens + P - 1) // P).sum()) * per_page
 
@@ -762,7 +767,7 @@ def run_decode_fp8(args):
         "config": {**workload_config(w, lens, cfg_id), "bytes_per_cached_token": per_token + per_page / P,
                    "l2": f"KV read per step {total / K / 1e9:.2f} GB >> 126 MB L2; activations rotate over {R} buffers"},
         "seq_steps_per_s": round(B * K / (ms * 1e-3), 1), "pct_of_measured_hbm_peak": round(100 * value / peak, 2),
-        "clocks": clocks, "gpu_launches": 3 * K,
+        "clocks": clocks, "gpu_launches": (2 if args.step == "fused" else 3) * K,
         "roofline": {"bound": "hbm", "kernel": "decode_attn_split_fp8_kernel", "achieved": round(achieved, 2), "peak": peak,
                      "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}", "traffic": None,
                      "algorithmic_bytes_per_launch": int(per_launch), "avg_launch_ms": round(split_ms, 5)},
@@ -885,14 +890,17 @@ def main():
     ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--step", default="fused", choices=["separate", "fused"],
-                    help="decode: pd_kv_append + pd_decode_attn (3 launches) or pd_decode_step (2 launches)")
+    ap.add_argument("--step", default=None, choices=["separate", "fused"],
+                    help="pd_kv_append + pd_decode_attn (3 launches) or pd_decode_step (2 launches); default: fused for "
+                         "--op decode, separate for --op decode_fp8 (there the fused kernel measured slower)")
     ap.add_argument("--op", default="decode", choices=["decode", "decode_fp8", "kv_transfer", "prefill", "fit_b", "pool_toggle"],
                     help="decode = the headline decode step; kv_transfer = page gather + scatter; "
                          "prefill = one append-prefill turn; fit_b = decode step time over batch size, fitted to A + b * B; "
                          "pool_toggle = release and restore of a KV pool's physical memory; "
                          "decode_fp8 = the decode step over FP8 (e4m3) KV pages")
     args = ap.parse_args()
+    if args.step is None:
+        args.step = "separate" if args.op == "decode_fp8" else "fused"
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
     if args.impl == "cuda":

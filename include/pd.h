@@ -393,6 +393,15 @@ int pd_decode_attn_fp8(pd_ctx *ctx, const void *q, const void *k8, const void *v
                        int32_t batch, float sm_scale, int32_t split_pages, void *stream);
 
 /*
+ * pd_decode_step for FP8 pools: pd_kv_append_fp8 (advancing) followed by pd_decode_attn_fp8 in two launches,
+ * with the append inside the split kernel; pools, scale records, lengths, output and LSE are bit-identical to
+ * the two-call path. ctx_lens holds the lengths BEFORE the append on entry. Errors as pd_decode_step.
+ */
+int pd_decode_step_fp8(pd_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *k8, void *v8,
+                       float *kv_scales, const int32_t *page_table, int32_t *ctx_lens, void *out, float *lse,
+                       int32_t batch, float sm_scale, int32_t split_pages, void *stream);
+
+/*
  * pd_kv_gather / pd_kv_scatter for FP8 pools: a packed page is the K block, the V block (num_kv_heads *
  * 16 * head_dim bytes each) and the page's num_kv_heads scale records (16 bytes each), so the scales
  * travel with their page. K = 2 * num_kv_heads * head_dim + num_kv_heads bytes per token per layer.

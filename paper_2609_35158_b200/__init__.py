@@ -30,7 +30,7 @@ EXPORTS = (
     "pd_kv_gather", "pd_kv_scatter", "pd_kv_append_tokens", "pd_prefill_attn", "pd_device_status", "pd_read_worker_trace",
     "pd_makespan_coloc", "pd_makespan_disagg", "pd_feasible_disagg", "pd_decide", "pd_min_change_plan", "pd_toggle_gate",
     "pd_fit_decode_cost",
-    "pd_kv_quantize_pages", "pd_kv_append_fp8", "pd_decode_attn_fp8", "pd_kv_gather_fp8", "pd_kv_scatter_fp8",
+    "pd_kv_quantize_pages", "pd_kv_append_fp8", "pd_decode_attn_fp8", "pd_decode_step_fp8", "pd_kv_gather_fp8", "pd_kv_scatter_fp8",
     "pd_pool_create", "pd_pool_resize", "pd_pool_base", "pd_pool_capacity", "pd_pool_chunk_bytes", "pd_pool_resident_bytes",
     "pd_pool_last_error", "pd_pool_destroy",
     "pd_set_profile_events", "pd_workspace_bytes", "pd_launch_count", "pd_last_plan", "pd_status_string", "pd_last_error", "pd_version",
@@ -108,6 +108,7 @@ def _load() -> ctypes.CDLL:
     lib.pd_kv_quantize_pages.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.pd_kv_append_fp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, ctypes.c_uint32, vp]
     lib.pd_decode_attn_fp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, vp]
+    lib.pd_decode_step_fp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, f32, i32, vp]
     lib.pd_kv_gather_fp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp]
     lib.pd_kv_scatter_fp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp]
     u64 = ctypes.c_uint64
@@ -264,6 +265,14 @@ def pd_decode_attn_fp8(ctx, q, k8, v8, kv_scales, page_table, ctx_lens, out, lse
     _check(_lib.pd_decode_attn_fp8(ctx, _ptr(q), _ptr(k8), _ptr(v8), _ptr(kv_scales), _ptr(page_table), _ptr(ctx_lens),
                                    _ptr(out), _ptr(lse), batch, sm_scale, split_pages, _stream(stream)),
            "pd_decode_attn_fp8", ctx)
+
+
+def pd_decode_step_fp8(ctx, q, k_new, v_new, k8, v8, kv_scales, page_table, ctx_lens, out, lse=None, batch=None,
+                       sm_scale=1.0, split_pages=0, stream=None):
+    batch = q.shape[0] if batch is None else batch
+    _check(_lib.pd_decode_step_fp8(ctx, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k8), _ptr(v8), _ptr(kv_scales),
+                                   _ptr(page_table), _ptr(ctx_lens), _ptr(out), _ptr(lse), batch, sm_scale, split_pages,
+                                   _stream(stream)), "pd_decode_step_fp8", ctx)
 
 
 def pd_kv_gather_fp8(ctx, k8, v8, kv_scales, page_table, page_begin, page_end, packed_page_offset, packed, batch=None,

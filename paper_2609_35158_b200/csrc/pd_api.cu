@@ -520,14 +520,19 @@ int pd_kv_append_fp8(pd_ctx *ctx, const void *k_new, const void *v_new, void *k8
     return PD_OK;
 }
 
-int pd_decode_attn_fp8(pd_ctx *ctx, const void *q, const void *k8, const void *v8, const float *kv_scales,
-                       const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse, int32_t batch,
-                       float sm_scale, int32_t split_pages, void *stream) {
+}  // extern "C"
+
+namespace {
+
+int decode_attn_fp8_impl(pd_ctx *ctx, const void *q, const void *k_new, const void *v_new, const void *k8, const void *v8,
+                         const float *kv_scales, const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse,
+                         int32_t batch, float sm_scale, int32_t split_pages, void *stream) {
+    const bool fused = k_new != nullptr;
     if (int rc = check_batch(ctx, batch)) return rc;
-    if (ctx->cfg.head_dim != 128) return fail(ctx, PD_ERR_UNSUPPORTED, "pd_decode_attn_fp8: head_dim must be 128");
+    if (ctx->cfg.head_dim != 128) return fail(ctx, PD_ERR_UNSUPPORTED, "FP8 attention: head_dim must be 128");
     if (!aligned16(q) || !aligned16(k8) || !aligned16(v8) || !aligned16(kv_scales) || !aligned16(out) ||
-        page_table == nullptr || ctx_lens == nullptr)
-        return fail(ctx, PD_ERR_INVALID_ARG, "pd_decode_attn_fp8: null or misaligned pointer");
+        page_table == nullptr || ctx_lens == nullptr || (fused && (!aligned16(k_new) || !aligned16(v_new))))
+        return fail(ctx, PD_ERR_INVALID_ARG, "FP8 attention: null or misaligned pointer");
     if (!(sm_scale > 0.f) || !(sm_scale < 3.0e38f)) return fail(ctx, PD_ERR_INVALID_ARG, "sm_scale must be finite and positive");
     if (split_pages < 0) return fail(ctx, PD_ERR_INVALID_ARG, "split_pages must be >= 0");
     if (batch == 0) return PD_OK;
@@ -549,6 +554,15 @@ int pd_decode_attn_fp8(pd_ctx *ctx, const void *q, const void *k8, const void *v
     pd::AttnParams p{};
     p.q = static_cast<const __nv_bfloat16 *>(q);
     p.kv_scales = kv_scales;
+    if (fused) {
+        p.k_new = static_cast<const __nv_bfloat16 *>(k_new);
+        p.v_new = static_cast<const __nv_bfloat16 *>(v_new);
+        p.k8_w = static_cast<uint8_t *>(const_cast<void *>(k8));
+        p.v8_w = static_cast<uint8_t *>(const_cast<void *>(v8));
+        p.scales_w = const_cast<float *>(kv_scales);
+        p.ctx_lens_w = const_cast<int32_t *>(ctx_lens);
+        p.fused = 1;
+    }
     p.page_table = page_table;
     p.ctx_lens = ctx_lens;
     p.out = static_cast<__nv_bfloat16 *>(out);
@@ -586,6 +600,26 @@ int pd_decode_attn_fp8(pd_ctx *ctx, const void *q, const void *k8, const void *v
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "lse_merge launch", err);
     ctx->launches += 2;
     return PD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int pd_decode_attn_fp8(pd_ctx *ctx, const void *q, const void *k8, const void *v8, const float *kv_scales,
+                       const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse, int32_t batch,
+                       float sm_scale, int32_t split_pages, void *stream) {
+    return decode_attn_fp8_impl(ctx, q, nullptr, nullptr, k8, v8, kv_scales, page_table, ctx_lens, out, lse, batch, sm_scale,
+                                split_pages, stream);
+}
+
+int pd_decode_step_fp8(pd_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *k8, void *v8,
+                       float *kv_scales, const int32_t *page_table, int32_t *ctx_lens, void *out, float *lse,
+                       int32_t batch, float sm_scale, int32_t split_pages, void *stream) {
+    if (ctx == nullptr) return PD_ERR_INVALID_ARG;
+    if (k_new == nullptr || v_new == nullptr) return fail(ctx, PD_ERR_INVALID_ARG, "pd_decode_step_fp8: null k_new / v_new");
+    return decode_attn_fp8_impl(ctx, q, k_new, v_new, k8, v8, kv_scales, page_table, ctx_lens, out, lse, batch, sm_scale,
+                                split_pages, stream);
 }
 
 int pd_kv_append_tokens(pd_ctx *ctx, const void *k_new, const void *v_new, const int32_t *q_indptr, void *k_pages,

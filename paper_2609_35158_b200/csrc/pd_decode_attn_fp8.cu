@@ -41,7 +41,18 @@ __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) {
     return *reinterpret_cast<const uint32_t *>(&h);
 }
 
-template <int WARPS, int STAGES>
+__device__ __forceinline__ uint32_t quantize4(const float (&x)[4], float scale) {
+    // IEEE division (the build uses fast-math, so spell it out), round to nearest even, saturate: as kv_append_fp8_kernel
+    const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(x[0], scale), __fdiv_rn(x[1], scale)), __NV_SATFINITE, __NV_E4M3);
+    const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(x[2], scale), __fdiv_rn(x[3], scale)), __NV_SATFINITE, __NV_E4M3);
+    return lo | (hi << 16);
+}
+
+// FUSED: ctx_lens holds the lengths before a one-token append; the worker that reads a pair's last page
+// quantises the new token's rows exactly as kv_append_fp8_kernel does (a token that opens a page sets the
+// page's scales), writes them to the pools and patches them into the tile it is about to use; the last
+// worker to finish advances the lengths.
+template <int WARPS, int STAGES, bool FUSED>
 __global__ void __launch_bounds__(WARPS * 32, 1)
 decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                              const AttnParams p) {
@@ -59,7 +70,8 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
     uint64_t *bars = reinterpret_cast<uint64_t *>(scale_slots + WARPS * STAGES);
     Plan *plan_s = reinterpret_cast<Plan *>(bars + WARPS * STAGES * 2);
     int32_t *stage_range = reinterpret_cast<int32_t *>(plan_s + 1);
-    int32_t *warp_sums = stage_range + WARPS * STAGES;
+    int32_t *stage_pid = stage_range + WARPS * STAGES;  // physical page in a stage, -1 if its id was out of range
+    int32_t *warp_sums = stage_pid + WARPS * STAGES;
     int32_t *cum = warp_sums + 32;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -104,6 +116,7 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
     const uint32_t scale0 = smem_u32(scale_slots + warp * STAGES);
     const float4 *my_scales = scale_slots + warp * STAGES;
     int32_t *my_stage_range = stage_range + warp * STAGES;
+    int32_t *my_stage_pid = stage_pid + warp * STAGES;
     const uint64_t policy = l2_policy_evict_first();
     const int quad_row = lane >> 2;       // g: token row of the accumulators; head whose Q this lane holds as B operand
     const int quad_t = lane & 3;          // t
@@ -148,9 +161,11 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
             p_rid = rid;
         }
         int pid = page_id(pt, p, prod.b, prod.page, lane);
+        bool pid_ok = true;
         if (pid < 0 || pid >= p.num_pages) {
             if (lane == 0) latch_status(p.status, kDevBadPage, prod.b, pid);
             pid = 0;
+            pid_ok = false;
         }
         {
             // lane 0: K box, lane 1: V box, lane 2: the scale record (16 B) - one warp instruction each kind
@@ -159,6 +174,7 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
             const uint32_t bk = bar0 + p_stage * 16, bv = bk + 8;
             if (lane == 0) {
                 my_stage_range[p_stage] = p_rid;
+                if (FUSED) my_stage_pid[p_stage] = pid_ok ? pid : -1;
                 mbar_arrive_expect_tx(bk, TILE_BYTES + 16);
                 mbar_arrive_expect_tx(bv, TILE_BYTES);
             }
@@ -187,7 +203,7 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
     cons.b = 0; cons.kvh = 0; cons.page = 0; cons.np = 1;
     int c_rid = -1, c_left = 0;
     uint32_t stage = 0, parity = 0;
-    bool alive = true, seg_open = false;
+    bool alive = true, seg_open = false, seg_append = false;
     int seg_page0 = 0, L = 0;
     // Q^T as the fp16 B operand: for chunk c, head quad_row, d = 16 c + 4 t + {0, 1} and + {2, 3}
     uint32_t qb[CHUNKS][2];
@@ -205,7 +221,9 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
         if (!seg_open) {
             seg_open = true;
             seg_page0 = cons.page;
-            L = clamp_len(__ldg(p.ctx_lens + cons.b), p.MP);
+            const int L_raw = __ldg(p.ctx_lens + cons.b) + (FUSED ? 1 : 0);
+            L = clamp_len(L_raw, p.MP);
+            seg_append = FUSED && L == L_raw && L > 0;  // never patch a row of a length that was clamped
             const __nv_bfloat16 *qrow = p.q + (static_cast<size_t>(cons.b) * p.Hq + cons.kvh * G + quad_row) * D;
 #pragma unroll
             for (int c = 0; c < CHUNKS; ++c) {
@@ -229,8 +247,56 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
         const uint32_t bk = bar0 + stage * 16, bv = bk + 8;
         const int valid = L - cons.page * kPageSize;
 
+        // fused append: this lane's four values of the new K row and of the new V row (d = 4 lane .. 4 lane + 3)
+        const bool appending = FUSED && seg_append && cons.page == cons.np - 1;
+        const int new_slot = (L - 1) & (kPageSize - 1);
+        float kx[4] = {0.f, 0.f, 0.f, 0.f}, vx[4] = {0.f, 0.f, 0.f, 0.f};
+        if (appending) {
+            const size_t row = (static_cast<size_t>(cons.b) * p.Hkv + cons.kvh) * D + lane * 4;
+            const uint2 kw = __ldg(reinterpret_cast<const uint2 *>(p.k_new + row));
+            const uint2 vw = __ldg(reinterpret_cast<const uint2 *>(p.v_new + row));
+            const float2 k01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&kw.x));
+            const float2 k23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&kw.y));
+            const float2 v01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&vw.x));
+            const float2 v23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&vw.y));
+            kx[0] = k01.x; kx[1] = k01.y; kx[2] = k23.x; kx[3] = k23.y;
+            vx[0] = v01.x; vx[1] = v01.y; vx[2] = v23.x; vx[3] = v23.y;
+        }
         if (!__all_sync(0xffffffffu, mbar_wait(bk, parity))) { alive = false; break; }
-        const float4 sc = my_scales[stage];  // {k_scale, v_scale, -, -} of this page
+        float4 sc = my_scales[stage];  // {k_scale, v_scale, -, -} of this page
+        uint32_t new_v8 = 0u;
+        if (appending) {
+            if (new_slot == 0) {  // the token opens the page: it sets both scales, with a factor two of headroom
+                float ak = 0.f, av = 0.f;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float a = fabsf(kx[i]), b2 = fabsf(vx[i]);
+                    if (a > ak) ak = a;  // NaN never wins
+                    if (b2 > av) av = b2;
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    ak = fmaxf(ak, __shfl_xor_sync(0xffffffffu, ak, o));
+                    av = fmaxf(av, __shfl_xor_sync(0xffffffffu, av, o));
+                }
+                sc.x = ak > 0.f ? __fdiv_rn(ak * 2.f, 448.f) : 1.f;
+                sc.y = av > 0.f ? __fdiv_rn(av * 2.f, 448.f) : 1.f;
+            }
+            const uint32_t new_k8 = quantize4(kx, sc.x);
+            new_v8 = quantize4(vx, sc.y);
+            const int pid = my_stage_pid[stage];
+            if (pid >= 0) {  // the append itself
+                const size_t tile = static_cast<size_t>(pid) * p.Hkv + cons.kvh;
+                const size_t at = (tile * kPageSize + new_slot) * D + lane * 4;
+                *reinterpret_cast<uint32_t *>(p.k8_w + at) = new_k8;
+                *reinterpret_cast<uint32_t *>(p.v8_w + at) = new_v8;
+                if (new_slot == 0 && lane == 0) *reinterpret_cast<float4 *>(p.scales_w + tile * 4) = make_float4(sc.x, sc.y, 0.f, 0.f);
+            }
+            // the tile in shared memory still holds whatever the pool had in that slot: patch the K row now
+            const uint32_t a = kbase + new_slot * 128 + ((((lane >> 2) ^ (new_slot & 7)) << 4)) + (lane & 3) * 4;
+            asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(new_k8) : "memory");
+            __syncwarp();
+        }
 
         // S^T = K8 Q^T: one ldmatrix.x4 feeds two MMAs (two 16-byte chunks of d)
         float Se[4] = {0.f, 0.f, 0.f, 0.f}, So[4] = {0.f, 0.f, 0.f, 0.f};
@@ -279,6 +345,11 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
         const uint32_t pb1 = movmatrix_trans(*reinterpret_cast<const uint32_t *>(&h23));
 
         if (!__all_sync(0xffffffffu, mbar_wait(bv, parity))) { alive = false; break; }
+        if (appending) {
+            const uint32_t a = vbase + new_slot * 128 + ((((lane >> 2) ^ (new_slot & 7)) << 4)) + (lane & 3) * 4;
+            asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(new_v8) : "memory");
+            __syncwarp();
+        }
         if (valid < kPageSize) {
             // V rows past the context may hold NaN codes; 0 * NaN is NaN, so clear them first
             for (int row = valid; row < kPageSize; ++row)
@@ -307,7 +378,7 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
             }
         }
         __syncwarp();
-        if (valid < kPageSize) fence_proxy_async();
+        if (valid < kPageSize || appending) fence_proxy_async();  // generic-proxy stores before the next TMA write
         --inflight;
         issue_next();
         if (++stage == STAGES) { stage = 0; parity ^= 1u; }
@@ -354,11 +425,22 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
         advance(cons, cum, p.B, p.Hkv);
     }
 
+    bool last_worker = false;
     if (lane == 0) {
         if (!alive) latch_status(p.status, kDevTimeout, -1, worker);
         if (atomicAdd(p.status + kSchedDone, 1) == n_workers - 1) {  // the last worker re-arms the claim counter
             p.status[kSchedNext] = 0;
             p.status[kSchedDone] = 0;
+            last_worker = true;
+        }
+    }
+    // fused append: the last worker to finish (every CTA has long read the old lengths) advances them
+    if (FUSED && __shfl_sync(0xffffffffu, static_cast<int>(last_worker), 0)) {
+        for (int i = lane; i < p.B; i += 32) {
+            const int Lold = p.ctx_lens_w[i];
+            if (Lold < 0 || Lold + 1 > p.MP * kPageSize) continue;  // latched as a bad length by the scan
+            const int pid = __ldg(p.page_table + static_cast<size_t>(i) * p.MP + Lold / kPageSize);
+            if (pid >= 0 && pid < p.num_pages) p.ctx_lens_w[i] = Lold + 1;
         }
     }
 }
@@ -366,7 +448,7 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
 template <int WARPS, int STAGES>
 constexpr size_t fp8_smem_bytes() {
     return static_cast<size_t>(WARPS) * STAGES * (2 * kPageSize * kD8) + 1024 + WARPS * STAGES * 16 + WARPS * STAGES * 2 * 8 +
-           sizeof(Plan) + WARPS * STAGES * 4 + 32 * 4 + (kMaxBatch + 1) * 4;
+           sizeof(Plan) + 2 * WARPS * STAGES * 4 + 32 * 4 + (kMaxBatch + 1) * 4;
 }
 
 
@@ -477,27 +559,30 @@ int fp8_shape() {
     }();
     return v;
 }
-template <typename F>
+template <bool FUSED, typename F>
 cudaError_t with_fp8_kernel(F &&f) {
     switch (fp8_shape()) {
-        case 8: return f(decode_attn_split_fp8_kernel<8, 6>, fp8_smem_bytes<8, 6>(), 8);
-        case 12: return f(decode_attn_split_fp8_kernel<12, 4>, fp8_smem_bytes<12, 4>(), 12);
-        default: return f(decode_attn_split_fp8_kernel<16, 3>, fp8_smem_bytes<16, 3>(), 16);
+        case 8: return f(decode_attn_split_fp8_kernel<8, 6, FUSED>, fp8_smem_bytes<8, 6>(), 8);
+        case 12: return f(decode_attn_split_fp8_kernel<12, 4, FUSED>, fp8_smem_bytes<12, 4>(), 12);
+        default: return f(decode_attn_split_fp8_kernel<16, 3, FUSED>, fp8_smem_bytes<16, 3>(), 16);
     }
 }
 }  // namespace
 
 cudaError_t prepare_decode_attn_fp8() {
-    return with_fp8_kernel([](auto *k, size_t bytes, int) {
+    auto set = [](auto *k, size_t bytes, int) {
         return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
-    });
+    };
+    const cudaError_t e = with_fp8_kernel<false>(set);
+    return e != cudaSuccess ? e : with_fp8_kernel<true>(set);
 }
 
 cudaError_t launch_decode_attn_fp8(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, int num_ctas,
                                    cudaStream_t stream) {
-    return with_fp8_kernel([&](auto *k, size_t bytes, int warps) {
+    auto go = [&](auto *k, size_t bytes, int warps) {
         return launch_pdl(k, dim3(num_ctas), dim3(warps * 32), bytes, stream, p.pdl != 0, tm_k, tm_v, p);
-    });
+    };
+    return p.fused != 0 ? with_fp8_kernel<true>(go) : with_fp8_kernel<false>(go);
 }
 
 cudaError_t launch_kv_quantize_pages(const QuantizeParams &p, cudaStream_t stream) {

@@ -55,6 +55,8 @@ struct AttnParams {
     int32_t fused;
     // FP8 pages (null for bf16 pools): {k_scale, v_scale, 0, 0} fp32 per (page, KV head)
     const float *kv_scales;
+    uint8_t *k8_w, *v8_w;       // fused append into FP8 pools: the pools and the scale records, writable
+    float *scales_w;
     int32_t merge_rows;         // rows per CTA of the merge kernel, 0 = chosen from the row count
     unsigned long long *trace;  // optional [workers][4] ns timestamps: kernel entry, first data, last data, exit
 };
@@ -171,7 +173,7 @@ cudaError_t launch_lse_merge(int head_dim, const AttnParams &p, cudaStream_t str
 // FP8 pages (head_dim 128): the split kernel writes the same partials and plan, so launch_lse_merge follows it
 cudaError_t prepare_decode_attn_fp8();
 cudaError_t launch_decode_attn_fp8(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, int num_ctas,
-                                   cudaStream_t stream);
+                                   cudaStream_t stream);  // p.fused selects the variant that appends the new token itself
 cudaError_t launch_kv_quantize_pages(const QuantizeParams &p, cudaStream_t stream);
 cudaError_t launch_kv_append_fp8(const AppendFp8Params &p, cudaStream_t stream);
 cudaError_t prepare_prefill_attn(int head_dim);  // opt-in shared memory, once

@@ -332,3 +332,49 @@ def test_fp8_gather_scatter_bit_exact_and_attention_on_the_moved_cache():
         pd.pd_decode_attn_fp8(cd.h, q, dk, dv, ds, dst.page_table, dst.ctx_lens, out_d, sm_scale=d ** -0.5, split_pages=7)
         torch.cuda.synchronize()
         assert torch.equal(out_s.view(torch.int16), out_d.view(torch.int16))
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(32, 8), (8, 8), (16, 2)])
+@pytest.mark.parametrize("split_pages", [0, 1, 100000])
+def test_fp8_fused_step_is_bit_identical_to_append_plus_attention(Hq, Hkv, split_pages):
+    """pd_decode_step_fp8 against pd_kv_append_fp8 + pd_decode_attn_fp8 over several steps: codes, scale
+    records, lengths, output and LSE bit for bit; and against the oracle at the end."""
+    import paper_2609_35158_b200 as pd
+
+    d, steps = 128, 6
+    lens0 = np.array([0, 1, 14, 15, 16, 17, 31, 32, 33, 100, 255, 256, 700], dtype=np.int32)
+    B = len(lens0)
+    cache = wl.build_paged_cache(lens0, Hkv, d, seed=95, device=DEV, reserve_tokens=steps)
+    k8, v8, sc, _ = quantized_on_host(cache, lens0, poison_codes=True)
+    sc[np.isnan(sc)] = 7.0  # pages that are not in use yet: any finite garbage
+    a = to_dev(k8, v8, sc)
+    b = to_dev(k8, v8, sc)
+    lens_a, lens_b = cache.ctx_lens.clone(), cache.ctx_lens.clone()
+    lens_h = lens0.copy()  # the oracle's own copy of the cache, appended to on the host
+    scale = d ** -0.5
+    with Ctx(Hq, Hkv, d, B, cache.page_table.shape[1], cache.k_pages.shape[0]) as ctx:
+        for t in range(steps):
+            q = wl.random_bf16((B, Hq, d), 960 + 3 * t, DEV)
+            kn = wl.random_bf16((B, Hkv, d), 961 + 3 * t, DEV) * (1.0 + 0.5 * t)
+            vn = wl.random_bf16((B, Hkv, d), 962 + 3 * t, DEV)
+            assert oracle.fp8_kv_append(oracle.bf16_bits(kn), oracle.bf16_bits(vn), k8, v8, sc, cache.page_table_host, lens_h) == B
+            out_a = torch.full((B, Hq, d), float("nan"), dtype=torch.bfloat16, device=DEV)
+            lse_a = torch.full((B, Hq), float("nan"), dtype=torch.float32, device=DEV)
+            out_b, lse_b = out_a.clone(), lse_a.clone()
+            pd.pd_kv_append_fp8(ctx.h, kn, vn, a[0], a[1], a[2], cache.page_table, lens_a)
+            pd.pd_decode_attn_fp8(ctx.h, q, a[0], a[1], a[2], cache.page_table, lens_a, out_a, lse_a, sm_scale=scale,
+                                  split_pages=split_pages)
+            pd.pd_decode_step_fp8(ctx.h, q, kn, vn, b[0], b[1], b[2], cache.page_table, lens_b, out_b, lse_b,
+                                  sm_scale=scale, split_pages=split_pages)
+            torch.cuda.synchronize()
+            assert pd.pd_device_status(ctx.h)[0] == 0
+            what = f"step {t}"
+            assert lens_b.cpu().tolist() == (lens0 + t + 1).tolist() and torch.equal(lens_a, lens_b), what
+            assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]), what + ": codes"
+            assert torch.equal(a[2].view(torch.int32), b[2].view(torch.int32)), what + ": scale records"
+            assert torch.equal(out_a.view(torch.int16), out_b.view(torch.int16)), what + ": output"
+            assert torch.equal(lse_a.view(torch.int32), lse_b.view(torch.int32)), what + ": lse"
+    assert np.array_equal(b[0].cpu().numpy(), k8) and np.array_equal(b[1].cpu().numpy(), v8)
+    assert np.array_equal(b[2].cpu().numpy().view(np.uint32), sc.view(np.uint32)) and np.array_equal(lens_h, lens0 + steps)
+    ref, _ = oracle.fp8_decode_attn(oracle.bf16_bits(q), k8, v8, sc, cache.page_table_host, lens_h, scale)
+    assert_parity(out_b, ref, "fused FP8 step", scale_abs_by_magnitude=True)
