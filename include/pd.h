@@ -296,6 +296,23 @@ int pd_last_plan(pd_ctx *ctx, void *stream, int64_t *total_units, int32_t *pages
                  int32_t *num_ranges, int32_t *num_workers);
 
 /*
+ * The decode kernels' work decomposition, run on the host (no device needed; the same functions the
+ * kernels execute). Units are (sequence, KV head, page) triples in that nesting order.
+ * pd_plan_ranges: the plan for `total_units` units and `n_workers` worker warps under the given
+ * parameters (split_pages as in pd_decode_attn; max_ranges, min_pages, halving_levels, tail_pages as a
+ * context holds them: 16 * workers, 4, 6, 16 by default). *n_ranges receives the number of ranges;
+ * range r covers units [starts[r], starts[r] + lens[r]). capacity = 0 only counts.
+ * pd_plan_walk: the triples of `count` consecutive units from `first_unit`, given the exclusive prefix
+ * sums of pages per sequence (cum_pages, batch + 1 entries): how a worker finds the start of a range and
+ * steps through it.
+ */
+int pd_plan_ranges(int64_t total_units, int32_t n_workers, int32_t split_pages, int32_t max_ranges,
+                   int32_t min_pages, int32_t halving_levels, int32_t tail_pages, int64_t *starts, int32_t *lens,
+                   int32_t capacity, int32_t *n_ranges);
+int pd_plan_walk(const int32_t *cum_pages, int32_t batch, int32_t num_kv_heads, int64_t first_unit,
+                 int32_t count, int32_t *seq, int32_t *kv_head, int32_t *page);
+
+/*
  * ---- PD decision engine (host-only, no CUDA): the paper's makespan models and plan arithmetic.
  * The decode-side inputs b and K are quantities this library measures: b is the slope of the decode
  * step time over the number of concurrent sequences (pd_fit_decode_cost on timings of pd_decode_attn),

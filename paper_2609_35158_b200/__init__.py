@@ -29,7 +29,7 @@ EXPORTS = (
     "pd_create", "pd_destroy", "pd_kv_append", "pd_decode_attn", "pd_decode_attn_static", "pd_decode_step", "pd_decode_step_host",
     "pd_kv_gather", "pd_kv_scatter", "pd_kv_append_tokens", "pd_prefill_attn", "pd_device_status", "pd_read_worker_trace",
     "pd_makespan_coloc", "pd_makespan_disagg", "pd_feasible_disagg", "pd_decide", "pd_min_change_plan", "pd_toggle_gate",
-    "pd_fit_decode_cost",
+    "pd_fit_decode_cost", "pd_plan_ranges", "pd_plan_walk",
     "pd_kv_quantize_pages", "pd_kv_append_fp8", "pd_decode_attn_fp8", "pd_decode_step_fp8", "pd_kv_gather_fp8", "pd_kv_scatter_fp8",
     "pd_pool_create", "pd_pool_resize", "pd_pool_base", "pd_pool_capacity", "pd_pool_chunk_bytes", "pd_pool_resident_bytes",
     "pd_pool_last_error", "pd_pool_destroy",
@@ -99,6 +99,8 @@ def _load() -> ctypes.CDLL:
     lib.pd_decide.argtypes = [pm, i32, pt, dbl, dbl, pt]
     lib.pd_min_change_plan.argtypes = [vp, vp, vp, i32, vp, i32, vp, ctypes.POINTER(i32), ctypes.POINTER(i32)]
     lib.pd_toggle_gate.argtypes = [dbl, dbl, dbl, dbl, dbl]
+    lib.pd_plan_ranges.argtypes = [i64, i32, i32, i32, i32, i32, i32, vp, vp, i32, ctypes.POINTER(i32)]
+    lib.pd_plan_walk.argtypes = [vp, i32, i32, i64, i32, vp, vp, vp]
     lib.pd_fit_decode_cost.argtypes = [vp, vp, i32, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
     lib.pd_status_string.argtypes = [ctypes.c_int]
     lib.pd_status_string.restype = ctypes.c_char_p
@@ -441,6 +443,32 @@ def pd_min_change_plan(cur_active, cur_role, dst_active, dst_role_count):
 
 def pd_toggle_gate(R, B, T_ded, T_full, T_toggle) -> bool:
     return bool(_lib.pd_toggle_gate(R, B, T_ded, T_full, T_toggle))
+
+
+def pd_plan_ranges(total_units, n_workers, split_pages=0, max_ranges=None, min_pages=4, halving_levels=6, tail_pages=16):
+    """(starts int64 [n], lens int32 [n]) of the decode kernels' plan, computed on the host."""
+    import numpy as np
+
+    max_ranges = 16 * n_workers if max_ranges is None else max_ranges
+    n = ctypes.c_int32(0)
+    _check(_lib.pd_plan_ranges(total_units, n_workers, split_pages, max_ranges, min_pages, halving_levels, tail_pages,
+                               None, None, 0, ctypes.byref(n)), "pd_plan_ranges")
+    starts = np.zeros(n.value, dtype=np.int64)
+    lens = np.zeros(n.value, dtype=np.int32)
+    _check(_lib.pd_plan_ranges(total_units, n_workers, split_pages, max_ranges, min_pages, halving_levels, tail_pages,
+                               starts.ctypes.data, lens.ctypes.data, n.value, ctypes.byref(n)), "pd_plan_ranges")
+    return starts, lens
+
+
+def pd_plan_walk(cum_pages, num_kv_heads, first_unit, count):
+    """(seq, kv_head, page) int32 arrays of `count` consecutive units starting at `first_unit`."""
+    import numpy as np
+
+    cum = np.ascontiguousarray(cum_pages, dtype=np.int32)
+    out = [np.zeros(count, dtype=np.int32) for _ in range(3)]
+    _check(_lib.pd_plan_walk(cum.ctypes.data, len(cum) - 1, num_kv_heads, first_unit, count, out[0].ctypes.data,
+                             out[1].ctypes.data, out[2].ctypes.data), "pd_plan_walk")
+    return tuple(out)
 
 
 def pd_fit_decode_cost(concurrency, step_seconds):

@@ -7,6 +7,7 @@
 #include <cstring>
 #include <new>
 
+#include "pd_decode_plan.cuh"
 #include "pd_kernels.cuh"
 
 namespace {
@@ -768,6 +769,50 @@ int pd_device_status(pd_ctx *ctx, void *stream, int32_t *code, int32_t *seq, int
     if (seq != nullptr) *seq = rc == PD_OK ? -1 : host[1];
     if (detail != nullptr) *detail = rc == PD_OK ? 0 : host[2];
     return rc;
+}
+
+int pd_plan_ranges(int64_t total_units, int32_t n_workers, int32_t split_pages, int32_t max_ranges, int32_t min_pages,
+                   int32_t halving_levels, int32_t tail_pages, int64_t *starts, int32_t *lens, int32_t capacity,
+                   int32_t *n_ranges) {
+    if (n_ranges == nullptr || total_units < 0 || n_workers < 1 || split_pages < 0 || max_ranges < 1 || min_pages < 1 ||
+        halving_levels < 0 || halving_levels > pd::kMaxLevels - 2 || tail_pages < 1 || capacity < 0 ||
+        (capacity > 0 && (starts == nullptr || lens == nullptr)))
+        return PD_ERR_INVALID_ARG;
+    pd::AttnParams p{};
+    p.split_pages = split_pages;
+    p.max_ranges = max_ranges;
+    p.min_pages_auto = min_pages;
+    p.halving_levels = halving_levels;
+    p.tail_pages = tail_pages;
+    pd::Plan pl;
+    pd::make_plan(pl, total_units, n_workers, p);  // the function the kernels run
+    *n_ranges = pl.n_ranges;
+    if (pl.n_ranges > capacity) return capacity == 0 ? PD_OK : PD_ERR_WORKSPACE;
+    for (int r = 0; r < pl.n_ranges; ++r) {
+        long long start;
+        int len;
+        pd::range_bounds(pl, r, start, len);
+        starts[r] = start;
+        lens[r] = len;
+    }
+    return PD_OK;
+}
+
+int pd_plan_walk(const int32_t *cum_pages, int32_t batch, int32_t num_kv_heads, int64_t first_unit, int32_t count,
+                 int32_t *seq, int32_t *kv_head, int32_t *page) {
+    if (cum_pages == nullptr || batch < 1 || num_kv_heads < 1 || first_unit < 0 || count < 0 ||
+        (count > 0 && (seq == nullptr || kv_head == nullptr || page == nullptr)))
+        return PD_ERR_INVALID_ARG;
+    if (first_unit + count > static_cast<int64_t>(num_kv_heads) * cum_pages[batch]) return PD_ERR_INVALID_ARG;
+    if (count == 0) return PD_OK;
+    pd::Cursor c = pd::locate(cum_pages, batch, num_kv_heads, first_unit);
+    for (int i = 0; i < count; ++i) {
+        seq[i] = c.b;
+        kv_head[i] = c.kvh;
+        page[i] = c.page;
+        pd::advance(c, cum_pages, batch, num_kv_heads);
+    }
+    return PD_OK;
 }
 
 int pd_set_profile_events(pd_ctx *ctx, void *before, void *after) {

@@ -80,7 +80,7 @@ __device__ void scan_pages(const AttnParams &p, int32_t *cum, int32_t *warp_sums
 
 // The plan is a pure function of (total, workers, parameters): every CTA and the
 // merge kernel's reader derive the same one.
-__device__ void make_plan(Plan &pl, long long total, int n_workers, const AttnParams &p) {
+__host__ __device__ inline void make_plan(Plan &pl, long long total, int n_workers, const AttnParams &p) {
     pl.total = total;
     int nl = 0, first = 0;
     long long pos = 0;
@@ -119,14 +119,14 @@ __device__ void make_plan(Plan &pl, long long total, int n_workers, const AttnPa
     pl.n_ranges = first;
 }
 
-__device__ __forceinline__ void range_bounds(const Plan &pl, int rid, long long &start, int &len) {
+__host__ __device__ __forceinline__ void range_bounds(const Plan &pl, int rid, long long &start, int &len) {
     int l = 0;
     while (l + 1 < pl.n_levels && rid >= pl.lv[l + 1].first) ++l;
     start = pl.lv[l].start + static_cast<long long>(rid - pl.lv[l].first) * pl.lv[l].size;
     len = static_cast<int>(min(static_cast<long long>(pl.lv[l].size), pl.lv[l + 1].start - start));
 }
 
-__device__ __forceinline__ Cursor locate(const int32_t *cum, int B, int Hkv, long long x) {
+__host__ __device__ __forceinline__ Cursor locate(const int32_t *cum, int B, int Hkv, long long x) {
     const int y = static_cast<int>(x / Hkv);  // largest b with cum[b] <= y owns unit x
     int lo = 0, hi = B - 1;
     while (lo < hi) {
@@ -142,7 +142,7 @@ __device__ __forceinline__ Cursor locate(const int32_t *cum, int B, int Hkv, lon
     return c;
 }
 
-__device__ __forceinline__ void advance(Cursor &c, const int32_t *cum, int B, int Hkv) {
+__host__ __device__ __forceinline__ void advance(Cursor &c, const int32_t *cum, int B, int Hkv) {
     if (++c.page >= c.np) {
         c.page = 0;
         if (++c.kvh == Hkv) {
