@@ -146,3 +146,12 @@ def test_reference_arm_prints_the_contract_line():
     assert r["cpu_baseline"]["kind"] == "oracle" and r["cpu_baseline"]["value"] == r["value"] and r["cpu_baseline"]["cores"] >= 1
     assert r["e2e"] == {"value": r["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert "workload" in r["config"] and r["data"] == "synthetic"
+
+
+def test_header_is_plain_c99_and_cxx():
+    """include/pd.h must be usable from C and from C++ without any CUDA header."""
+    hdr = os.path.join(ROOT, "include", "pd.h")
+    for cmd in (["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c", hdr],
+                ["g++", "-std=c++17", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", hdr]):
+        res = subprocess.run(cmd, capture_output=True, text=True)
+        assert res.returncode == 0, res.stderr
