@@ -103,7 +103,7 @@ def test_small_ragged_poisoned(Hq, Hkv, d, split_pages):
     assert plan["total_units"] == total
     # the plan the device used is the one the host-side function gives for the same inputs
     _starts, host_lens = ctx.pd.pd_plan_ranges(total, plan["num_workers"], split_pages)
-    assert len(host_lens) == plan["num_ranges"] and int(host_lens[0]) == plan["pages_per_range"]
+    assert len(host_lens) == plan["num_ranges"] and int(host_lens[0]) == min(plan["pages_per_range"], total)
     if split_pages:
         assert plan["pages_per_range"] >= split_pages
         assert plan["num_ranges"] == -(-total // plan["pages_per_range"])
