@@ -22,12 +22,21 @@ def bits(x):
 def test_e4m3_decode_matches_the_format_definition_and_torch():
     codes = np.arange(256, dtype=np.uint8)
     got = oracle.e4m3_to_f64(codes)
-    # OCP 8-bit floating point, E4M3: bias 7, subnormals m/8 * 2^-6, S.1111.111 is NaN, no infinities
-    spec = {0x00: 0.0, 0x01: 2.0 ** -9, 0x07: 7 * 2.0 ** -9, 0x08: 2.0 ** -6, 0x38: 1.0, 0x3C: 1.5, 0x40: 2.0,
-            0x77: 240.0, 0x7E: 448.0, 0xB8: -1.0, 0xFE: -448.0}
-    for c, v in spec.items():
-        assert got[c] == v
-    assert math.isnan(got[0x7F]) and math.isnan(got[0xFF])
+    # the format's own values (tests/golden/e4m3_codes.txt: bias 7, subnormals m/8 * 2^-6, S.1111.111 is NaN)
+    import os
+
+    n_checked = 0
+    for line in open(os.path.join(os.path.dirname(__file__), "golden", "e4m3_codes.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        code, value = line.split()
+        c, v = int(code, 16), float(value)
+        if math.isnan(v):
+            assert math.isnan(got[c])
+        else:
+            assert got[c] == v and math.copysign(1.0, got[c]) == math.copysign(1.0, v)
+        n_checked += 1
+    assert n_checked == 19
     ref = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).to(torch.float64).numpy()
     finite = ~np.isnan(ref)
     assert finite.sum() == 254 and np.array_equal(got[finite], ref[finite])
