@@ -350,10 +350,14 @@ int32_t pd_feasible_disagg(const pd_cost_model *m, int32_t N_P, int32_t N_D);
 /*
  * Online decision (Sec. 4.3.2): enumerates N_P in [1, N_k - 1] over the feasible splits, compares the
  * best with colocation and returns the configuration of minimal predicted makespan. With `current` set,
- * mode-dependent hysteresis applies: the switch is taken only if the relative gain over the current
- * configuration exceeds ratio_threshold (same mode) or mode_threshold (colocation <-> disaggregation);
- * a current configuration that is infeasible or sized for another N_k forces the switch. The paper
- * publishes no threshold values; they are parameters.
+ * mode-dependent hysteresis applies: an alternative is admitted only if its predicted makespan is lower
+ * than the current one by more than threshold x current makespan (strictly), the threshold being
+ * ratio_threshold for another ratio of the current mode and mode_threshold for a colocation <->
+ * disaggregation switch; the best admitted alternative is returned (a refused mode switch does not block a
+ * ratio adjustment that clears ratio_threshold), else `current` with its makespan. A current
+ * configuration that is infeasible or sized for another N_k forces the switch to the overall minimum.
+ * The paper publishes no threshold values and does not say whether the gain is absolute or relative;
+ * they are parameters and the gain is relative here.
  */
 int pd_decide(const pd_cost_model *m, int32_t N_k, const pd_target *current, double ratio_threshold,
               double mode_threshold, pd_target *out);

@@ -36,7 +36,15 @@ def feasible_disagg(m: dict, N_P: int, N_D: int) -> bool:
 
 
 def decide(m: dict, N_k: int, current=None, ratio_threshold=0.0, mode_threshold=0.0):
-    """Sec. 4.3.2. Configurations are (N_P, N_D, N_C) tuples; returns (configuration, predicted makespan)."""
+    """Sec. 4.3.2. Configurations are (N_P, N_D, N_C) tuples; returns (configuration, predicted makespan).
+
+    Without a current configuration: the argmin over colocation and every feasible split. With one that is
+    still realisable, hysteresis: an alternative is admitted only if its predicted makespan is lower than the
+    current one by more than a threshold, taken here as a fraction of the current makespan, strictly;
+    alternatives in the other mode (colocation <-> disaggregation) answer to ``mode_threshold``, other ratios
+    of the same mode to ``ratio_threshold``. Every alternative is judged by its own threshold and the best
+    admitted one wins, so a refused mode switch does not block a ratio adjustment that clears the smaller
+    threshold. A current configuration that cannot be kept forces the switch to the argmin."""
     cands = [((0, 0, N_k), makespan_coloc(m, N_k))]
     for n_p in range(1, N_k):
         if feasible_disagg(m, n_p, N_k - n_p):
@@ -53,12 +61,15 @@ def decide(m: dict, N_k: int, current=None, ratio_threshold=0.0, mode_threshold=
     if not cur_ok:
         return best, t_best  # forced switch: the current topology cannot be kept
     t_cur = makespan_coloc(m, N_k) if cur_coloc else makespan_disagg(m, current[0], current[1])[0]
-    if tuple(current) == best:
-        return best, t_cur
-    threshold = mode_threshold if (best[2] > 0) != cur_coloc else ratio_threshold
-    if t_cur - t_best > threshold * t_cur:
-        return best, t_best
-    return tuple(current), t_cur
+    choice, t_choice = tuple(current), t_cur
+    for c, t in cands:  # same order as above, so ties between admitted alternatives resolve the same way
+        if c == tuple(current):
+            continue
+        threshold = mode_threshold if (c[2] > 0) != cur_coloc else ratio_threshold
+        admitted = t_cur - t > threshold * t_cur
+        if admitted and t < t_choice:
+            choice, t_choice = c, t
+    return choice, t_choice
 
 
 def change_counts(cur_active, cur_role, dst_active, dst_role_count):

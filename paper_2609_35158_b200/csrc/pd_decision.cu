@@ -70,15 +70,23 @@ int pd_decide(const pd_cost_model *m, int32_t N_k, const pd_target *current, dou
                                                        : pd_feasible_disagg(m, current->N_P, current->N_D) != 0);
     if (!cur_ok) return PD_OK;
     const double t_cur = cur_coloc ? pd_makespan_coloc(m, N_k) : pd_makespan_disagg(m, current->N_P, current->N_D, nullptr, nullptr);
-    const bool same = best.N_P == current->N_P && best.N_D == current->N_D && best.N_C == current->N_C;
-    if (same) {
-        out->makespan = t_cur;
-        return PD_OK;
+    // Hysteresis: an alternative is admitted only if it beats the current makespan by more than its threshold
+    // (a fraction of the current makespan, strictly) -- mode_threshold for a colocation <-> disaggregation
+    // switch, ratio_threshold for another ratio of the same mode. The best admitted alternative wins, so a
+    // refused mode switch does not block a ratio adjustment that clears the smaller threshold.
+    pd_target choice{current->N_P, current->N_D, current->N_C, t_cur};
+    auto consider = [&](const pd_target &c) {
+        if (c.N_P == current->N_P && c.N_D == current->N_D && c.N_C == current->N_C) return;
+        const double threshold = ((c.N_C > 0) != cur_coloc) ? mode_threshold : ratio_threshold;
+        if (t_cur - c.makespan > threshold * t_cur && c.makespan < choice.makespan) choice = c;
+    };
+    consider(pd_target{0, 0, N_k, pd_makespan_coloc(m, N_k)});
+    for (int32_t np = 1; np <= N_k - 1; ++np) {
+        const int32_t nd = N_k - np;
+        if (!pd_feasible_disagg(m, np, nd)) continue;
+        consider(pd_target{np, nd, 0, pd_makespan_disagg(m, np, nd, nullptr, nullptr)});
     }
-    // hysteresis: the relative gain must exceed the threshold, a larger one for a colocation <-> disaggregation switch
-    const bool mode_switch = (best.N_C > 0) != cur_coloc;
-    const double threshold = mode_switch ? mode_threshold : ratio_threshold;
-    if (!(t_cur - best.makespan > threshold * t_cur)) *out = pd_target{current->N_P, current->N_D, current->N_C, t_cur};
+    *out = choice;
     return PD_OK;
 }
 

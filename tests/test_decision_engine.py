@@ -60,30 +60,95 @@ def test_feasibility_constraints():
     assert [od.feasible_disagg(m, n_p, 8) for n_p in (3, 4)] == [False, True]
 
 
-def test_decide_is_the_argmin_and_hysteresis_holds_small_gains():
-    m = model(A=0.005, b=2e-3, t_prefill=4e-5, H_max_bytes=100e9)
-    N = 12
-    cfg, t = od.decide(m, N)
+def enumerate_candidates(m, N):
     cands = {(0, 0, N): od.makespan_coloc(m, N)}
     for n_p in range(1, N):
         if od.feasible_disagg(m, n_p, N - n_p):
             cands[(n_p, N - n_p, 0)] = od.makespan_disagg(m, n_p, N - n_p)[0]
+    return cands
+
+
+def test_decide_is_the_argmin_and_forced_switches_ignore_thresholds():
+    m = model(A=0.005, b=2e-3, t_prefill=4e-5, H_max_bytes=100e9)
+    N = 12
+    cfg, t = od.decide(m, N)
+    cands = enumerate_candidates(m, N)
     assert t == min(cands.values()) and cands[cfg] == t
-    # a neighbouring ratio: taken without hysteresis, refused when the gain is below the threshold
-    if cfg[2] == 0:
-        near = (cfg[0] + 1, cfg[1] - 1, 0)
-        gain = (cands[near] - t) / cands[near]
-        assert od.decide(m, N, current=near, ratio_threshold=0.0)[0] == cfg
-        assert od.decide(m, N, current=near, ratio_threshold=gain * 1.01)[0] == near
-        assert od.decide(m, N, current=near, ratio_threshold=gain * 0.99)[0] == cfg
-        # mode switches use the other threshold
-        coloc = (0, 0, N)
-        g2 = (cands[coloc] - t) / cands[coloc]
-        assert od.decide(m, N, current=coloc, ratio_threshold=10.0, mode_threshold=g2 * 0.99)[0] == cfg
-        assert od.decide(m, N, current=coloc, ratio_threshold=0.0, mode_threshold=g2 * 1.01)[0] == coloc
     # a current configuration that no longer fits forces the switch whatever the thresholds
     assert od.decide(m, N, current=(1, 1, 0), ratio_threshold=10.0, mode_threshold=10.0)[0] == cfg
     assert od.decide(m, N, current=(N - 1, 1, 0), ratio_threshold=10.0, mode_threshold=10.0)[0] == cfg  # KV does not fit
+
+
+# Two hand-evaluated six-worker models for the hysteresis of Sec. 4.3.2 (theta = 0, A = 0, no transfer, no
+# environment time, one turn): per turn the prefill work is B dL t_prefill = 6 worker-seconds and the decode work
+# r b B = 60 worker-seconds, so Eq. 1 gives 6/6 + 60/6 + T_over = 11 + T_over and Eq. 2-3 give
+# max(6 / N_P, 60 / N_D): (1,5) -> 12, (2,4) -> 15, (3,3) -> 20, (4,2) -> 30, (5,1) -> 60.
+HAND = dict(B=60.0, S=1.0, r=100.0, dL=100.0, theta=0.0, A=0.0, b=0.01, t_prefill=0.001, T_env=0.0, K_bytes=0.0, BW=1.0,
+            K_seq_bytes=0.0, H_max_bytes=1.0)
+DISAGG_WINS = dict(HAND, T_over=5.0)   # colocation 16: the argmin is (1, 5, 0) at 12
+COLOC_WINS = dict(HAND, T_over=0.0)    # colocation 11: the argmin is colocation
+
+
+def hysteresis_cases():
+    """(model, current, ratio_threshold, mode_threshold, expected configuration, expected makespan)."""
+    D, C = model(**DISAGG_WINS), model(**COLOC_WINS)
+    return [
+        # ratio move inside disaggregation: (2,4) at 15 -> (1,5) at 12, relative gain 3/15 = 0.2;
+        # the (large) mode threshold must play no part
+        (D, (2, 4, 0), 0.19, 0.9, (1, 5, 0), 12.0),
+        (D, (2, 4, 0), 0.21, 0.9, (2, 4, 0), 15.0),
+        # colocation -> disaggregation: 16 -> 12, gain 4/16 = 0.25; the ratio threshold must play no part
+        (D, (0, 0, 6), 0.9, 0.24, (1, 5, 0), 12.0),
+        (D, (0, 0, 6), 0.0, 0.26, (0, 0, 6), 16.0),
+        # disaggregation -> colocation: (1,5) at 12 -> 11, gain 1/12 = 0.0833
+        (C, (1, 5, 0), 0.9, 0.08, (0, 0, 6), 11.0),
+        (C, (1, 5, 0), 0.0, 0.09, (1, 5, 0), 12.0),
+        # the best alternative is a refused mode switch (colocation 11 from (3,3) at 20: gain 0.45 < 0.5) while
+        # a ratio of the same mode clears its own threshold ((1,5) at 12: gain 0.4 > 0.1): the ratio move is taken
+        (C, (3, 3, 0), 0.1, 0.5, (1, 5, 0), 12.0),
+        (C, (3, 3, 0), 0.1, 0.44, (0, 0, 6), 11.0),
+        (C, (3, 3, 0), 0.41, 0.5, (3, 3, 0), 20.0),
+        # among admitted ratios the best one wins, not the nearest: from (4,2) at 30 both (3,3) and (1,5) clear 0.3
+        (C, (4, 2, 0), 0.3, 0.9, (1, 5, 0), 12.0),
+    ]
+
+
+def test_hand_models_have_the_intended_minima():
+    D, C = model(**DISAGG_WINS), model(**COLOC_WINS)
+    want = {(1, 5, 0): 12.0, (2, 4, 0): 15.0, (3, 3, 0): 20.0, (4, 2, 0): 30.0, (5, 1, 0): 60.0}
+    for m, coloc in ((D, 16.0), (C, 11.0)):
+        cands = enumerate_candidates(m, 6)
+        assert cands.pop((0, 0, 6)) == pytest.approx(coloc, rel=1e-14)
+        assert set(cands) == set(want)
+        for c, t in want.items():
+            assert cands[c] == pytest.approx(t, rel=1e-14)
+    cfg, t = od.decide(D, 6)
+    assert cfg == (1, 5, 0) and cfg[2] == 0 and t == pytest.approx(12.0, rel=1e-14)   # disaggregated argmin
+    cfg, t = od.decide(C, 6)
+    assert cfg == (0, 0, 6) and t == pytest.approx(11.0, rel=1e-14)                   # colocated argmin
+
+
+def test_mode_dependent_hysteresis_hand_cases():
+    for m, cur, rt, mt, want_cfg, want_t in hysteresis_cases():
+        cfg, t = od.decide(m, 6, current=cur, ratio_threshold=rt, mode_threshold=mt)
+        assert cfg == want_cfg, (cur, rt, mt, cfg)
+        assert t == pytest.approx(want_t, rel=1e-14)
+
+
+# Two workers, every quantity a power of two, so the comparison at the threshold is exact in binary:
+# colocation = 8192/2 * 2^-10 + 64 * (2^-6 * 64 / 2) + 92 = 4 + 32 + 92 = 128, (1,1) = max(8, 64) = 64, gain exactly 1/2.
+EXACT = dict(B=64.0, S=1.0, r=64.0, dL=128.0, theta=0.0, A=0.0, b=2.0 ** -6, t_prefill=2.0 ** -10, T_over=92.0, T_env=0.0,
+             K_bytes=0.0, BW=1.0, K_seq_bytes=0.0, H_max_bytes=1.0)
+
+
+def test_hysteresis_is_strict_at_the_threshold():
+    m = model(**EXACT)
+    assert od.makespan_coloc(m, 2) == 128.0 and od.makespan_disagg(m, 1, 1)[0] == 64.0
+    assert od.decide(m, 2, current=(0, 0, 2), mode_threshold=0.5) == ((0, 0, 2), 128.0)      # gain == threshold: stay
+    assert od.decide(m, 2, current=(0, 0, 2), mode_threshold=0.4375) == ((1, 1, 0), 64.0)
+    # relative, not absolute: an absolute reading of 0.4375 s would also pass, one of 60 s would too (64 > 60),
+    # while 60 as a fraction of the current makespan can never be exceeded
+    assert od.decide(m, 2, current=(0, 0, 2), mode_threshold=60.0)[0] == (0, 0, 2)
 
 
 def test_change_counts_match_brute_force_minimum():
@@ -142,6 +207,19 @@ def test_c_functions_match_the_oracle():
         assert (got_t.N_P, got_t.N_D, got_t.N_C) == want_cfg
         assert got_t.makespan == pytest.approx(want_t, rel=1e-13)
     assert math.isnan(pd.pd_makespan_coloc(c_model(model(B=-1.0)), 4))
+
+
+def test_c_decide_hand_cases():
+    import paper_2609_35158_b200 as pd
+
+    for m, cur, rt, mt, want_cfg, want_t in hysteresis_cases():
+        got = pd.pd_decide(c_model(m), 6, pd.pd_target(*cur, 0.0), rt, mt)
+        assert (got.N_P, got.N_D, got.N_C) == want_cfg, (cur, rt, mt)
+        assert got.makespan == pytest.approx(want_t, rel=1e-14)
+    cm = c_model(model(**EXACT))
+    for mt, want in ((0.5, (0, 0, 2)), (0.4375, (1, 1, 0)), (60.0, (0, 0, 2))):
+        got = pd.pd_decide(cm, 2, pd.pd_target(0, 0, 2, 0.0), 0.0, mt)
+        assert (got.N_P, got.N_D, got.N_C) == want
 
 
 def test_c_min_change_plan_is_valid_and_minimal():
