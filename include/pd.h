@@ -218,19 +218,22 @@ int pd_kv_scatter(pd_ctx *ctx, const void *packed, const int64_t *packed_page_of
  * KV-cache pool, a plugin that lives inside another framework's memory budget,
  * a process whose allocator is frozen after warm-up. pd_create calls cudaMalloc
  * and is therefore closed to them; this function needs no context. It computes
- * exactly what pd_decode_attn computes with split_pages = 0, with the kernels'
- * scratch (fp32 partials, page prefix sums, plan and status words) held in a
- * fixed 16 MiB array inside the library image. Every device that loads the
+ * what pd_decode_attn computes, within the same tolerances (the ranges are one
+ * level of equal size, one per worker warp, so that the number of partials is
+ * known in advance; the summation order and hence the last bits differ), with
+ * the kernels' scratch (fp32 partials, page prefix sums, plan and status words)
+ * held in a fixed 16 MiB array inside the library image. Every device that loads the
  * library carries that array until the process exits. The function calls no
  * cudaMalloc, cudaFree or allocating library routine.
  *
  * Geometry comes from *cfg (num_q_heads, num_kv_heads, head_dim, page_size,
  * max_pages_per_seq, num_pages, device; max_batch and flags are ignored); the
  * tensors are the caller's, as for pd_decode_attn. Limit: the partials must fit
- * the fixed array, i.e. roughly (SM count * 8 + batch * num_kv_heads) *
- * group * (head_dim * 4 + 8) bytes <= 16 MiB - on a 148-SM device about
- * batch <= 350 at 32/8 heads, head_dim 128. Larger batches return
- * PD_ERR_WORKSPACE and launch nothing.
+ * the fixed array, i.e. (SM count * 8 + batch * num_kv_heads) * group *
+ * (head_dim * 4 + 8) bytes plus 4 * (batch + 1) bytes of prefix sums and about
+ * 1.5 KB of rounding and control words <= 16 MiB - on a 148-SM device batch <=
+ * 860 at 32/8 heads and head_dim 128, batch <= 712 at 32/4 heads. Larger
+ * batches return PD_ERR_WORKSPACE and launch nothing.
  *
  * The first call on each device resolves the array's device address and sets
  * the kernel's shared-memory attribute; make that first call outside any CUDA
@@ -238,9 +241,11 @@ int pd_kv_scatter(pd_ctx *ctx, const void *packed, const int64_t *packed_page_of
  * previous call's contents (the function itself clears the few words that must
  * start at zero: the status latch and the range-claim counters): two calls whose kernels may overlap on
  * the GPU - different streams, or concurrent host threads - race on it. Issue
- * them on one stream or order them with events. Out-of-range page ids are
- * clamped to page 0 as in pd_decode_attn but are not reported, since there is
- * no context to query.
+ * them on one stream or order them with events. There is no context to query,
+ * so nothing a kernel latches is reported: an out-of-range page id is clamped
+ * to page 0, a length outside [0, max_pages_per_seq * page_size] is clamped to
+ * that interval, and rows whose worker gave up a bounded wait stay unwritten,
+ * all silently. Callers that need those reports use pd_decode_attn.
  */
 int pd_decode_attn_static(const pd_config *cfg, const void *q, const void *k_pages, const void *v_pages,
                           const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse,

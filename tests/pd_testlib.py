@@ -23,15 +23,22 @@ def error_metrics(out_gpu_bf16: torch.Tensor, out_ref: np.ndarray):
     return max_abs, float(rel.max()) if rel.size else 0.0
 
 
-def assert_parity(out_gpu_bf16, out_ref, what="", scale_abs_by_magnitude=False):
-    """``scale_abs_by_magnitude``: the absolute bound becomes 1e-2 * max(1, |ref|) per element. bf16 cannot
-    hold a value of magnitude 4 to better than 1.6e-2, so outputs that are single V rows (contexts of a
-    handful of tokens, as the first queries of a prefill see) need the bound to follow the magnitude."""
+def assert_parity(out_gpu_bf16, out_ref, what="", scale_abs_by_magnitude=False, scale_abs_above=None):
+    """Max abs error <= 1e-2 over all elements and per-row relative L2 <= 5e-3 for every row.
+
+    bf16 holds a value of magnitude in [4, 8) only to 1.6e-2 (half a unit in the last place), in [2, 4) to
+    7.8e-3: an output that is nearly a single V row (a context of a handful of tokens) can exceed a flat 1e-2
+    by rounding alone. Two widenings exist for such elements, never for the relative bound:
+    ``scale_abs_above=2.0`` (decode and the fused step): 1e-2 wherever |ref| <= 2, 1e-2 * |ref| / 2 beyond,
+    i.e. the flat bound wherever bf16 can meet it with margin and 5e-3 relative elsewhere;
+    ``scale_abs_by_magnitude`` (prefill, whose single bf16 P adds 2^-9 relative per probability, and FP8):
+    1e-2 * max(1, |ref|)."""
     assert torch.isfinite(out_gpu_bf16.float()).all(), f"{what}: non-finite output"
     max_abs, rel = error_metrics(out_gpu_bf16, out_ref)
-    if scale_abs_by_magnitude:
+    if scale_abs_by_magnitude or scale_abs_above is not None:
+        knee = 1.0 if scale_abs_by_magnitude else float(scale_abs_above)
         got = out_gpu_bf16.detach().float().cpu().numpy().astype(np.float64)
-        max_abs = float((np.abs(got - out_ref) / np.maximum(1.0, np.abs(out_ref))).max())
+        max_abs = float((np.abs(got - out_ref) / np.maximum(1.0, np.abs(out_ref) / knee)).max()) if got.size else 0.0
     assert max_abs <= MAX_ABS_TOL, f"{what}: max abs error {max_abs:.3e} > {MAX_ABS_TOL}"
     assert rel <= REL_L2_TOL, f"{what}: per-row relative L2 {rel:.3e} > {REL_L2_TOL}"
     return max_abs, rel

@@ -61,8 +61,8 @@ def step_both_ways(lens, Hq, Hkv, d, seed, split_pages, steps=1, sm_scale=None, 
             assert torch.equal(lse_a.view(torch.int32), lse_b.view(torch.int32)), what + ": lse"
             if check_oracle and (t == 0 or t == steps - 1):
                 ref, ref_lse = oracle_on_cache(q, b, lens + t + 1, sm_scale)
-                assert_parity(out_b, ref, what, scale_abs_by_magnitude=True)
-                assert np.allclose(lse_b.cpu().numpy(), ref_lse, atol=2e-3, rtol=0), what
+                assert_parity(out_b, ref, what, scale_abs_above=2.0)
+                np.testing.assert_allclose(lse_b.cpu().numpy(), ref_lse, rtol=2e-5, atol=2e-5, err_msg=what)
     return b
 
 
@@ -94,6 +94,8 @@ def test_config0_step():
 
 
 def test_full_size_config1_step_equals_two_call_path():
+    """Bit-identity only: the two-call path at this size is checked against the oracle, every row, by
+    test_gpu_parity.py::test_full_size_configs_all_rows, and identical bits need no second comparison."""
     w = wl.WORKLOADS[1]
     lens = wl.context_lengths(1)
     step_both_ways(lens, w.num_q_heads, w.num_kv_heads, w.head_dim, seed=15, split_pages=0, steps=2,
@@ -139,7 +141,7 @@ def test_no_room_or_bad_page_is_reported_and_leaves_the_cache_alone():
         assert torch.equal(bits(cache.k_pages), bits(twin.k_pages))
         assert torch.equal(bits(cache.v_pages), bits(twin.v_pages))
         ref, _ = oracle_on_cache(q, cache, np.array([16, 6, 41]), 0.125, seq_ids=[1, 2])
-        assert_parity(out[1:], ref, "sequences beside the faulty one", scale_abs_by_magnitude=True)
+        assert_parity(out[1:], ref, "sequences beside the faulty one", scale_abs_above=2.0)
 
     # a table row that is full: the length is reported, nothing is written
     lens = np.array([32, 7], dtype=np.int32)

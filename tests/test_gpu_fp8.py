@@ -94,7 +94,7 @@ def test_fp8_attention_small_ragged_poisoned(Hq, Hkv, split_pages):
     # outputs here are ~0.02 in magnitude: compare relative to the output scale
     live = lens > 0
     assert_parity((out[torch.from_numpy(live).to(DEV)].float() * 50).to(torch.bfloat16), ref[live] * 50,
-                  f"{Hq}/{Hkv} split {split_pages}", scale_abs_by_magnitude=True)
+                  f"{Hq}/{Hkv} split {split_pages}", scale_abs_above=2.0)
     got_lse = lse.cpu().numpy()
     assert np.all(np.isneginf(got_lse[~live])) and np.all(out[torch.from_numpy(~live).to(DEV)].float().cpu().numpy() == 0)
     np.testing.assert_allclose(got_lse[live], ref_lse[live], rtol=3e-5, atol=3e-5)
@@ -157,7 +157,7 @@ def test_fp8_append_bit_exact_then_attend():
         torch.cuda.synchronize()
         assert pd.pd_device_status(ctx.h)[0] == 0
     ref, _ = oracle.fp8_decode_attn(oracle.bf16_bits(q), k8, v8, sc, cache.page_table_host, lens, d ** -0.5)
-    assert_parity(out, ref, "after 20 FP8 appends", scale_abs_by_magnitude=True)
+    assert_parity(out, ref, "after 20 FP8 appends", scale_abs_above=2.0)
 
 
 def test_fp8_append_errors_are_reported_and_skipped():
@@ -192,7 +192,10 @@ def test_fp8_attention_needs_head_dim_128():
 
 
 @pytest.mark.parametrize("config", [1, 3])
-def test_fp8_full_size_config_sampled_sequences(config):
+def test_fp8_full_size_config_all_rows(config):
+    """Configs 1 and 3 at full size in the automatic split mode: every (sequence, query head) row against the
+    FP8 oracle, whose inputs are the ORACLE's own quantisation of the same bf16 cache (the GPU quantiser's codes
+    and scale bits are checked against it on the way, page by page)."""
     import paper_2609_35158_b200 as pd
 
     w = wl.WORKLOADS[config]
@@ -206,32 +209,34 @@ def test_fp8_full_size_config_sampled_sequences(config):
     tip = tokens_in_page(cache, lens)
     q = wl.random_bf16((B, w.num_q_heads, w.head_dim), 87, DEV)
     out = torch.empty_like(q)
+    lse = torch.empty((B, w.num_q_heads), dtype=torch.float32, device=DEV)
     with Ctx(w.num_q_heads, w.num_kv_heads, w.head_dim, B, cache.page_table.shape[1], NP) as ctx:
-        # the GPU quantiser prepares the cache (it is bit-identical to the oracle's, checked on the sample below)
         pd.pd_kv_quantize_pages(ctx.h, cache.k_pages, cache.v_pages, torch.from_numpy(tip).to(DEV), k8d, v8d, scd)
-        pd.pd_decode_attn_fp8(ctx.h, q, k8d, v8d, scd, cache.page_table, cache.ctx_lens, out, sm_scale=w.sm_scale)
+        pd.pd_decode_attn_fp8(ctx.h, q, k8d, v8d, scd, cache.page_table, cache.ctx_lens, out, lse, sm_scale=w.sm_scale)
         torch.cuda.synchronize()
         assert pd.pd_device_status(ctx.h)[0] == 0
-    sample = sorted({int(np.argmin(lens)), int(np.argmax(lens)), 0, B - 1})
-    # oracle inputs come from the oracle: quantise the sampled sequences' pages on the host
-    pages = np.concatenate([cache.page_table_host[b, :(int(lens[b]) + P - 1) // P] for b in sample])
-    idx = torch.from_numpy(pages.astype(np.int64)).to(DEV)
-    kb = oracle.bf16_bits(cache.k_pages.index_select(0, idx))
-    vb = oracle.bf16_bits(cache.v_pages.index_select(0, idx))
-    k8, v8, sc = oracle.fp8_quantize_pages(kb, vb, tip[pages])
-    assert np.array_equal(k8d.index_select(0, idx).cpu().numpy(), k8)
-    assert np.array_equal(scd.index_select(0, idx).cpu().numpy().view(np.uint32), sc.view(np.uint32))
-    table = np.full((len(sample), cache.page_table.shape[1]), -1, dtype=np.int32)
-    cur = 0
-    for i, b in enumerate(sample):
-        n = (int(lens[b]) + P - 1) // P
-        table[i, :n] = np.arange(cur, cur + n)
-        cur += n
-    qs = oracle.bf16_bits(q[torch.tensor(sample, device=DEV)])
-    ref, _ = oracle.fp8_decode_attn(qs, k8, v8, sc, table, lens[sample], w.sm_scale)
-    # long contexts average unit-variance values to outputs of ~0.02: compare at that scale
-    assert_parity((out[torch.tensor(sample, device=DEV)].float() * 32).to(torch.bfloat16), ref * 32,
-                  f"config {config}", scale_abs_by_magnitude=True)
+    worst = [0.0, 0.0]
+    for c0 in range(0, B, 16):  # 16 sequences at a time keeps the host copies small
+        ids = list(range(c0, min(B, c0 + 16)))
+        pages = np.concatenate([cache.page_table_host[b, :(int(lens[b]) + P - 1) // P] for b in ids])
+        idx = torch.from_numpy(pages.astype(np.int64)).to(DEV)
+        kb = oracle.bf16_bits(cache.k_pages.index_select(0, idx))
+        vb = oracle.bf16_bits(cache.v_pages.index_select(0, idx))
+        k8, v8, sc = oracle.fp8_quantize_pages(kb, vb, tip[pages])
+        assert np.array_equal(k8d.index_select(0, idx).cpu().numpy(), k8)
+        assert np.array_equal(v8d.index_select(0, idx).cpu().numpy(), v8)
+        assert np.array_equal(scd.index_select(0, idx).cpu().numpy().view(np.uint32), sc.view(np.uint32))
+        table = np.full((len(ids), cache.page_table.shape[1]), -1, dtype=np.int32)
+        cur = 0
+        for i, b in enumerate(ids):
+            n = (int(lens[b]) + P - 1) // P
+            table[i, :n] = np.arange(cur, cur + n)
+            cur += n
+        ref, ref_lse = oracle.fp8_decode_attn(oracle.bf16_bits(q[c0:c0 + len(ids)]), k8, v8, sc, table, lens[ids], w.sm_scale)
+        m_abs, m_rel = assert_parity(out[c0:c0 + len(ids)], ref, f"config {config} sequences {c0}..")
+        np.testing.assert_allclose(lse[c0:c0 + len(ids)].cpu().numpy(), ref_lse, rtol=3e-5, atol=3e-5)
+        worst = [max(worst[0], m_abs), max(worst[1], m_rel)]
+    print(f"FP8 config {config}: worst max_abs {worst[0]:.2e} rel_l2 {worst[1]:.2e}")
 
 
 @pytest.mark.parametrize("seed", range(12))
@@ -377,4 +382,4 @@ def test_fp8_fused_step_is_bit_identical_to_append_plus_attention(Hq, Hkv, split
     assert np.array_equal(b[0].cpu().numpy(), k8) and np.array_equal(b[1].cpu().numpy(), v8)
     assert np.array_equal(b[2].cpu().numpy().view(np.uint32), sc.view(np.uint32)) and np.array_equal(lens_h, lens0 + steps)
     ref, _ = oracle.fp8_decode_attn(oracle.bf16_bits(q), k8, v8, sc, cache.page_table_host, lens_h, scale)
-    assert_parity(out_b, ref, "fused FP8 step", scale_abs_by_magnitude=True)
+    assert_parity(out_b, ref, "fused FP8 step", scale_abs_above=2.0)

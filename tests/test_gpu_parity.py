@@ -357,54 +357,112 @@ def test_full_size_configs_all_rows(config):
     print(f"config {config}: max_abs {max_abs:.2e} rel_l2 {rel:.2e} plan {plan}")
 
 
-@pytest.mark.parametrize("fused", [False, True])
-def test_config4_multiturn_loop_with_page_allocation(fused):
-    """Config 4 at full batch: 128 steps of (allocate, append, attend) with the host free list in the
-    loop, as two calls and as the fused step the benchmark times. Every append is checked on the slot it
-    must fill; attention is checked against the oracle on steps 0, 1, 63, 126 and 127 for a sample of
-    sequences that holds the shortest, the longest and several that open a new page during the loop."""
+def _compact_host_mirror(cache, lens, seq_ids, extra_pages):
+    """Host copy of the pages the given sequences own, renumbered 0, 1, 2, ... with `extra_pages` fresh
+    (NaN-filled) pages of room behind each sequence, and the table that goes with it."""
+    P = wl.PAGE_SIZE
+    n_pages = [(int(lens[b]) + P - 1) // P for b in seq_ids]
+    table = np.full((len(seq_ids), max(n_pages) + extra_pages), -1, dtype=np.int32)
+    src, cur = [], 0
+    for i, (b, n) in enumerate(zip(seq_ids, n_pages)):
+        table[i, :n + extra_pages] = np.arange(cur, cur + n + extra_pages)
+        src.append((cur, cache.page_table_host[b, :n].astype(np.int64)))
+        cur += n + extra_pages
+    shape = (cur,) + tuple(cache.k_pages.shape[1:])
+    k = np.full(shape, wl.NAN_BF16_BITS, dtype=np.uint16)
+    v = np.full(shape, wl.NAN_BF16_BITS, dtype=np.uint16)
+    for (start, phys) in src:
+        idx = torch.from_numpy(phys).to(cache.k_pages.device)
+        k[start:start + len(phys)] = oracle.bf16_bits(cache.k_pages.index_select(0, idx))
+        v[start:start + len(phys)] = oracle.bf16_bits(cache.v_pages.index_select(0, idx))
+    return k, v, table
+
+
+def test_config4_multiturn_loop_with_page_allocation():
+    """Config 4 at full batch: 128 steps of (allocate, append, attend) with the host free list in the loop,
+    run in both forms side by side on two caches: pd_kv_append + pd_decode_attn on one, the fused
+    pd_decode_step (what the benchmark times) on the other, every output of every step compared bit for bit.
+    Against the oracle: the whole batch (all 512 sequences, every row) on steps 0, 1, 63, 126 and 127, and 16
+    fixed sequences (shortest, longest, page openers, page fillers) on all 128 steps. The 16 live in a host
+    mirror that the ORACLE's append grows from the same k_new / v_new, so their check covers the GPU append
+    and the attention together; at the end the mirror must equal the device pages byte for byte."""
     w = wl.WORKLOADS[4]
     lens0 = wl.context_lengths(4)
-    B, steps = w.batch, 128
-    check_steps = (0, 1, 63, 126, 127)
-    cache = wl.build_paged_cache(lens0, w.num_kv_heads, w.head_dim, seed=4, device=DEV, reserve_tokens=steps,
-                                 preassign_reserve=False, poison=False)
-    alloc = wl.PageAllocator(cache)
+    B, steps, P = w.batch, 128, wl.PAGE_SIZE
+    full_steps = (0, 1, 63, 126, 127)
+    caches = [wl.build_paged_cache(lens0, w.num_kv_heads, w.head_dim, seed=4, device=DEV, reserve_tokens=steps,
+                                   preassign_reserve=False, poison=False) for _ in range(2)]
+    allocs = [wl.PageAllocator(c) for c in caches]
     lens = lens0.copy()
-    sample = sorted(set([int(np.argmin(lens0)), int(np.argmax(lens0))] + list(range(6))))
+    by_slot = lambda r: [int(b) for b in np.nonzero(lens0 % P == r)[0][:3]]
+    sample = [int(np.argmin(lens0)), int(np.argmax(lens0))] + by_slot(0) + by_slot(15) + by_slot(1)
+    sample = sorted(set(sample))
+    sample += [b for b in range(B) if b not in sample][:16 - len(sample)]
+    sample = sorted(sample)
+    assert len(sample) == 16
+    sample_dev = torch.tensor(sample, device=DEV)
+    mk, mv, mtable = _compact_host_mirror(caches[0], lens0, sample, extra_pages=steps // P + 1)
+    mlens = lens0[sample].astype(np.int32).copy()
     ar = torch.arange(B, device=DEV)
     allocated = 0
-    with ctx_for(cache, w.num_q_heads) as ctx:
+    worst = [0.0, 0.0]
+    with ctx_for(caches[0], w.num_q_heads) as ctx_a, ctx_for(caches[1], w.num_q_heads) as ctx_b:
+        pd = ctx_a.pd
         for step in range(steps):
-            need, logical, phys = alloc.assign(lens)
+            for cache, alloc in zip(caches, allocs):
+                need, logical, phys = alloc.assign(lens)
+                if len(need):
+                    cache.page_table[torch.from_numpy(need).to(DEV), torch.from_numpy(logical).to(DEV)] = \
+                        torch.from_numpy(phys).to(DEV)
             allocated += len(need)
-            if len(need):
-                cache.page_table[torch.from_numpy(need).to(DEV), torch.from_numpy(logical).to(DEV)] = \
-                    torch.from_numpy(phys).to(DEV)
+            assert np.array_equal(caches[0].page_table_host, caches[1].page_table_host)
             q = wl.random_bf16((B, w.num_q_heads, w.head_dim), 4000 + step, DEV)
             kn = wl.random_bf16((B, w.num_kv_heads, w.head_dim), 5000 + step, DEV)
             vn = wl.random_bf16((B, w.num_kv_heads, w.head_dim), 6000 + step, DEV)
-            out = torch.empty((B, w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=DEV)
-            if fused:
-                ctx.pd.pd_decode_step(ctx.h, q, kn, vn, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens,
-                                      out, sm_scale=w.sm_scale)
-            else:
-                ctx.pd.pd_kv_append(ctx.h, kn, vn, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens)
-                ctx.pd.pd_decode_attn(ctx.h, q, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, out,
-                                      sm_scale=w.sm_scale)
-            # append: the slot of every sequence holds exactly the new rows
+            out_a = torch.empty((B, w.num_q_heads, w.head_dim), dtype=torch.bfloat16, device=DEV)
+            out_b = torch.empty_like(out_a)
+            a, b = caches
+            pd.pd_kv_append(ctx_a.h, kn, vn, a.k_pages, a.v_pages, a.page_table, a.ctx_lens)
+            pd.pd_decode_attn(ctx_a.h, q, a.k_pages, a.v_pages, a.page_table, a.ctx_lens, out_a, sm_scale=w.sm_scale)
+            pd.pd_decode_step(ctx_b.h, q, kn, vn, b.k_pages, b.v_pages, b.page_table, b.ctx_lens, out_b,
+                              sm_scale=w.sm_scale)
+            assert torch.equal(out_a.view(torch.int16), out_b.view(torch.int16)), f"step {step}: fused != two calls"
+            # append: the slot of every sequence holds exactly the new rows, in both caches
             pos = torch.from_numpy(lens.astype(np.int64)).to(DEV)
-            page = cache.page_table[ar, pos // 16].long()
-            assert torch.equal(cache.k_pages[page, :, pos % 16], kn)
-            assert torch.equal(cache.v_pages[page, :, pos % 16], vn)
+            for cache in caches:
+                page = cache.page_table[ar, pos // P].long()
+                assert torch.equal(cache.k_pages[page, :, pos % P], kn)
+                assert torch.equal(cache.v_pages[page, :, pos % P], vn)
             lens = lens + 1
-            if step in check_steps:
-                assert ctx.pd.pd_device_status(ctx.h)[0] == 0
-                assert np.array_equal(cache.ctx_lens.cpu().numpy(), lens)
-                ref, _ = oracle_on_cache(q, cache, lens, w.sm_scale, seq_ids=sample)
-                assert_parity(out[sample], ref, f"config 4 step {step}")
-        assert ctx.pd.pd_device_status(ctx.h)[0] == 0
+            # the 16 fixed sequences, every step: oracle append + oracle attention on the host mirror
+            assert oracle.kv_append(oracle.bf16_bits(kn[sample_dev]), oracle.bf16_bits(vn[sample_dev]), mk, mv, mtable,
+                                    mlens) == 0
+            ref, _ = oracle.decode_attn(oracle.bf16_bits(q[sample_dev]), mk, mv, mtable, mlens, w.sm_scale)
+            m_abs, m_rel = assert_parity(out_b[sample_dev], ref, f"config 4 step {step}, 16 fixed sequences")
+            worst = [max(worst[0], m_abs), max(worst[1], m_rel)]
+            if step in full_steps:
+                assert pd.pd_device_status(ctx_a.h)[0] == 0 and pd.pd_device_status(ctx_b.h)[0] == 0
+                assert np.array_equal(a.ctx_lens.cpu().numpy(), lens) and np.array_equal(b.ctx_lens.cpu().numpy(), lens)
+                for c0 in range(0, B, 64):  # the whole batch, 64 sequences (about 3 GB of pages) at a time
+                    ids = list(range(c0, min(B, c0 + 64)))
+                    ref, _ = oracle_on_cache(q, b, lens, w.sm_scale, seq_ids=ids)
+                    m_abs, m_rel = assert_parity(out_b[c0:c0 + len(ids)], ref, f"config 4 step {step}, sequences {c0}..")
+                    worst = [max(worst[0], m_abs), max(worst[1], m_rel)]
+        assert pd.pd_device_status(ctx_a.h)[0] == 0 and pd.pd_device_status(ctx_b.h)[0] == 0
+    assert torch.equal(caches[0].k_pages.view(torch.int16), caches[1].k_pages.view(torch.int16))
+    assert torch.equal(caches[0].v_pages.view(torch.int16), caches[1].v_pages.view(torch.int16))
+    # the mirror the oracle grew equals the device pages of those sequences, byte for byte
+    for i, bseq in enumerate(sample):
+        n = (int(lens[bseq]) + P - 1) // P
+        idx = torch.from_numpy(caches[1].page_table_host[bseq, :n].astype(np.int64)).to(DEV)
+        dk, dv = oracle.bf16_bits(caches[1].k_pages.index_select(0, idx)), oracle.bf16_bits(caches[1].v_pages.index_select(0, idx))
+        full, tail = int(lens[bseq]) // P, int(lens[bseq]) % P
+        hk, hv = mk[mtable[i, :n]], mv[mtable[i, :n]]
+        assert np.array_equal(dk[:full], hk[:full]) and np.array_equal(dv[:full], hv[:full])
+        if tail:
+            assert np.array_equal(dk[full, :, :tail], hk[full, :, :tail]) and np.array_equal(dv[full, :, :tail], hv[full, :, :tail])
     assert allocated >= B * (steps // 16)  # every sequence crossed page boundaries during the loop
+    print(f"config 4: worst max_abs {worst[0]:.2e} rel_l2 {worst[1]:.2e}")
 
 
 def test_maximum_batch_with_empty_and_tiny_contexts():

@@ -46,7 +46,7 @@ def test_decode_random_case(seed):
         assert ctx.pd.pd_device_status(ctx.h)[0] == 0
     ref, ref_lse = oracle_on_cache(q, cache, lens, scale)
     what = f"seed {seed}: B={B} {Hq}/{Hkv} d={d} split={split} lens={lens.tolist()}"
-    assert_parity(out, ref, what, scale_abs_by_magnitude=True)
+    assert_parity(out, ref, what, scale_abs_above=2.0)
     got_lse = lse.cpu().numpy()
     empty = lens == 0
     assert np.all(np.isneginf(got_lse[empty])) and np.all(out[torch.from_numpy(empty).to(DEV)].float().cpu().numpy() == 0)
