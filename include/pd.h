@@ -252,38 +252,13 @@ int pd_decode_attn_static(const pd_config *cfg, const void *q, const void *k_pag
                           int32_t batch, float sm_scale, void *stream);
 
 /*
- * Waits for `stream`, then reports and clears the first fault a kernel of this
- * context latched since the last call: *code is PD_OK, PD_ERR_DEVICE_FAULT or
+ * Waits for `stream` (pass the stream the context's kernels were issued on, so
+ * that the report covers them), then reports and clears the first fault a kernel
+ * of this context latched since the last call: *code is PD_OK, PD_ERR_DEVICE_FAULT or
  * PD_ERR_TIMEOUT; *seq the sequence index (or -1); *detail the offending page
  * id / position. Any of the three output pointers may be NULL. Returns *code.
  */
 int pd_device_status(pd_ctx *ctx, void *stream, int32_t *code, int32_t *seq, int32_t *detail);
-
-/*
- * Timing hook for benchmarks: the NEXT pd_decode_attn of this context records
- * `before` on its stream just ahead of the split kernel and `after` right behind
- * it (both cudaEvent_t passed as void*, owned by the caller, who must keep them
- * alive until the work has run), then the hook clears itself. That call launches
- * its kernels without programmatic overlap, so the events bracket the split
- * kernel alone, not the merge. Two event records cost several microseconds of
- * stream time: hook a sample of the steps, not all of them. Passing two NULLs
- * cancels a pending hook.
- */
-int pd_set_profile_events(pd_ctx *ctx, void *before, void *after);
-
-/*
- * Per-worker timestamps of the most recent pd_decode_attn, for profiling the
- * start-up and tail of the split kernel. Available only when the environment
- * variable PD_TRACE_WORKERS=1 was set at pd_create (otherwise
- * PD_ERR_UNSUPPORTED). Waits for `stream`, then copies up to max_workers
- * records of four uint64 nanosecond values (%globaltimer: kernel entry, first
- * tile landed, last tile landed, exit) to host_out (HOST pointer) and stores
- * the number of records in *num_workers. After a pd_prefill_attn the same
- * buffer holds, per CTA (in launch order) and as four consecutive records, the
- * SM-clock cycles row thread 0 spent waiting for S, loading S, in the softmax
- * arithmetic, waiting for O, storing P, in total, and its block count.
- */
-int pd_read_worker_trace(pd_ctx *ctx, void *stream, uint64_t *host_out, int32_t max_workers, int32_t *num_workers);
 
 /* Bytes of device workspace the context holds. */
 int pd_workspace_bytes(const pd_ctx *ctx, size_t *bytes);

@@ -373,7 +373,7 @@ def pd_set_profile_events(ctx, before=None, after=None) -> None:
 
 
 def pd_read_worker_trace(ctx, max_workers=4096, stream=None):
-    """uint64 array [workers, 4] of ns timestamps (needs PD_TRACE_WORKERS=1 at pd_create)."""
+    """uint64 array [workers, 4] of ns timestamps (needs a PD_ENABLE_TUNING build and PD_TRACE_WORKERS=1 at pd_create)."""
     import numpy as np
 
     buf = np.zeros((max_workers, 4), dtype=np.uint64)

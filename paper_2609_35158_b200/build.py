@@ -17,7 +17,8 @@ NVCC_FLAGS = [
 
 def _inputs():
     files = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh"))]
-    files.append(os.path.join(os.path.dirname(_HERE), "include", "pd.h"))
+    inc = os.path.join(os.path.dirname(_HERE), "include")
+    files += [os.path.join(inc, f) for f in os.listdir(inc) if f.endswith(".h")]
     return files
 
 

@@ -1,6 +1,7 @@
 // C ABI of the paged decode-attention library: context, argument checks,
 // tensor-map encoding and kernel launches. See include/pd.h for the contract.
 #include "../../include/pd.h"
+#include "../../include/pd_debug.h"
 
 #include <cstdio>
 #include <cstdlib>
@@ -44,6 +45,7 @@ struct pd_ctx {
     int tail_pages = 16;
     int pdl = 1;
     int merge_rows = 0;
+    int prefill_reverse = 1, prefill_order = 1;
     size_t slots = 0;
     // device workspace (one allocation)
     void *workspace = nullptr;
@@ -53,7 +55,7 @@ struct pd_ctx {
     int32_t *cum_pages = nullptr;
     int32_t *plan = nullptr;
     int32_t *status = nullptr;
-    unsigned long long *trace = nullptr;  // per-worker timestamps, only with PD_TRACE_WORKERS=1
+    unsigned long long *trace = nullptr;  // per-worker timestamps, only in a PD_ENABLE_TUNING build with PD_TRACE_WORKERS=1
     int trace_workers = 0;
     // staging for pd_decode_step_host
     __nv_bfloat16 *stage_q = nullptr, *stage_k = nullptr, *stage_v = nullptr, *stage_out = nullptr;
@@ -85,10 +87,16 @@ int fail(pd_ctx *ctx, int code, const char *what, cudaError_t err = cudaSuccess)
 
 bool aligned16(const void *p) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int env_int(const char *name, int fallback) {
+// Kernel shape and plan parameters are fixed in the shipped build. A build with -DPD_ENABLE_TUNING reads them
+// from the environment once, at pd_create, for experiments; no call after pd_create looks at the environment.
+#ifdef PD_ENABLE_TUNING
+int tune_int(const char *name, int fallback) {
     const char *v = std::getenv(name);
     return (v != nullptr && *v != '\0') ? std::atoi(v) : fallback;
 }
+#else
+constexpr int tune_int(const char *, int fallback) { return fallback; }
+#endif
 
 // 2-D view of a pool: rows = (page, KV head, slot), columns = head_dim bf16.
 // Box = 16 rows x 64 columns (128 B) with the 128-byte swizzle.
@@ -185,16 +193,18 @@ int pd_create(const pd_config *cfg, pd_ctx **out) {
     // kernel shape: one CTA per SM, each warp an independent worker with its own stage ring
     pd::AttnVariant v{};
     v.head_dim = cfg->head_dim;
-    v.warps = env_int("PD_TUNE_WARPS", 8);
-    v.stages = env_int("PD_TUNE_STAGES", cfg->head_dim == 128 ? 3 : 6);
-    v.hilo = env_int("PD_TUNE_HILO", 1);
+    v.warps = tune_int("PD_TUNE_WARPS", 8);
+    v.stages = tune_int("PD_TUNE_STAGES", cfg->head_dim == 128 ? 3 : 6);
+    v.hilo = tune_int("PD_TUNE_HILO", 1);
     ctx->variant = v;
-    ctx->num_ctas = ctx->num_sms * env_int("PD_TUNE_CTAS_PER_SM", 1);
-    ctx->min_pages_auto = env_int("PD_TUNE_MIN_PAGES", 4);
-    ctx->halving_levels = env_int("PD_TUNE_LEVELS", 6);
-    ctx->tail_pages = env_int("PD_TUNE_TAIL", 16);
-    ctx->pdl = env_int("PD_TUNE_PDL", 1);
-    ctx->merge_rows = env_int("PD_TUNE_MERGE_ROWS", 0);
+    ctx->num_ctas = ctx->num_sms * tune_int("PD_TUNE_CTAS_PER_SM", 1);
+    ctx->min_pages_auto = tune_int("PD_TUNE_MIN_PAGES", 4);
+    ctx->halving_levels = tune_int("PD_TUNE_LEVELS", 6);
+    ctx->tail_pages = tune_int("PD_TUNE_TAIL", 16);
+    ctx->pdl = tune_int("PD_TUNE_PDL", 1);
+    ctx->merge_rows = tune_int("PD_TUNE_MERGE_ROWS", 0);
+    ctx->prefill_reverse = tune_int("PD_TUNE_PREFILL_REVERSE", 1);
+    ctx->prefill_order = tune_int("PD_TUNE_PREFILL_ORDER", 1);
     if (ctx->halving_levels < 0 || ctx->halving_levels > pd::kMaxLevels - 2 || ctx->tail_pages < 1) {
         delete ctx;
         return PD_ERR_INVALID_ARG;
@@ -226,7 +236,7 @@ int pd_create(const pd_config *cfg, pd_ctx **out) {
     const size_t b_status = round256(pd::kStatusWords * sizeof(int32_t));
     const size_t b_q = round256(static_cast<size_t>(cfg->max_batch) * cfg->num_q_heads * cfg->head_dim * 2);
     const size_t b_kv = round256(static_cast<size_t>(cfg->max_batch) * cfg->num_kv_heads * cfg->head_dim * 2);
-    const size_t b_trace = env_int("PD_TRACE_WORKERS", 0) ? round256(static_cast<size_t>(n_workers) * 4 * 8) : 0;
+    const size_t b_trace = tune_int("PD_TRACE_WORKERS", 0) ? round256(static_cast<size_t>(n_workers) * 4 * 8) : 0;
     ctx->workspace_bytes = b_part_o + b_part_ml + b_cum + b_plan + b_status + 2 * b_q + 2 * b_kv + b_trace;
     err = cudaMalloc(&ctx->workspace, ctx->workspace_bytes);
     if (err != cudaSuccess) {
@@ -698,8 +708,8 @@ int pd_prefill_attn(pd_ctx *ctx, const void *q, const int32_t *q_indptr, const v
     p.pdl = ctx->pdl;
     p.trace = ctx->trace;                    // the worker-trace buffer doubles as [CTA][16] phase counters
     p.trace_ctas = ctx->trace_workers / 4;
-    p.reverse_tiles = env_int("PD_TUNE_PREFILL_REVERSE", 1);
-    p.order = env_int("PD_TUNE_PREFILL_ORDER", 1) ? ctx->cum_pages : nullptr;  // the decode kernels' prefix-sum buffer is free here
+    p.reverse_tiles = ctx->prefill_reverse;
+    p.order = ctx->prefill_order ? ctx->cum_pages : nullptr;  // the decode kernels' prefix-sum buffer is free here
     if (ctx->trace != nullptr) cudaMemsetAsync(ctx->trace, 0, static_cast<size_t>(ctx->trace_workers) * 32, static_cast<cudaStream_t>(stream));
     const cudaError_t err = pd::launch_prefill_attn(ctx->cfg.head_dim, ctx->tm_k, ctx->tm_v, p, max_q_len,
                                                     static_cast<cudaStream_t>(stream));
@@ -757,7 +767,9 @@ int pd_device_status(pd_ctx *ctx, void *stream, int32_t *code, int32_t *seq, int
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    int32_t host[pd::kStatusWords] = {0, 0, 0, 0};
+    // only the fault latch (words 0..3) is read and cleared: the words behind it are the range-claim counters
+    // of the split kernel, which a launch in flight on another stream must find untouched
+    int32_t host[4] = {0, 0, 0, 0};
     cudaError_t err = cudaMemcpyAsync(host, ctx->status, sizeof host, cudaMemcpyDeviceToHost, s);
     if (err == cudaSuccess) err = cudaMemsetAsync(ctx->status, 0, sizeof host, s);
     if (err == cudaSuccess) err = cudaStreamSynchronize(s);
@@ -825,7 +837,7 @@ int pd_set_profile_events(pd_ctx *ctx, void *before, void *after) {
 int pd_read_worker_trace(pd_ctx *ctx, void *stream, uint64_t *host_out, int32_t max_workers, int32_t *num_workers) {
     if (ctx == nullptr || host_out == nullptr || num_workers == nullptr || max_workers < 0) return PD_ERR_INVALID_ARG;
     *num_workers = 0;
-    if (ctx->trace == nullptr) return fail(ctx, PD_ERR_UNSUPPORTED, "tracing is off (set PD_TRACE_WORKERS=1 before pd_create)");
+    if (ctx->trace == nullptr) return fail(ctx, PD_ERR_UNSUPPORTED, "tracing is off (needs a PD_ENABLE_TUNING build and PD_TRACE_WORKERS=1 at pd_create)");
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
     const int n = ctx->trace_workers < max_workers ? ctx->trace_workers : max_workers;

@@ -570,11 +570,7 @@ cudaError_t dispatch(const AttnVariant &v, F &&f) {
                       : f(decode_attn_split_kernel<D_, W_, S_, false>, smem_bytes_for<D_, W_, S_, false>()); \
     }
     PD_CASE(128, 8, 3)
-    PD_CASE(128, 4, 6)
-    PD_CASE(128, 12, 2)
-    PD_CASE(128, 6, 4)
     PD_CASE(64, 8, 6)
-    PD_CASE(64, 8, 3)
 #undef PD_CASE
     return cudaErrorInvalidValue;
 }

@@ -550,22 +550,11 @@ namespace {
 // Worker warps per CTA x stages per warp: the bytes in flight per SM stay at 192 KB. The conversions make a
 // page cost ~380 instructions in half the time a bf16 page has, and with two warps per scheduler the
 // dependent chains (convert, MMA, softmax) left the issue slots idle: measured 4.4 TB/s with 8 warps x 6
-// stages, 5.5 with 12 x 4, 6.3 with 16 x 3 (128 registers, no spills), which is the default.
-int fp8_shape() {
-    static const int v = [] {
-        const char *e = std::getenv("PD_TUNE_FP8_WARPS");
-        const int w = e != nullptr ? std::atoi(e) : 16;
-        return (w == 8 || w == 12) ? w : 16;
-    }();
-    return v;
-}
+// stages, 5.5 with 12 x 4, 6.3 with 16 x 3 (128 registers, no spills), which is the shape that is built.
+constexpr int kFp8Warps = 16, kFp8Stages = 3;
 template <bool FUSED, typename F>
 cudaError_t with_fp8_kernel(F &&f) {
-    switch (fp8_shape()) {
-        case 8: return f(decode_attn_split_fp8_kernel<8, 6, FUSED>, fp8_smem_bytes<8, 6>(), 8);
-        case 12: return f(decode_attn_split_fp8_kernel<12, 4, FUSED>, fp8_smem_bytes<12, 4>(), 12);
-        default: return f(decode_attn_split_fp8_kernel<16, 3, FUSED>, fp8_smem_bytes<16, 3>(), 16);
-    }
+    return f(decode_attn_split_fp8_kernel<kFp8Warps, kFp8Stages, FUSED>, fp8_smem_bytes<kFp8Warps, kFp8Stages>(), kFp8Warps);
 }
 }  // namespace
 

@@ -7,8 +7,6 @@
 // the decode worker scatters. A pool page holds all KV heads contiguously
 // ([H_kv][16][d] bf16), so a packed page is the K block followed by the V block
 // and every copy is a run of 16-byte vectors. Pure bandwidth, bit-exact.
-#include <cstdlib>
-
 #include "pd_kernels.cuh"
 #include "pd_ptx.cuh"
 
@@ -16,50 +14,7 @@ namespace pd {
 
 namespace {
 
-template <bool SCATTER>
-__global__ void __launch_bounds__(256) kv_transfer_kernel(const TransferParams p) {
-    const int b = blockIdx.y;
-    grid_dependency_wait();
-    launch_dependents();
-    const int pb = p.page_begin[b], pe = p.page_end[b];
-    const long long base = p.packed_page_offset[b];
-    const size_t vec_per_block = static_cast<size_t>(p.Hkv) * kPageSize * p.D / 8;  // 16-byte vectors in a K (or V) block
-    for (int lp = pb + blockIdx.x; lp < pe; lp += gridDim.x) {
-        int page = (lp >= 0 && lp < p.MP) ? p.page_table[static_cast<size_t>(b) * p.MP + lp] : -1;
-        if (page < 0 || page >= p.num_pages) {
-            if (threadIdx.x == 0 && atomicCAS(p.status, kDevOk, kDevBadPage) == kDevOk) {
-                p.status[1] = b;
-                p.status[2] = page;
-            }
-            continue;
-        }
-        uint4 *packed = reinterpret_cast<uint4 *>(p.packed) + (static_cast<size_t>(base) + (lp - pb)) * 2 * vec_per_block;
-        uint4 *kpool = reinterpret_cast<uint4 *>(p.k_pages) + static_cast<size_t>(page) * vec_per_block;
-        uint4 *vpool = reinterpret_cast<uint4 *>(p.v_pages) + static_cast<size_t>(page) * vec_per_block;
-        // four independent 16-byte loads in flight per thread before the first store
-        for (size_t i = threadIdx.x; i < 2 * vec_per_block; i += 4 * 256) {
-            uint4 v[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const size_t j = i + u * 256;
-                if (j < 2 * vec_per_block) {
-                    const uint4 *pool = j < vec_per_block ? kpool + j : vpool + (j - vec_per_block);
-                    v[u] = SCATTER ? __ldcs(packed + j) : __ldcs(pool);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const size_t j = i + u * 256;
-                if (j < 2 * vec_per_block) {
-                    uint4 *pool = j < vec_per_block ? kpool + j : vpool + (j - vec_per_block);
-                    if (SCATTER) *pool = v[u]; else __stcs(packed + j, v[u]);
-                }
-            }
-        }
-    }
-}
-
-// The same copy driven by the bulk-copy engine: one thread per CTA streams 16 KB chunks global -> shared
+// The copy is driven by the bulk-copy engine: one thread per CTA streams 16 KB chunks global -> shared
 // memory -> global through a ring of stages, with no register traffic at all. Loads run kBulkAhead chunks
 // ahead of stores; the stage of chunk i was last read by the store of chunk i - kBulkStages, after which
 // kBulkStages - kBulkAhead - 1 further store groups were committed, so that many may still be pending when
@@ -153,33 +108,20 @@ __global__ void __launch_bounds__(32) kv_transfer_bulk_kernel(const TransferPara
 
 cudaError_t launch_kv_transfer(const TransferParams &p, bool scatter, int num_sms, cudaStream_t stream) {
     if (p.B == 0) return cudaSuccess;
-    static const int use_bulk = [] {
-        const char *e = std::getenv("PD_TUNE_TRANSFER_BULK");
-        return e != nullptr ? std::atoi(e) : 128;
-    }();
-    if (use_bulk > 0 || p.elem_bytes != 2) {  // FP8 pools always take the bulk kernel
-        // CTAs per sequence: `use_bulk` per SM over the batch. Many short-lived CTAs of a page or two each
-        // measured 6.7 TB/s against 6.0 TB/s for two long-lived CTAs per SM: SMs that get more bandwidth simply
-        // take more CTAs.
-        int per_seq = ((use_bulk > 0 ? use_bulk : 128) * num_sms + p.B - 1) / p.B;
-        per_seq = per_seq < 1 ? 1 : (per_seq > p.MP ? p.MP : per_seq);
-        const dim3 grid(per_seq, p.B);
-        const size_t smem = static_cast<size_t>(kBulkStages) * kBulkChunk;
-        // the opt-in is per device and costs a microsecond: set it on every launch rather than track devices
-        const cudaError_t e = scatter ? cudaFuncSetAttribute(kv_transfer_bulk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                             static_cast<int>(smem))
-                                      : cudaFuncSetAttribute(kv_transfer_bulk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                             static_cast<int>(smem));
-        if (e != cudaSuccess) return e;
-        if (scatter) return launch_pdl(kv_transfer_bulk_kernel<true>, grid, dim3(32), smem, stream, p.pdl != 0, p);
-        return launch_pdl(kv_transfer_bulk_kernel<false>, grid, dim3(32), smem, stream, p.pdl != 0, p);
-    }
-    int per_seq = (16 * num_sms + p.B - 1) / p.B;  // CTAs per sequence: about 16 per SM over the batch
-    if (per_seq < 1) per_seq = 1;
-    if (per_seq > p.MP) per_seq = p.MP;
+    // CTAs per sequence: about 128 per SM over the batch. Many short-lived CTAs of a page or two each measured
+    // 6.7 TB/s against 6.0 TB/s for two long-lived CTAs per SM: SMs that get more bandwidth simply take more CTAs.
+    int per_seq = (128 * num_sms + p.B - 1) / p.B;
+    per_seq = per_seq < 1 ? 1 : (per_seq > p.MP ? p.MP : per_seq);
     const dim3 grid(per_seq, p.B);
-    if (scatter) return launch_pdl(kv_transfer_kernel<true>, grid, dim3(256), 0, stream, p.pdl != 0, p);
-    return launch_pdl(kv_transfer_kernel<false>, grid, dim3(256), 0, stream, p.pdl != 0, p);
+    const size_t smem = static_cast<size_t>(kBulkStages) * kBulkChunk;
+    // the opt-in is per device and costs a microsecond: set it on every launch rather than track devices
+    const cudaError_t e = scatter ? cudaFuncSetAttribute(kv_transfer_bulk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                         static_cast<int>(smem))
+                                  : cudaFuncSetAttribute(kv_transfer_bulk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                         static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    if (scatter) return launch_pdl(kv_transfer_bulk_kernel<true>, grid, dim3(32), smem, stream, p.pdl != 0, p);
+    return launch_pdl(kv_transfer_bulk_kernel<false>, grid, dim3(32), smem, stream, p.pdl != 0, p);
 }
 
 }  // namespace pd

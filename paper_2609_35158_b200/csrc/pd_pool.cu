@@ -194,8 +194,11 @@ int pd_pool_destroy(pd_pool *pool) {
     {
         DeviceScope scope(pool->device);
         if (scope.ok) cudaDeviceSynchronize();
-        while (!pool->handles.empty())
+        while (!pool->handles.empty()) {
+            const size_t before = pool->handles.size();
             if (int e = drop_chunk(pool)) rc = e;
+            if (pool->handles.size() == before) break;  // the unmap failed and the chunk stays: do not spin on it
+        }
         if (pool->base != 0 && driver().ok && driver().addr_free(pool->base, pool->capacity) != CUDA_SUCCESS) rc = PD_ERR_CUDA;
     }
     delete pool;

@@ -14,9 +14,13 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def header_functions():
-    text = open(os.path.join(ROOT, "include", "pd.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(pd_[a-z0-9_]+)\s*\(", text)))
+    names = set()
+    for f in sorted(os.listdir(os.path.join(ROOT, "include"))):
+        if f.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", f)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(pd_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_library_builds_and_exports_every_declared_symbol():
@@ -149,9 +153,27 @@ def test_reference_arm_prints_the_contract_line():
 
 
 def test_header_is_plain_c99_and_cxx():
-    """include/pd.h must be usable from C and from C++ without any CUDA header."""
-    hdr = os.path.join(ROOT, "include", "pd.h")
-    for cmd in (["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c", hdr],
-                ["g++", "-std=c++17", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", hdr]):
-        res = subprocess.run(cmd, capture_output=True, text=True)
-        assert res.returncode == 0, res.stderr
+    """The public headers must be usable from C and from C++ without any CUDA header."""
+    for name in ("pd.h", "pd_debug.h"):
+        hdr = os.path.join(ROOT, "include", name)
+        for cmd in (["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c", hdr],
+                    ["g++", "-std=c++17", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", hdr]):
+            res = subprocess.run(cmd, capture_output=True, text=True)
+            assert res.returncode == 0, res.stderr
+
+
+def test_shipped_build_reads_no_environment_variable_after_create():
+    """Tuning knobs exist only in a -DPD_ENABLE_TUNING build: the one getenv of the sources sits under that macro."""
+    csrc = os.path.join(ROOT, "paper_2609_35158_b200", "csrc")
+    hits = []
+    for f in sorted(os.listdir(csrc)):
+        lines = open(os.path.join(csrc, f)).read().splitlines()
+        hits += [(f, i) for i, line in enumerate(lines) if "getenv" in line]
+    assert len(hits) == 1 and hits[0][0] == "pd_api.cu"
+    lines = open(os.path.join(csrc, "pd_api.cu")).read().splitlines()
+    before = lines[:hits[0][1]]
+    assert max(i for i, l in enumerate(before) if l.startswith("#ifdef PD_ENABLE_TUNING")) > \
+        max([i for i, l in enumerate(before) if l.startswith("#endif")] + [-1])
+    from paper_2609_35158_b200 import build as pd_build
+
+    assert not any("PD_ENABLE_TUNING" in flag for flag in pd_build.NVCC_FLAGS)
