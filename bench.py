@@ -8,8 +8,14 @@ synthetic, shaped like the paper's rollout workloads (see ``workloads``).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl cuda|reference]
 
-Prints ONE JSON line on rank 0. ``--impl reference`` times the CPU oracle (test
-infrastructure, run as it stands) on the host cores instead of the CUDA path.
+Prints ONE JSON line on rank 0. Without ``--config`` the headline is the largest
+single-GPU workload (the multi-turn loop with page allocation) and the other
+three target workloads are measured the same way in the same process and
+reported under ``per_config``. ``--gpus N`` runs N independent replicas, one
+process per GPU: under a launcher that sets WORLD_SIZE the script is one of the
+ranks, otherwise it starts the ranks itself. ``--impl reference`` times the CPU
+oracle (test infrastructure, run as it stands) on the host cores instead of the
+CUDA path.
 """
 from __future__ import annotations
 
@@ -29,10 +35,13 @@ import numpy as np  # noqa: E402
 METRIC = "decode-attn achieved HBM GB/s (% of B200 peak) and seq-steps/s per layer"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes (read + write) per launch of the split kernel in the committed ncu capture
-# (profiles/decode_attn_split_config3_ncu.md: 1.577338 GB + 7.53 MB), as a ratio to the
-# algorithmic KV bytes of that launch (1.576878 GB); traffic grows in proportion to the pages read.
-NCU_TRAFFIC_RATIO = 1.0051
+HEADLINE_CONFIG = 4        # the largest single-GPU workload: the multi-turn loop with page allocation
+PER_CONFIG = (1, 2, 3)     # the other target workloads, measured in the same process
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the split kernel in the committed ncu
+# captures, as a ratio to the algorithmic KV bytes of the captured launch; traffic grows in proportion to the
+# pages read, so the ratio of a captured slice of a batch stands for the whole batch.
+NCU_TRAFFIC_SOURCE = "profiles/decode_attn_split_traffic_ncu.md"
+NCU_TRAFFIC_RATIO = {1: 1.0044, 2: 1.0044, 3: 1.0048, 4: 1.0030}
 
 
 def measured_hbm_peak():
@@ -53,7 +62,7 @@ class ClockSampler(threading.Thread):
         0x100: "display_clock_setting",
     }
 
-    def __init__(self, device_index: int, period_s: float = 0.002):
+    def __init__(self, device_index: int, period_s: float = 0.001):
         super().__init__(daemon=True)
         self.period = period_s
         self.samples, self.reasons = [], set()
@@ -90,14 +99,20 @@ class ClockSampler(threading.Thread):
                 pass
             time.sleep(self.period)
 
-    def stop(self):
+    def stop(self, also=None):
+        """Stops sampling and summarises; ``also`` = samplers already stopped whose samples join the summary
+        (the clocks of two timed regions of one measurement)."""
         self._stop_evt.set()
         if self.is_alive():
             self.join(timeout=2)
-        if not self.ok or not self.samples:
+        samples, reasons = list(self.samples), set(self.reasons)
+        for other in also or ():
+            samples += other.samples
+            reasons |= other.reasons
+        if not self.ok or not samples:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["nvml unavailable"]}
-        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        return {"sm_mhz": float(np.median(samples)), "sm_min_mhz": float(np.min(samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(reasons), "samples": len(samples)}
 
 
 def aggregate_over_ranks(local_ms: float, local_units: float, world_size: int, backend_device=None):
@@ -116,7 +131,7 @@ def aggregate_over_ranks(local_ms: float, local_units: float, world_size: int, b
 
 def workload_config(w, lens, cfg_id):
     return {
-        "workload": f"configs[{cfg_id}] {w.name}", "batch": int(w.batch), "num_q_heads": w.num_q_heads,
+        "workload": f"configs[{cfg_id}] {w.name}", "batch": int(len(lens)), "num_q_heads": w.num_q_heads,
         "num_kv_heads": w.num_kv_heads, "head_dim": w.head_dim, "page_size": w.page_size,
         "ctx_tokens_total": int(np.sum(lens)), "ctx_len_min": int(np.min(lens)), "ctx_len_max": int(np.max(lens)),
     }
@@ -124,28 +139,39 @@ def workload_config(w, lens, cfg_id):
 
 # ------------------------------------------------------------------------------------------ CUDA arm
 
-def run_cuda(args):
+def hooked_steps(K: int):
+    """Timed steps whose split kernel is bracketed by events: every 4th step of a short run, every 16th of a
+    long one, and never fewer than three (or all of them when K < 3)."""
+    stride = 4 if K < 48 else 16
+    picks = [i for i in range(K) if i % stride == stride // 2]
+    if len(picks) < 3:
+        picks = sorted({min(K - 1, (2 * j + 1) * K // 6) for j in range(3)})
+    return picks
+
+
+def oracle_sample_size(lens, max_tokens: int = 600_000) -> int:
+    """Leading sequences whose cached tokens stay within the CPU baseline's budget (at least one)."""
+    csum = np.cumsum(np.asarray(lens, dtype=np.int64))
+    return max(1, int(np.searchsorted(csum, max_tokens, side="right")))
+
+
+def measure_decode(cfg_id, args, rank, world, local_rank, want_cpu_baseline=True):
+    """Times one workload: K steps with device-resident inputs, K steps through the host-buffer entry point,
+    the split kernel's own duration on a sample of the timed steps, and the oracle on the host cores."""
     import torch
 
     import paper_2609_35158_b200 as pd
     import workloads as wl
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        import torch.distributed as dist
-
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
-    torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
-    cfg_id = args.config
     w = wl.WORKLOADS[cfg_id]
     K, W = args.steps, args.warmup
     # weak scaling: every rank holds its own batch of the same shape (sequences are independent)
     seed = cfg_id + 1000 * rank
     lens0 = wl.context_lengths(cfg_id, seed=seed)
-    B = w.batch
+    if args.batch is not None:
+        lens0 = lens0[:args.batch]
+    B = len(lens0)
     total_steps = 2 * (W + K) + 8  # device-resident loop, then the host-buffer loop
     dynamic_alloc = cfg_id == 4   # pages handed out by the host free list inside the loop
     cache = wl.build_paged_cache(lens0, w.num_kv_heads, w.head_dim, seed=seed, device=dev,
@@ -165,7 +191,6 @@ def run_cuda(args):
     stage_rows = 2 * (W + K) + 8
     staging = torch.empty((stage_rows, 3, B), dtype=torch.int64).pin_memory() if dynamic_alloc else None
     alloc_calls = [0]
-
     alloc_seconds = [0.0]
 
     def allocate_pages():
@@ -173,21 +198,18 @@ def run_cuda(args):
             return
         t_alloc = time.perf_counter()
         try:
-            _allocate_pages()
+            need, logical, phys = alloc.assign(lens)
+            n = len(need)
+            if n:
+                row = staging[alloc_calls[0] % stage_rows]
+                alloc_calls[0] += 1
+                row[0, :n] = torch.from_numpy(need)
+                row[1, :n] = torch.from_numpy(logical)
+                row[2, :n] = torch.from_numpy(phys.astype(np.int64))
+                upd = row[:, :n].to(dev, non_blocking=True)
+                cache.page_table[upd[0], upd[1]] = upd[2].to(torch.int32)
         finally:
             alloc_seconds[0] += time.perf_counter() - t_alloc
-
-    def _allocate_pages():
-        need, logical, phys = alloc.assign(lens)
-        n = len(need)
-        if n:
-            row = staging[alloc_calls[0] % stage_rows]
-            alloc_calls[0] += 1
-            row[0, :n] = torch.from_numpy(need)
-            row[1, :n] = torch.from_numpy(logical)
-            row[2, :n] = torch.from_numpy(phys.astype(np.int64))
-            upd = row[:, :n].to(dev, non_blocking=True)
-            cache.page_table[upd[0], upd[1]] = upd[2].to(torch.int32)
 
     def device_step(i):
         nonlocal lens
@@ -217,8 +239,9 @@ def run_cuda(args):
     assert code[0] == 0, f"device fault during warm-up: {code}"
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     # The library's event hook brackets the split kernel of one step. Two event records cost several
-    # microseconds of stream time and switch off launch overlap for that step, so one step in sixteen is hooked.
-    hooked = [i for i in range(K) if i % 16 == min(8, K - 1)]
+    # microseconds of stream time and switch off launch overlap for that step, so only a sample of the timed
+    # steps is hooked.
+    hooked = hooked_steps(K)
     befores = {i: torch.cuda.Event(enable_timing=True) for i in hooked}
     afters = {i: torch.cuda.Event(enable_timing=True) for i in hooked}
     sampler = ClockSampler(local_rank)
@@ -227,7 +250,7 @@ def run_cuda(args):
     sampler.start()
     t0.record()
     kv_bytes = 0
-    split_bytes = 0
+    hooked_bytes = {}
     alloc_seconds[0] = 0.0
     for i in range(K):
         if i in befores:
@@ -235,15 +258,17 @@ def run_cuda(args):
         step_bytes = device_step(W + i)
         kv_bytes += step_bytes
         if i in befores:
-            split_bytes += step_bytes
+            hooked_bytes[i] = step_bytes
     t1.record()
     barrier()
     clocks = sampler.stop()
     launches = pd.pd_launch_count(ctx) - launches0
     local_ms = t0.elapsed_time(t1)
     alloc_host_us = 1e6 * alloc_seconds[0] / K  # host time of the page allocator per step of the device-resident loop
-    split_ms = float(np.mean([befores[i].elapsed_time(afters[i]) for i in hooked]))
-    split_bytes_per_launch = split_bytes / len(hooked)
+    split_times = [befores[i].elapsed_time(afters[i]) for i in hooked]
+    split_ms = float(np.mean(split_times))
+    split_bytes_per_launch = float(np.mean([hooked_bytes[i] for i in hooked]))
+    best = int(np.argmin(split_times))
     plan = pd.pd_last_plan(ctx)
     assert pd.pd_device_status(ctx)[0] == 0
     total_ms, total_bytes = aggregate_over_ranks(local_ms, float(kv_bytes), world, dev)
@@ -251,51 +276,63 @@ def run_cuda(args):
     bytes_per_step_local = kv_bytes / K
 
     # ---- host-buffer loop: same step through pd_decode_step_host, copies inside the timed region
-    # one pinned slab per rotation slot, q then k_new then v_new: adjacent host buffers travel in one copy
-    hq, hk, hv = [], [], []
-    for tq, tk, tv in zip(qs, kns, vns):
-        slab = torch.empty(tq.numel() + tk.numel() + tv.numel(), dtype=torch.bfloat16).pin_memory()
-        a, b2 = tq.numel(), tq.numel() + tk.numel()
-        slab[:a].copy_(tq.reshape(-1)); slab[a:b2].copy_(tk.reshape(-1)); slab[b2:].copy_(tv.reshape(-1))
-        hq.append(slab[:a].view(tq.shape)); hk.append(slab[a:b2].view(tk.shape)); hv.append(slab[b2:].view(tv.shape))
-    hout = torch.empty((B, w.num_q_heads, w.head_dim), dtype=torch.bfloat16).pin_memory()
+    e2e = None
+    if not args.no_e2e:
+        # one pinned slab per rotation slot, q then k_new then v_new: adjacent host buffers travel in one copy
+        hq, hk, hv = [], [], []
+        for tq, tk, tv in zip(qs, kns, vns):
+            slab = torch.empty(tq.numel() + tk.numel() + tv.numel(), dtype=torch.bfloat16).pin_memory()
+            a, b2 = tq.numel(), tq.numel() + tk.numel()
+            slab[:a].copy_(tq.reshape(-1)); slab[a:b2].copy_(tk.reshape(-1)); slab[b2:].copy_(tv.reshape(-1))
+            hq.append(slab[:a].view(tq.shape)); hk.append(slab[a:b2].view(tk.shape)); hv.append(slab[b2:].view(tv.shape))
+        hout = torch.empty((B, w.num_q_heads, w.head_dim), dtype=torch.bfloat16).pin_memory()
 
-    def host_step(i):
-        nonlocal lens
-        allocate_pages()
-        pd.pd_decode_step_host(ctx, hq[i % R], hk[i % R], hv[i % R], cache.k_pages, cache.v_pages, cache.page_table,
-                               cache.ctx_lens, hout, sm_scale=w.sm_scale)
-        lens = lens + 1
-        return int(lens.sum()) * bpt
+        def host_step(i):
+            nonlocal lens
+            allocate_pages()
+            pd.pd_decode_step_host(ctx, hq[i % R], hk[i % R], hv[i % R], cache.k_pages, cache.v_pages, cache.page_table,
+                                   cache.ctx_lens, hout, sm_scale=w.sm_scale)
+            lens = lens + 1
+            return int(lens.sum()) * bpt
 
-    for i in range(W):
-        host_step(i)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    e2e_bytes = 0
-    for i in range(K):
-        e2e_bytes += host_step(W + i)
-    e1.record()
-    barrier()
-    e2e_ms, e2e_total = aggregate_over_ranks(e0.elapsed_time(e1), float(e2e_bytes), world, dev)
-    e2e_gbs = e2e_total / (e2e_ms * 1e-3) / 1e9
-    h2d = (hq[0].numel() + hk[0].numel() + hv[0].numel()) * 2
-    d2h = hout.numel() * 2
-    assert pd.pd_device_status(ctx)[0] == 0
+        for i in range(W):
+            host_step(i)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler2 = ClockSampler(local_rank)
+        sampler2.start()
+        e0.record()
+        e2e_bytes = 0
+        for i in range(K):
+            e2e_bytes += host_step(W + i)
+        e1.record()
+        barrier()
+        clocks = sampler2.stop(also=[sampler])  # samples of both timed regions of this workload
+        clocks["regions"] = "device-resident loop + host-buffer loop"
+        e2e_ms, e2e_total = aggregate_over_ranks(e0.elapsed_time(e1), float(e2e_bytes), world, dev)
+        e2e_gbs = e2e_total / (e2e_ms * 1e-3) / 1e9
+        h2d = (hq[0].numel() + hk[0].numel() + hv[0].numel()) * 2
+        d2h = hout.numel() * 2
+        assert pd.pd_device_status(ctx)[0] == 0
+        e2e = {"value": round(e2e_gbs, 2), "unit": "GB/s", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+               "ms_per_step": round(e2e_ms / K, 5),
+               "note": "pd_decode_step_host: q/k_new/v_new from one pinned host slab (one H2D copy), out back to host, "
+                       "every step; the KV cache is device-resident state"}
 
     # ---- CPU baseline: the oracle as it stands, on this machine's host cores (rank 0, N = 1 only)
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if want_cpu_baseline and rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = time_oracle_once(w, cache, qs[0], lens)
 
     peak, peak_kind = measured_hbm_peak()
     achieved = split_bytes_per_launch / (split_ms * 1e-3) / 1e9
+    ratio = NCU_TRAFFIC_RATIO.get(cfg_id) if args.batch is None else None
     result = {
         "metric": METRIC, "value": round(value_gbs, 2), "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": round(total_ms / K, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {**workload_config(w, lens, cfg_id),
+        "config": {**workload_config(w, lens0, cfg_id),
+                   "ctx_tokens_after_run": int(np.sum(lens)),
                    "l2": f"KV read per step {bytes_per_step_local / 1e9:.2f} GB per GPU >> 126 MB L2; activations rotate over {R} buffers",
                    "parallelism": "1 GPU" if world == 1 else f"{world} independent replicas, sequences sharded by batch, no collective",
                    "plan": plan,
@@ -306,18 +343,51 @@ def run_cuda(args):
         "pct_of_nominal_8tbs": round(100 * value_gbs / world / NOMINAL_HBM_GBS, 2),
         "seq_steps_per_s": round(B * world * K / (total_ms * 1e-3), 1),
         "clocks": clocks,
-        "e2e": {"value": round(e2e_gbs, 2), "unit": "GB/s", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                "ms_per_step": round(e2e_ms / K, 5),
-                "note": "pd_decode_step_host: q/k_new/v_new from one pinned host slab (one H2D copy), out back to host, every step; the KV cache is device-resident state"},
+        "e2e": e2e,
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "decode_attn_split_kernel", "achieved": round(achieved, 2), "peak": peak,
                      "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}",
-                     "traffic": None if NCU_TRAFFIC_RATIO is None else int(NCU_TRAFFIC_RATIO * split_bytes_per_launch),
+                     "traffic": None if ratio is None else int(ratio * split_bytes_per_launch),
+                     "traffic_source": None if ratio is None else NCU_TRAFFIC_SOURCE,
                      "algorithmic_bytes_per_launch": int(split_bytes_per_launch), "avg_launch_ms": round(split_ms, 5),
+                     "min_launch_ms": round(float(split_times[best]), 5),
+                     "achieved_best": round(hooked_bytes[hooked[best]] / (split_times[best] * 1e-3) / 1e9, 2),
+                     "launches_timed": len(hooked),
                      "timed": f"CUDA events recorded by the library around the split kernel, {len(hooked)} of the {K} timed launches"},
         "cpu_baseline": cpu_baseline,
     }
     pd.pd_destroy(ctx)
+    del cache, qs, kns, vns, out
+    torch.cuda.empty_cache()
+    return result
+
+
+def run_cuda(args):
+    import torch
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    torch.cuda.set_device(local_rank)
+    # default run: the headline is the largest single-GPU workload (the multi-turn loop); the other three
+    # target workloads are measured the same way in the same process and reported under per_config
+    head_cfg, others = (HEADLINE_CONFIG, PER_CONFIG) if args.config is None else (args.config, ())
+    per = {}
+    for c in others:
+        try:
+            r = measure_decode(c, args, rank, world, local_rank)
+            per[f"configs[{c}]"] = {k: r[k] for k in ("value", "unit", "ms_per_step", "pct_of_measured_hbm_peak",
+                                                     "pct_of_nominal_8tbs", "seq_steps_per_s", "clocks", "e2e", "gpu_launches",
+                                                     "roofline", "cpu_baseline", "config")}
+        except Exception as e:  # the headline must still be measured
+            per[f"configs[{c}]"] = {"error": repr(e)}
+    result = measure_decode(head_cfg, args, rank, world, local_rank)
+    if others:
+        result["per_config"] = per
     if rank == 0:
         print(json.dumps(result), flush=True)
     if world > 1:
@@ -334,8 +404,9 @@ def time_oracle_once(w, cache, q, lens, max_seconds_hint: float = 30.0):
 
     cores = os.cpu_count() or 1
     B = len(lens)
-    # bounded sample: the oracle handles roughly 1.5e6 (token x query head) per core-second
-    n = B
+    # bounded sample: a prefix of the batch of at most ~600 k cached tokens (2.4 GB of KV at 32/8 heads);
+    # the oracle handles roughly 1.5e6 (token x query head) per core-second
+    n = oracle_sample_size(lens)
     while n > 1 and float(np.sum(lens[:n])) * w.num_q_heads / (1.5e6 * cores) > max_seconds_hint:
         n //= 2
     # bring only the pages those sequences own to the host, renumbered (the result does not depend on page ids)
@@ -842,6 +913,40 @@ def run_pool_toggle(args):
     }), flush=True)
 
 
+# ------------------------------------------------------------------------------------------ read ceiling
+
+def run_read_ceiling(args):
+    """Read-only HBM ceiling of this GPU: a plain streaming kernel (16-byte loads, nothing stored) over 4 GB,
+    best of several grid shapes, set beside the measured copy bandwidth that is the roofline denominator."""
+    import torch
+
+    import paper_2609_35158_b200 as pd
+
+    torch.cuda.set_device(0)
+    buf = torch.full((4 << 30,), 1, dtype=torch.uint8, device="cuda:0")
+    sink = torch.zeros(16, dtype=torch.uint8, device="cuda:0")
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    rows = []
+    for per_sm in (2, 4, 8, 16, 32):
+        for threads in (256, 512, 1024):
+            for _ in range(max(3, args.warmup)):
+                pd.pd_read_probe(buf, sms * per_sm, threads, sink)
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            t0.record()
+            for _ in range(args.steps):
+                pd.pd_read_probe(buf, sms * per_sm, threads, sink)
+            t1.record()
+            torch.cuda.synchronize()
+            rows.append({"blocks_per_sm": per_sm, "threads": threads,
+                         "gbs": round(buf.numel() * args.steps / (t0.elapsed_time(t1) * 1e-3) / 1e9, 1)})
+    best = max(rows, key=lambda r: r["gbs"])
+    peak, kind = measured_hbm_peak()
+    print(json.dumps({"metric": "read-only streaming bandwidth (16-byte loads over 4 GB, nothing stored)", "value": best["gbs"],
+                      "unit": "GB/s", "best_shape": best, "steps": args.steps, "copy_bandwidth_gbs": peak,
+                      "copy_bandwidth_kind": kind, "ratio_to_copy": round(best["gbs"] / peak, 4), "by_shape": rows}), flush=True)
+
+
 # ------------------------------------------------------------------------------------------ reference arm
 
 def run_reference(args):
@@ -852,11 +957,13 @@ def run_reference(args):
     import oracle
     import workloads as wl
 
-    cfg_id = args.config
+    cfg_id = HEADLINE_CONFIG if args.config is None else args.config
     w = wl.WORKLOADS[cfg_id]
     K, W = args.steps, args.warmup
     cores = os.cpu_count() or 1
     lens_all = wl.context_lengths(cfg_id)
+    if args.batch is not None:
+        lens_all = lens_all[:args.batch]
     # bounded sample: whole run (K + W steps) within about two minutes. The oracle handles
     # roughly 2e6 (token x query head) per core-second; stay well below that.
     budget_tokens = 120.0 * 1.5e6 * cores / w.num_q_heads / max(1, K + W)
@@ -885,10 +992,11 @@ def run_reference(args):
               f"{nbytes / 1e9:.4f} GB of KV per step)")
     result = {
         "impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": "GB/s",
-        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": K, "warmup": W,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", str(args.gpus))), "steps": K, "warmup": W,
         "ms_per_step": round(dt / K * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {**workload_config(w, lens, cfg_id), "sample": sample},
+        # the workload is the CUDA arm's (same lengths, same totals); `sample` says which part of it a step covers
+        "config": {**workload_config(w, lens_all, cfg_id), "sample": sample},
         "cpu_baseline": {"value": round(value, 4), "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": round(value, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -896,27 +1004,100 @@ def run_reference(args):
     print(json.dumps(result), flush=True)
 
 
+# ------------------------------------------------------------------------------------------ replicas
+
+def spawn_replicas(args) -> int:
+    """`--gpus N` without a launcher: start N ranks of this script, one process per GPU (RANK = LOCAL_RANK =
+    0 .. N-1, rendezvous on 127.0.0.1). The ranks are independent replicas: every one builds its own cache
+    (seed + 1000 * rank) and the only communication is the barrier around the timed region and the max / sum
+    of two scalars. Rank 0 prints the line."""
+    import socket
+    import subprocess
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    procs = []
+    for r in range(args.gpus):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(args.gpus), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__), *sys.argv[1:]], env=env))
+    rc = 0
+    for p in procs:
+        try:
+            rc = max(rc, abs(p.wait(timeout=3600)))
+        except subprocess.TimeoutExpired:
+            rc = 1
+        if rc:  # one rank failed: the others would wait for it at the barrier
+            for other in procs:
+                if other.poll() is None:
+                    other.kill()
+    return rc
+
+
+def run_stub(args):
+    """The multi-rank plumbing with a host stand-in for the step (no GPU, gloo): barrier, K timed 'steps' that
+    sleep, max-over-ranks time and summed units, one line from rank 0. It exists so that the spawn path and the
+    aggregation can be tested on a machine without GPUs; it measures nothing."""
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    t = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep(0.001 * (rank + 1))
+    local_ms = (time.perf_counter() - t) * 1e3
+    if world > 1:
+        dist.barrier()
+    ms, units = aggregate_over_ranks(local_ms, float(100 * (rank + 1)), world)
+    if rank == 0:
+        print(json.dumps({"impl": "stub", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                          "ms_per_step": round(ms / args.steps, 4), "units": units, "scaling": "weak",
+                          "seeds": [HEADLINE_CONFIG + 1000 * r for r in range(world)]}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", type=int, default=1, choices=[0, 1, 2, 3, 4])
-    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--gpus", type=int, default=1, help="ranks, one per GPU; without a launcher (no WORLD_SIZE in the "
+                    "environment) the script starts them itself")
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", type=int, default=None, choices=[0, 1, 2, 3, 4],
+                    help="default: headline on configs[4], configs[1..3] under per_config")
+    ap.add_argument("--batch", type=int, default=None, help="only the first N sequences of the workload (small ncu captures)")
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference", "stub"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer loop (small ncu captures)")
     ap.add_argument("--step", default=None, choices=["separate", "fused"],
                     help="pd_kv_append + pd_decode_attn (3 launches) or pd_decode_step (2 launches); default: fused for "
                          "--op decode, separate for --op decode_fp8 (there the fused kernel measured slower)")
-    ap.add_argument("--op", default="decode", choices=["decode", "decode_fp8", "kv_transfer", "prefill", "fit_b", "pool_toggle"],
+    ap.add_argument("--op", default="decode", choices=["decode", "decode_fp8", "kv_transfer", "prefill", "fit_b", "pool_toggle", "read_ceiling"],
                     help="decode = the headline decode step; kv_transfer = page gather + scatter; "
                          "prefill = one append-prefill turn; fit_b = decode step time over batch size, fitted to A + b * B; "
                          "pool_toggle = release and restore of a KV pool's physical memory; "
-                         "decode_fp8 = the decode step over FP8 (e4m3) KV pages")
+                         "decode_fp8 = the decode step over FP8 (e4m3) KV pages; "
+                         "read_ceiling = a plain read-only streaming kernel, the practical ceiling of a read-once scan")
     args = ap.parse_args()
+    if args.gpus < 1:
+        ap.error("--gpus must be >= 1")
+    world_env = os.environ.get("WORLD_SIZE")
+    if world_env is not None and int(world_env) != args.gpus:
+        ap.error(f"--gpus {args.gpus} but the launcher set WORLD_SIZE={world_env}")
+    if args.gpus > 1 and world_env is None and args.impl != "reference":
+        if args.op != "decode":
+            ap.error("--gpus N > 1 runs replicas of the decode step only")
+        sys.exit(spawn_replicas(args))
     if args.step is None:
         args.step = "separate" if args.op == "decode_fp8" else "fused"
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
+    if args.op != "decode" and args.config is None:
+        args.config = 1
     if args.impl == "cuda":
         # the built library is not tracked: compile it if this checkout has none yet (rank 0 first under torchrun)
         import __graft_entry__ as entry
@@ -930,6 +1111,8 @@ def main():
                 time.sleep(0.5)
     if args.impl == "reference":
         run_reference(args)
+    elif args.impl == "stub":
+        run_stub(args)
     elif args.op == "kv_transfer":
         run_transfer(args)
     elif args.op == "prefill":
@@ -940,6 +1123,8 @@ def main():
         run_decode_fp8(args)
     elif args.op == "pool_toggle":
         run_pool_toggle(args)
+    elif args.op == "read_ceiling":
+        run_read_ceiling(args)
     else:
         run_cuda(args)
 

@@ -42,6 +42,15 @@ int pd_set_profile_events(pd_ctx *ctx, void *before, void *after);
  */
 int pd_read_worker_trace(pd_ctx *ctx, void *stream, uint64_t *host_out, int32_t max_workers, int32_t *num_workers);
 
+/*
+ * Read-only streaming probe: launches a kernel of `blocks` x `threads` that reads `bytes` (a multiple of 16
+ * is read) from src once with 16-byte streaming loads and stores nothing (sink16 is a 16-byte device
+ * buffer the kernel is formally allowed to write). Timed with events by the caller, it gives the read-only
+ * HBM ceiling of the GPU, to set beside the copy bandwidth that serves as the roofline denominator of the
+ * decode kernels (Eq. 1's b is a read). No context is needed; src and sink16 are device pointers, 16-byte aligned.
+ */
+int pd_read_probe(const void *src, size_t bytes, int32_t blocks, int32_t threads, void *sink16, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

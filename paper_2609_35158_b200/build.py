@@ -8,7 +8,7 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libpd.so")
-SOURCES = ["pd_api.cu", "pd_decode_attn.cu", "pd_decode_attn_fp8.cu", "pd_kv_append.cu", "pd_kv_transfer.cu", "pd_prefill_attn.cu", "pd_static.cu", "pd_decision.cu", "pd_pool.cu"]
+SOURCES = ["pd_api.cu", "pd_decode_attn.cu", "pd_decode_attn_fp8.cu", "pd_kv_append.cu", "pd_kv_transfer.cu", "pd_prefill_attn.cu", "pd_prefill_attn_d128.cu", "pd_static.cu", "pd_decision.cu", "pd_pool.cu", "pd_probe.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-Xcompiler", "-fPIC", "-shared", "--use_fast_math", "-Xptxas", "-v",

@@ -495,26 +495,28 @@ size_t prefill_smem_bytes(int head_dim) {
     return static_cast<size_t>(halves) * (kQHalfBytes + 2 * kStages * kHalfBytes) + 1024 + (2 * kStages + 6) * 8 + 64;
 }
 
+// head_dim 128 has its own kernel (pd_prefill_attn_d128.cu: two query tiles per CTA, 128-token blocks)
+cudaError_t prepare_prefill_attn_d128();
+cudaError_t launch_prefill_attn_d128(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const PrefillParams &p, int max_q_len,
+                                     cudaStream_t stream);
+
 cudaError_t prepare_prefill_attn(int head_dim) {
+    if (head_dim == 128) return prepare_prefill_attn_d128();
     const int bytes = static_cast<int>(prefill_smem_bytes(head_dim));
-    if (head_dim == 128)
-        return cudaFuncSetAttribute(prefill_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     return cudaFuncSetAttribute(prefill_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 
 cudaError_t launch_prefill_attn(int head_dim, const CUtensorMap &tm_k, const CUtensorMap &tm_v, const PrefillParams &p,
                                 int max_q_len, cudaStream_t stream) {
     if (p.B == 0 || max_q_len <= 0) return cudaSuccess;
-    const int tok = kRows / p.G;
-    const dim3 grid((max_q_len + tok - 1) / tok, p.Hkv, p.B);
-    const size_t smem = prefill_smem_bytes(head_dim);
     if (p.order != nullptr) {
         const cudaError_t e = launch_pdl(prefill_order_kernel, dim3((p.B + 255) / 256), dim3(256), 0, stream, p.pdl != 0, p);
         if (e != cudaSuccess) return e;
     }
-    if (head_dim == 128)
-        return launch_pdl(prefill_attn_kernel<128>, grid, dim3(kThreads), smem, stream, p.pdl != 0, tm_k, tm_v, p);
-    return launch_pdl(prefill_attn_kernel<64>, grid, dim3(kThreads), smem, stream, p.pdl != 0, tm_k, tm_v, p);
+    if (head_dim == 128) return launch_prefill_attn_d128(tm_k, tm_v, p, max_q_len, stream);
+    const int tok = kRows / p.G;
+    const dim3 grid((max_q_len + tok - 1) / tok, p.Hkv, p.B);
+    return launch_pdl(prefill_attn_kernel<64>, grid, dim3(kThreads), prefill_smem_bytes(head_dim), stream, p.pdl != 0, tm_k, tm_v, p);
 }
 
 cudaError_t launch_kv_append_tokens(const AppendTokensParams &p, int max_q_len, cudaStream_t stream) {

@@ -152,6 +152,37 @@ def test_reference_arm_prints_the_contract_line():
     assert "workload" in r["config"] and r["data"] == "synthetic"
 
 
+def test_gpus_flag_spawns_that_many_ranks():
+    """`bench.py --gpus 2` with no launcher starts two ranks itself (here with the host stand-in step over gloo):
+    rank 0 prints one line that carries n_gpus = 2, the max over ranks of the time and the sum of the units."""
+    import json
+
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "stub", "--gpus", "2", "--steps", "5",
+                          "--warmup", "1"], capture_output=True, text=True, timeout=300, cwd=ROOT, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, res.stdout
+    r = json.loads(lines[0])
+    assert r["n_gpus"] == 2 and r["steps"] == 5 and r["units"] == 300.0 and r["scaling"] == "weak"
+    assert r["ms_per_step"] >= 2.0          # rank 1 sleeps 2 ms per step: the slower rank sets the time
+    assert r["seeds"] == [4, 1004]          # every replica draws its own batch
+    # a launcher that disagrees with --gpus is an error, not a silent 1-GPU run
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "stub", "--gpus", "2"],
+                         capture_output=True, text=True, timeout=60, cwd=ROOT, env=dict(env, WORLD_SIZE="1", RANK="0"))
+    assert res.returncode != 0 and "WORLD_SIZE" in res.stderr
+
+
+def test_hooked_steps_are_at_least_three():
+    import bench
+
+    for K in (1, 2, 3, 5, 11, 12, 20, 47, 48, 200):
+        picks = bench.hooked_steps(K)
+        assert len(picks) == len(set(picks)) and all(0 <= i < K for i in picks)
+        assert len(picks) >= min(3, K), (K, picks)
+    assert len(bench.hooked_steps(20)) == 5 and len(bench.hooked_steps(200)) == 12
+
+
 def test_header_is_plain_c99_and_cxx():
     """The public headers must be usable from C and from C++ without any CUDA header."""
     for name in ("pd.h", "pd_debug.h"):

@@ -94,7 +94,7 @@ def test_fp8_attention_small_ragged_poisoned(Hq, Hkv, split_pages):
     # outputs here are ~0.02 in magnitude: compare relative to the output scale
     live = lens > 0
     assert_parity((out[torch.from_numpy(live).to(DEV)].float() * 50).to(torch.bfloat16), ref[live] * 50,
-                  f"{Hq}/{Hkv} split {split_pages}", scale_abs_above=2.0)
+                  f"{Hq}/{Hkv} split {split_pages}", scale_abs_by_magnitude=True)
     got_lse = lse.cpu().numpy()
     assert np.all(np.isneginf(got_lse[~live])) and np.all(out[torch.from_numpy(~live).to(DEV)].float().cpu().numpy() == 0)
     np.testing.assert_allclose(got_lse[live], ref_lse[live], rtol=3e-5, atol=3e-5)
@@ -157,7 +157,7 @@ def test_fp8_append_bit_exact_then_attend():
         torch.cuda.synchronize()
         assert pd.pd_device_status(ctx.h)[0] == 0
     ref, _ = oracle.fp8_decode_attn(oracle.bf16_bits(q), k8, v8, sc, cache.page_table_host, lens, d ** -0.5)
-    assert_parity(out, ref, "after 20 FP8 appends", scale_abs_above=2.0)
+    assert_parity(out, ref, "after 20 FP8 appends", scale_abs_by_magnitude=True)
 
 
 def test_fp8_append_errors_are_reported_and_skipped():
@@ -382,4 +382,4 @@ def test_fp8_fused_step_is_bit_identical_to_append_plus_attention(Hq, Hkv, split
     assert np.array_equal(b[0].cpu().numpy(), k8) and np.array_equal(b[1].cpu().numpy(), v8)
     assert np.array_equal(b[2].cpu().numpy().view(np.uint32), sc.view(np.uint32)) and np.array_equal(lens_h, lens0 + steps)
     ref, _ = oracle.fp8_decode_attn(oracle.bf16_bits(q), k8, v8, sc, cache.page_table_host, lens_h, scale)
-    assert_parity(out_b, ref, "fused FP8 step", scale_abs_above=2.0)
+    assert_parity(out_b, ref, "fused FP8 step", scale_abs_by_magnitude=True)
