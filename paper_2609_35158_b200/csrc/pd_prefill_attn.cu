@@ -1,4 +1,5 @@
-// Append-prefill attention over the paged KV cache, and the multi-token KV append.
+// Append-prefill attention over the paged KV cache for head_dim 64, the multi-token KV append, and the launch
+// dispatch of both prefill kernels (head_dim 128 has its own kernel, pd_prefill_attn_d128.cu).
 //
 // Every turn of a multi-turn rollout starts by prefilling the new tokens of the
 // turn (observation plus template, dL per trajectory in the prefill terms of
@@ -8,26 +9,26 @@
 // contraction: 128 query rows share every K/V tile, so it runs on the
 // fifth-generation tensor cores.
 //
-// One CTA (128 softmax threads + one issuing warp) owns 128 rows = 128/g consecutive new tokens x the g
+// One CTA (128 softmax threads + four service warps) owns 128 rows = 128/g consecutive new tokens x the g
 // query heads of one KV head, row = head * (128/g) + token. It walks the context
 // in blocks of 64 tokens (4 pages):
-//   TMA      pages -> shared memory, [half of d][token][128 B] with the 128-byte
+//   TMA      pages -> shared memory, [token][128 B] with the 128-byte
 //            swizzle: K is a K-major operand, V an MN-major one, no transposes;
 //            two stages of K+V; pages past the context are zero-filled
-//   tcgen05  S = Q K^T into tensor memory (8 MMAs of 128x64x16, one thread)
+//   tcgen05  S = Q K^T into tensor memory (4 MMAs of 128x64x16, one thread)
 //   threads  one thread per row: load its 64 logits from tensor memory, mask,
-//            running max with a slack of 8 log2 units, exp2, row sum, P as bf16
-//            back into tensor memory (head_dim 64: a high and a low bf16 part);
+//            running max with a slack of 8 log2 units, exp2, row sum, P as a high and a low bf16
+//            part back into tensor memory (a 64-element output row does not average the 2^-9
+//            rounding of a single bf16 P away when a handful of tokens carry the row);
 //            a rare correction pass rescales O
-//   tcgen05  O += P V (P from tensor memory, 4 MMAs of 128x128x16; head_dim 64:
-//            4 + 4 of 128x64x16 for the two parts of P)
+//   tcgen05  O += P V (P from tensor memory, 4 + 4 MMAs of 128x64x16 for the two parts of P)
 // Four service warps issue the S MMAs, the O MMAs, the TMA loads of K and those
 // of V (one box per lane), so the row threads never run issue code or meet at a
-// CTA barrier: they hand over through mbarriers (logits read, probabilities written). The S MMA of block j+1 is issued as soon as
-// every row holds block j's logits in registers, and two CTAs share each SM (96 KB of shared memory, 256
-// tensor-memory columns each), so one CTA's softmax overlaps the other's MMAs. All waits are
+// CTA barrier: they hand over through mbarriers (logits read, probabilities written). The S MMA of block j+1 is
+// issued as soon as every row holds block j's logits in registers, and two CTAs share each SM (tensor-memory
+// columns 256 each), so one CTA's softmax overlaps the other's MMAs. All waits are
 // bounded; a wait that runs out latches PD_ERR_TIMEOUT and the CTA unwinds and
-// frees its tensor memory.
+// frees its tensor memory. (The kernel is a template over head_dim; only 64 is instantiated.)
 #include "pd_kernels.cuh"
 #include "pd_ptx.cuh"
 #include "pd_tcgen05.cuh"

@@ -13,7 +13,8 @@
 //   TMA      pages -> shared memory as [half of d][token][128 B] with the 128-byte swizzle (K is a K-major
 //            operand, V an MN-major one, no transposes); two K tiles and two V tiles in flight
 //   tcgen05  one issuing thread, order  O0(j) S0(j+1) O1(j) S1(j+1):  S_t = Q_t K^T (8 x 128x128x16) into the
-//            tile's 128 logit columns of tensor memory, O_t += P_t V (8 x 128x128x16, P_t from tensor memory)
+//            tile's 128 logit columns of tensor memory, O_t += P_t V in two parts of 64 tokens (4 x 128x128x16
+//            each, P_t from tensor memory), the first part issued while the row threads work on the second
 //   softmax  one warpgroup per tile, one thread per row: 128 logits -> registers, running max with 8 log2
 //            units of slack, exp2 (a share of the elements on the FMA pipe by a polynomial, the rest on the
 //            special-function unit), P as bf16 over the first 64 columns of the tile's own logit buffer.
@@ -48,9 +49,18 @@ constexpr int kColS = 0, kColO = 256;          // S_t at kColS + 128 t, O_t at k
 // Exponentials per group of 8 logits that run on the FMA pipe as a polynomial instead of the special-function
 // unit (0..8). The two units work side by side inside one warp, which shortens the softmax of a block.
 #ifndef PD_PREFILL_POLY_PER_8
-#define PD_PREFILL_POLY_PER_8 3
+#define PD_PREFILL_POLY_PER_8 2
 #endif
 constexpr int kPolyPer8 = PD_PREFILL_POLY_PER_8;
+
+constexpr int kPParts = 2;                     // P and the O product of a block go in two parts of 64 tokens
+constexpr int kPartKeys = kBlock / kPParts;
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 
 __device__ __forceinline__ void latch(int32_t *status, int code, int seq, int detail) {
     if (atomicCAS(status, kDevOk, code) == kDevOk) {
@@ -136,15 +146,17 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     const uint32_t bar_kfree = smem_u32(bars + 4), bar_vfree = smem_u32(bars + 6);
     // [2] S_t of the current block is in tensor memory (and every earlier product has completed)
     const uint32_t bar_s = smem_u32(bars + 8);
-    // [2] every warp of tile t's warpgroup wrote its rows of P_t
+    // [2 tiles][2 parts] every warp of tile t's warpgroup wrote its rows of that part of P_t. One barrier per part:
+    // the warps of a warpgroup are not in step, and a fast warp's second arrival must not count towards the first
+    // part (with one barrier and two phases per block a waiter that looks late finds the parity it waits for two
+    // phases on and never wakes)
     const uint32_t bar_p = smem_u32(bars + 10);
     // [2] the last O_t product has completed
-    const uint32_t bar_o = smem_u32(bars + 12);
+    const uint32_t bar_o = smem_u32(bars + 14);
 
     if (tid == 0) {
         for (int i = 0; i < 10; ++i) mbar_init(smem_u32(bars + i), 1);
-        mbar_init(bar_p, kRows / 32);
-        mbar_init(bar_p + 8, kRows / 32);
+        for (int i = 0; i < 4; ++i) mbar_init(bar_p + i * 8, kRows / 32);
         mbar_init(bar_o, 1);
         mbar_init(bar_o + 8, 1);
         mbar_init_fence();
@@ -195,14 +207,16 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                 umma_commit(bar_s + t * 8);
                 if (t == kTiles - 1) umma_commit(bar_kfree + (j % kStages) * 8);
             };
-            auto issue_o = [&](int t, int j) {  // O_t += P_t(j) V_j, P_t in the first 64 columns of S_t
-                const uint32_t vst = v_ring + (j % kStages) * kTileBytes;
+            auto issue_o = [&](int t, int j, int part) {  // O_t += P_t(j)[:, part] V_j[part], P_t in the first 64 columns of S_t
+                const uint32_t vst = v_ring + (j % kStages) * kTileBytes + part * (kPartKeys / 16) * 2048;
 #pragma unroll
-                for (int ks = 0; ks < kBlock / 16; ++ks)
-                    umma_ts(tm + kColO + t * kD, tm + kColS + t * kBlock + ks * 8,
-                            umma_smem_desc(vst + ks * 2048, kHalfBytes, 1024), idesc_o, (j | ks) != 0);
-                if (t == kTiles - 1) umma_commit(bar_vfree + (j % kStages) * 8);
-                if (j == nb - 1) umma_commit(bar_o + t * 8);
+                for (int ks = 0; ks < kPartKeys / 16; ++ks)
+                    umma_ts(tm + kColO + t * kD, tm + kColS + t * kBlock + (part * (kPartKeys / 16) + ks) * 8,
+                            umma_smem_desc(vst + ks * 2048, kHalfBytes, 1024), idesc_o, (j | part | ks) != 0);
+                if (part == kPParts - 1) {
+                    if (t == kTiles - 1) umma_commit(bar_vfree + (j % kStages) * 8);
+                    if (j == nb - 1) umma_commit(bar_o + t * 8);
+                }
             };
             ok = mbar_wait(bar_k, 0);
             if (ok) {
@@ -211,21 +225,28 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                 issue_s(1, 0);
             }
             for (int j = 0; j < nb && ok; ++j) {
-                const uint32_t par = (j >> 1) & 1;  // slot j % 2 is in its (j / 2)-th use
-                ok = mbar_wait(bar_p, j & 1) && mbar_wait(bar_v + (j % kStages) * 8, par);
+                ok = mbar_wait(bar_p, j & 1) && mbar_wait(bar_v + (j % kStages) * 8, (j >> 1) & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
-                issue_o(0, j);
+                issue_o(0, j, 0);
+                ok = mbar_wait(bar_p + 8, j & 1);
+                if (!ok) break;
+                tc_fence_after_sync();
+                issue_o(0, j, 1);
                 if (j + 1 < nb) {
                     ok = mbar_wait(bar_k + ((j + 1) % kStages) * 8, ((j + 1) >> 1) & 1);
                     if (!ok) break;
                     tc_fence_after_sync();
                     issue_s(0, j + 1);
                 }
-                ok = mbar_wait(bar_p + 8, j & 1);
+                ok = mbar_wait(bar_p + 16, j & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
-                issue_o(1, j);
+                issue_o(1, j, 0);
+                ok = mbar_wait(bar_p + 24, j & 1);
+                if (!ok) break;
+                tc_fence_after_sync();
+                issue_o(1, j, 1);
                 if (j + 1 < nb) issue_s(1, j + 1);
             }
             if (!ok) latch(p.status, kDevTimeout, b, blockIdx.x);
@@ -308,10 +329,10 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                 float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
                 for (int c = 0; c < kBlock; c += 8) {
-                    m0 = fmaxf(m0, fmaxf(__uint_as_float(s[c]), __uint_as_float(s[c + 1])));
-                    m1 = fmaxf(m1, fmaxf(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])));
-                    m2 = fmaxf(m2, fmaxf(__uint_as_float(s[c + 4]), __uint_as_float(s[c + 5])));
-                    m3 = fmaxf(m3, fmaxf(__uint_as_float(s[c + 6]), __uint_as_float(s[c + 7])));
+                    m0 = max3(m0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+                    m1 = max3(m1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+                    m2 = max3(m2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
+                    m3 = max3(m3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
                 }
                 mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
             }
@@ -335,33 +356,8 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                     tmem_st16(o_buf + c * 16, o);
                 }
             }
-            // ---- exponentials: x = s * scale - m; a share of them by the polynomial on the FMA pipe
-            const float2 nm2 = make_float2(-m_run, -m_run);
-            float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int c0 = 0; c0 < kBlock; c0 += 32) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int c = c0; c < c0 + 32; c += 8) {
-                    float2 e[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[c + 2 * u]), __uint_as_float(s[c + 2 * u + 1])), sc2, nm2);
-                        // pairs 0 .. kPolyPer8/2 - 1 of every eight go to the FMA pipe; an odd share alternates
-                        const bool poly = 2 * u + 1 < kPolyPer8 || (2 * u < kPolyPer8 && ((c >> 3) & 1));
-                        e[u] = poly ? exp2_poly2(x) : make_float2(fast_exp2(x.x), fast_exp2(x.y));
-                    }
-                    acc0 = __fadd2_rn(acc0, __fadd2_rn(e[0], e[1]));
-                    acc1 = __fadd2_rn(acc1, __fadd2_rn(e[2], e[3]));
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) pk[((c - c0) >> 1) + u] = pack_bf16x2(e[u].x, e[u].y);
-                }
-                tmem_st16(s_buf + (c0 >> 1), pk);  // P over the logits this thread already holds in registers
-            }
-            l_run = l_run * alpha + ((acc0.x + acc0.y) + (acc1.x + acc1.y));
-            tmem_wait_st();
             // V rows past the context inside the last page may hold NaN; 0 * NaN is NaN, so tile 0's warpgroup
-            // clears them (both tiles' products of this block are issued after its arrival below)
+            // clears them (both tiles' products of this block are issued after its first arrival below)
             const int valid_rows = L - t0;
             if (t == 0 && valid_rows < kBlock) {
                 const uint32_t vst = v_ring + (j % kStages) * kTileBytes;
@@ -373,9 +369,39 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                 }
                 fence_proxy_async();
             }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_p + t * 8);
+            // ---- exponentials: x = s * scale - m; a share of them by the polynomial on the FMA pipe. P overwrites
+            // the first 64 columns of the logits (all held in registers by now), one part of the block at a time,
+            // so that the first part's product runs while the second part is computed.
+            const float2 nm2 = make_float2(-m_run, -m_run);
+            float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int part = 0; part < kPParts; ++part) {
+#pragma unroll
+                for (int c0 = part * kPartKeys; c0 < (part + 1) * kPartKeys; c0 += 32) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int c = c0; c < c0 + 32; c += 8) {
+                        float2 e[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[c + 2 * u]), __uint_as_float(s[c + 2 * u + 1])), sc2, nm2);
+                            // pairs 0 .. kPolyPer8/2 - 1 of every eight go to the FMA pipe; an odd share alternates
+                            const bool poly = 2 * u + 1 < kPolyPer8 || (2 * u < kPolyPer8 && ((c >> 3) & 1));
+                            e[u] = poly ? exp2_poly2(x) : make_float2(fast_exp2(x.x), fast_exp2(x.y));
+                        }
+                        acc0 = __fadd2_rn(acc0, __fadd2_rn(e[0], e[1]));
+                        acc1 = __fadd2_rn(acc1, __fadd2_rn(e[2], e[3]));
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) pk[((c - c0) >> 1) + u] = pack_bf16x2(e[u].x, e[u].y);
+                    }
+                    tmem_st16(s_buf + (c0 >> 1), pk);
+                }
+                tmem_wait_st();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_p + (t * 2 + part) * 8);
+            }
+            l_run = l_run * alpha + ((acc0.x + acc0.y) + (acc1.x + acc1.y));
         }
 
         // ---- epilogue: O_t / l -> bf16 rows
@@ -411,7 +437,7 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
 
 }  // namespace
 
-size_t prefill_d128_smem_bytes() { return static_cast<size_t>(kTiles) * kQTileBytes + 2 * kStages * kTileBytes + 1024 + 14 * 8 + 64; }
+size_t prefill_d128_smem_bytes() { return static_cast<size_t>(kTiles) * kQTileBytes + 2 * kStages * kTileBytes + 1024 + 16 * 8 + 64; }
 
 cudaError_t prepare_prefill_attn_d128() {
     return cudaFuncSetAttribute(prefill_attn_d128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
