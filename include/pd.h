@@ -145,6 +145,10 @@ int pd_decode_step(pd_ctx *ctx, const void *q, const void *k_new, const void *v_
  * the stream, so out_host is valid on return. The cache itself (k_pages,
  * v_pages, page_table, ctx_lens) stays on the device. If k_new_host starts where
  * q_host ends and v_new_host where k_new_host ends, the three travel in one copy.
+ * A result of at most 256 KB whose buffer is pinned host memory the device can
+ * address is stored there by the merge kernel itself, which then raises a pinned
+ * flag the call polls (no copy-back operation, no stream synchronisation);
+ * larger or pageable results are staged on the device and copied back.
  */
 int pd_decode_step_host(pd_ctx *ctx, const void *q_host, const void *k_new_host, const void *v_new_host,
                         void *k_pages, void *v_pages, const int32_t *page_table, int32_t *ctx_lens,

@@ -43,6 +43,13 @@ int pd_set_profile_events(pd_ctx *ctx, void *before, void *after);
 int pd_read_worker_trace(pd_ctx *ctx, void *stream, uint64_t *host_out, int32_t max_workers, int32_t *num_workers);
 
 /*
+ * How many pd_decode_step_host calls of this context delivered their result straight into the caller's pinned
+ * host buffer (the merge kernel stores the rows and raises a pinned flag the call polls) and how many staged it
+ * on the device and copied it back. Either pointer may be NULL.
+ */
+int pd_host_step_counts(const pd_ctx *ctx, int64_t *direct, int64_t *staged);
+
+/*
  * Read-only streaming probe: launches a kernel of `blocks` x `threads` that reads `bytes` (a multiple of 16
  * is read) from src once with 16-byte streaming loads and stores nothing (sink16 is a 16-byte device
  * buffer the kernel is formally allowed to write). Timed with events by the caller, it gives the read-only

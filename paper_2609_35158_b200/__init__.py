@@ -33,7 +33,7 @@ EXPORTS = (
     "pd_kv_quantize_pages", "pd_kv_append_fp8", "pd_decode_attn_fp8", "pd_decode_step_fp8", "pd_kv_gather_fp8", "pd_kv_scatter_fp8",
     "pd_pool_create", "pd_pool_resize", "pd_pool_base", "pd_pool_capacity", "pd_pool_chunk_bytes", "pd_pool_resident_bytes",
     "pd_pool_last_error", "pd_pool_destroy",
-    "pd_set_profile_events", "pd_read_probe", "pd_workspace_bytes", "pd_launch_count", "pd_last_plan", "pd_status_string", "pd_last_error", "pd_version",
+    "pd_set_profile_events", "pd_read_probe", "pd_host_step_counts", "pd_workspace_bytes", "pd_launch_count", "pd_last_plan", "pd_status_string", "pd_last_error", "pd_version",
 )
 
 
@@ -85,6 +85,7 @@ def _load() -> ctypes.CDLL:
     lib.pd_device_status.argtypes = [vp, vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
     lib.pd_set_profile_events.argtypes = [vp, vp, vp]
     lib.pd_read_probe.argtypes = [vp, ctypes.c_size_t, i32, i32, vp, vp]
+    lib.pd_host_step_counts.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
     lib.pd_read_worker_trace.argtypes = [vp, vp, vp, i32, ctypes.POINTER(i32)]
     lib.pd_workspace_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
     lib.pd_launch_count.argtypes = [vp, ctypes.POINTER(i64)]
@@ -371,6 +372,13 @@ def pd_set_profile_events(ctx, before=None, after=None) -> None:
             ev.record()
         return ev.cuda_event
     _check(_lib.pd_set_profile_events(ctx, handle(before), handle(after)), "pd_set_profile_events", ctx)
+
+
+def pd_host_step_counts(ctx):
+    """(calls whose result went straight to the pinned host buffer, calls that staged it on the device)."""
+    d, s = ctypes.c_int64(0), ctypes.c_int64(0)
+    _check(_lib.pd_host_step_counts(ctx, ctypes.byref(d), ctypes.byref(s)), "pd_host_step_counts", ctx)
+    return int(d.value), int(s.value)
 
 
 def pd_read_probe(src, blocks: int, threads: int, sink, stream=None) -> None:

@@ -3,6 +3,7 @@
 #include "../../include/pd.h"
 #include "../../include/pd_debug.h"
 
+#include <chrono>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -68,6 +69,12 @@ struct pd_ctx {
     const void *map_k8_ptr = nullptr, *map_v8_ptr = nullptr;
     alignas(64) CUtensorMap tm_k8{};
     alignas(64) CUtensorMap tm_v8{};
+    // pd_decode_step_host with pinned host buffers: the merge kernel writes the result to the host itself and
+    // reports completion through this pinned word, which the host polls instead of synchronising the stream
+    int32_t *done_flag_host = nullptr, *done_flag_dev = nullptr;
+    int32_t done_seq = 0;
+    int64_t host_steps_direct = 0, host_steps_staged = 0;
+    __nv_bfloat16 *host_out_alias = nullptr;  // set for the duration of one pd_decode_step_host call
     cudaEvent_t ev_before = nullptr, ev_after = nullptr;  // optional timing hook around the split kernel
     bool prefill_ready = false;
     bool fp8_ready = false;
@@ -263,6 +270,18 @@ int pd_create(const pd_config *cfg, pd_ctx **out) {
         delete ctx;
         return PD_ERR_CUDA;
     }
+    // optional: without the pinned word pd_decode_step_host keeps to copies and a stream synchronisation
+    void *flag = nullptr, *flag_dev = nullptr;
+    if (cudaHostAlloc(&flag, 64, cudaHostAllocMapped) == cudaSuccess) {
+        if (cudaHostGetDevicePointer(&flag_dev, flag, 0) == cudaSuccess) {
+            ctx->done_flag_host = static_cast<int32_t *>(flag);
+            ctx->done_flag_dev = static_cast<int32_t *>(flag_dev);
+            *ctx->done_flag_host = 0;
+        } else {
+            cudaFreeHost(flag);
+        }
+    }
+    (void)cudaGetLastError();
     *out = ctx;
     return PD_OK;
 }
@@ -272,6 +291,7 @@ int pd_destroy(pd_ctx *ctx) {
     DeviceGuard guard(ctx->cfg.device);
     cudaDeviceSynchronize();
     cudaFree(ctx->workspace);
+    if (ctx->done_flag_host != nullptr) cudaFreeHost(ctx->done_flag_host);
     delete ctx;
     return PD_OK;
 }
@@ -432,6 +452,11 @@ int decode_attn_impl(pd_ctx *ctx, const char *who, const void *q, const void *k_
     p.pdl = hooked ? 0 : ctx->pdl;  // timing events must bracket the split kernel alone: no overlap with neighbours
     p.merge_rows = ctx->merge_rows;
     p.trace = ctx->trace;
+    if (ctx->host_out_alias != nullptr) {
+        p.out_host = ctx->host_out_alias;
+        p.done_flag = ctx->done_flag_dev;
+        p.done_value = ctx->done_seq;
+    }
     if (fused) {
         p.k_new = static_cast<const __nv_bfloat16 *>(k_new);
         p.v_new = static_cast<const __nv_bfloat16 *>(v_new);
@@ -753,12 +778,53 @@ int pd_decode_step_host(pd_ctx *ctx, const void *q_host, const void *k_new_host,
         if (err == cudaSuccess) err = cudaMemcpyAsync(dv, v_new_host, nkv, cudaMemcpyHostToDevice, s);
     }
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "host-to-device copy", err);
-    if (int rc = pd_decode_step(ctx, dq, dk, dv, k_pages, v_pages, page_table, ctx_lens,
-                                ctx->stage_out, nullptr, batch, sm_scale, split_pages, stream))
-        return rc;
+    // Result: if out_host is pinned memory the device can address, the merge kernel stores the rows there itself
+    // and raises a pinned flag that this thread polls: no device-to-host copy operation and no stream
+    // synchronisation sit behind the kernels. Otherwise the result is staged and copied.
+    void *out_alias = nullptr;
+    // (Measured on B200: the direct path saves ~15 us of a 270 us step with a 64 KB result and loses ~10 us of a
+    // 420 us step with a 512 KB one, where the copy engine moves the rows faster than the merge kernel's stores
+    // cross PCIe; hence the size limit.)
+    constexpr size_t kDirectResultLimit = 256 * 1024;
+    const bool direct = ctx->done_flag_host != nullptr && nq <= kDirectResultLimit &&
+                        (reinterpret_cast<uintptr_t>(out_host) & 15u) == 0 &&
+                        cudaHostGetDevicePointer(&out_alias, out_host, 0) == cudaSuccess && out_alias != nullptr;
+    if (!direct) (void)cudaGetLastError();
+    if (direct) {
+        ctx->done_seq = ctx->done_seq == 0x7fffffff ? 1 : ctx->done_seq + 1;
+        ctx->host_out_alias = static_cast<__nv_bfloat16 *>(out_alias);
+    }
+    const int rc = pd_decode_step(ctx, dq, dk, dv, k_pages, v_pages, page_table, ctx_lens, ctx->stage_out, nullptr, batch,
+                                  sm_scale, split_pages, stream);
+    ctx->host_out_alias = nullptr;
+    if (rc != PD_OK) return rc;
+    if (direct) {
+        const volatile int32_t *flag = ctx->done_flag_host;
+        const auto t0 = std::chrono::steady_clock::now();
+        for (unsigned spins = 0; *flag != ctx->done_seq; ++spins) {
+            if ((spins & 0xfff) == 0xfff) {
+                if (cudaStreamQuery(s) == cudaSuccess && *flag != ctx->done_seq)  // the stream drained without the flag: a kernel gave up
+                    return fail(ctx, PD_ERR_TIMEOUT, "pd_decode_step_host: the kernels finished without reporting the result");
+                if (std::chrono::steady_clock::now() - t0 > std::chrono::seconds(10)) {
+                    cudaStreamSynchronize(s);
+                    return fail(ctx, PD_ERR_TIMEOUT, "pd_decode_step_host: no completion report within 10 s");
+                }
+            }
+        }
+        ctx->host_steps_direct += 1;
+        return PD_OK;
+    }
     err = cudaMemcpyAsync(out_host, ctx->stage_out, nq, cudaMemcpyDeviceToHost, s);
     if (err == cudaSuccess) err = cudaStreamSynchronize(s);
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "device-to-host copy", err);
+    ctx->host_steps_staged += 1;
+    return PD_OK;
+}
+
+int pd_host_step_counts(const pd_ctx *ctx, int64_t *direct, int64_t *staged) {
+    if (ctx == nullptr) return PD_ERR_INVALID_ARG;
+    if (direct != nullptr) *direct = ctx->host_steps_direct;
+    if (staged != nullptr) *staged = ctx->host_steps_staged;
     return PD_OK;
 }
 

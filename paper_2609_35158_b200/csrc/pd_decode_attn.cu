@@ -450,7 +450,7 @@ __device__ __forceinline__ long long range_of_unit(const int32_t *plan, long lon
 // running (max, sum, output); the warps of a row are then combined through shared memory in warp
 // order. The order of operations is fixed, so reruns are bit-identical.
 template <int D, int WARPS, int R>
-__global__ void __launch_bounds__(WARPS * 32) lse_merge_kernel(const AttnParams p) {
+__device__ __forceinline__ void lse_merge_rows(const AttnParams &p) {
     constexpr int VEC = D / 32;
     constexpr int UNROLL = 8;
     constexpr int S = WARPS / R;  // warps sharing one row
@@ -472,7 +472,8 @@ __global__ void __launch_bounds__(WARPS * 32) lse_merge_kernel(const AttnParams 
         sm_plan[i] = i < kPlanWords ? p.plan[i] : p.cum_pages[b + (i - kPlanWords)];
     __syncthreads();
     const int c0 = sm_plan[kPlanWords], np = sm_plan[kPlanWords + 1] - c0;
-    __nv_bfloat16 *orow = p.out + static_cast<size_t>(row) * D + lane * VEC;
+    // final rows go to the caller's device buffer, or straight to its pinned host buffer when that is given
+    __nv_bfloat16 *orow = (p.out_host != nullptr ? p.out_host : p.out) + static_cast<size_t>(row) * D + lane * VEC;
     if (np == 0) {  // empty context: zero row, lse = -inf
         if (sub == 0) {
 #pragma unroll
@@ -483,7 +484,15 @@ __global__ void __launch_bounds__(WARPS * 32) lse_merge_kernel(const AttnParams 
     }
     const long long u0 = static_cast<long long>(p.Hkv) * c0 + static_cast<long long>(kvh) * np;
     const long long first = range_of_unit(sm_plan, u0), last = range_of_unit(sm_plan, u0 + np - 1);
-    if (first == last) return;  // written directly by the split kernel (the same for every row of the CTA)
+    if (first == last) {  // written directly by the split kernel (the same for every row of the CTA)
+        if (p.out_host != nullptr && sub == 0) {  // forward the row to the host buffer
+            const __nv_bfloat16 *src = p.out + static_cast<size_t>(row) * D + lane * VEC;
+#pragma unroll
+            for (int v = 0; v < VEC; v += 2)
+                *reinterpret_cast<__nv_bfloat162 *>(orow + v) = *reinterpret_cast<const __nv_bfloat162 *>(src + v);
+        }
+        return;
+    }
     const int n = static_cast<int>(last - first) + 1;
     const size_t slot0 = static_cast<size_t>(first) + static_cast<size_t>(b) * p.Hkv + kvh;
 
@@ -552,6 +561,24 @@ __global__ void __launch_bounds__(WARPS * 32) lse_merge_kernel(const AttnParams 
         for (int v = 0; v < VEC; v += 2)
             *reinterpret_cast<__nv_bfloat162 *>(orow + v) = __floats2bfloat162_rn(out[v] * inv, out[v + 1] * inv);
         if (p.lse != nullptr && lane == 0) p.lse[row] = (M + log2f(Lsum)) * kLn2;
+    }
+}
+
+template <int D, int WARPS, int R>
+__global__ void __launch_bounds__(WARPS * 32) lse_merge_kernel(const AttnParams p) {
+    lse_merge_rows<D, WARPS, R>(p);
+    if (p.done_flag != nullptr) {
+        // completion report for a host that polls pinned memory instead of synchronising the stream: every CTA
+        // makes its rows visible system-wide and takes a ticket; the last one stores the flag
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            __threadfence_system();
+            if (atomicAdd(p.status + kMergeDone, 1) == static_cast<int>(gridDim.x) - 1) {
+                p.status[kMergeDone] = 0;
+                __threadfence_system();
+                *reinterpret_cast<volatile int32_t *>(p.done_flag) = p.done_value;
+            }
+        }
     }
 }
 

@@ -16,9 +16,10 @@ constexpr int kMaxLevels = 12;      // levels of the range plan (geometrically s
 // words per level (start lo, start hi, pages per range, index of its first range) plus a closing sentinel
 constexpr int kPlanHeaderWords = 8;
 constexpr int kPlanWords = kPlanHeaderWords + 4 * (kMaxLevels + 1);
-// status[0] code, [1] sequence, [2] detail, [3] unused, [4] next range to claim, [5] workers finished
+// status[0] code, [1] sequence, [2] detail, [3] unused, [4] next range to claim, [5] workers finished,
+// [6] merge CTAs finished (only counted when the merge kernel reports completion to the host itself)
 constexpr int kStatusWords = 8;
-constexpr int kSchedNext = 4, kSchedDone = 5;
+constexpr int kSchedNext = 4, kSchedDone = 5, kMergeDone = 6;
 
 // Device-side fault codes latched in status[0] (first one wins).
 constexpr int kDevOk = 0;
@@ -58,6 +59,12 @@ struct AttnParams {
     uint8_t *k8_w, *v8_w;       // fused append into FP8 pools: the pools and the scale records, writable
     float *scales_w;
     int32_t merge_rows;         // rows per CTA of the merge kernel, 0 = chosen from the row count
+    // Host-visible result (null / 0 otherwise): the merge kernel delivers every final row to out_host, the
+    // device alias of a pinned host buffer [B][Hq][D] (rows the split kernel wrote to `out` are forwarded), and
+    // its last CTA stores done_value to done_flag (device alias of a pinned host word) once all rows are out
+    __nv_bfloat16 *out_host;
+    int32_t *done_flag;
+    int32_t done_value;
     unsigned long long *trace;  // optional [workers][4] ns timestamps: kernel entry, first data, last data, exit
 };
 

@@ -269,6 +269,16 @@ def test_host_step_equals_append_plus_attention():
                                    c2.k_pages, c2.v_pages, c2.page_table, c2.ctx_lens, out_slab, sm_scale=w.sm_scale)
         assert torch.equal(out_slab, out_host)
         assert torch.equal(c2.k_pages, caches[0].k_pages) and torch.equal(c2.v_pages, caches[0].v_pages)
+        # pinned result buffers take the direct path (the merge kernel stores the rows on the host and raises a
+        # flag), a pageable one is staged on the device and copied back: same bits either way
+        direct0, staged0 = ctx.pd.pd_host_step_counts(ctx.h)
+        assert direct0 == 2 and staged0 == 0
+        c3 = wl.build_paged_cache(lens, w.num_kv_heads, w.head_dim, seed=0, device=DEV, reserve_tokens=4)
+        out_pageable = torch.empty((B, w.num_q_heads, w.head_dim), dtype=torch.bfloat16)
+        ctx.pd.pd_decode_step_host(ctx.h, q.cpu(), kn.cpu(), vn.cpu(), c3.k_pages, c3.v_pages, c3.page_table, c3.ctx_lens,
+                                   out_pageable, sm_scale=w.sm_scale)
+        assert ctx.pd.pd_host_step_counts(ctx.h) == (2, 1)
+        assert torch.equal(out_pageable, out_host)
 
 
 def test_bad_page_id_is_reported_not_fatal():
