@@ -15,10 +15,12 @@
 //   tcgen05  one issuing thread, order  O0(j) S0(j+1) O1(j) S1(j+1):  S_t = Q_t K^T (8 x 128x128x16) into the
 //            tile's 128 logit columns of tensor memory, O_t += P_t V in two parts of 64 tokens (4 x 128x128x16
 //            each, P_t from tensor memory), the first part issued while the row threads work on the second
-//   softmax  one warpgroup per tile, one thread per row: 128 logits -> registers, running max with 8 log2
-//            units of slack, exp2 (a share of the elements on the FMA pipe by a polynomial, the rest on the
-//            special-function unit), P as bf16 over the first 64 columns of the tile's own logit buffer.
-//            While tile 0's warpgroup works, the tensor pipe runs tile 1's products, and vice versa.
+//   softmax  one warpgroup per tile, one thread per row, 64 logits (one part) at a time: x = s * scale - m in
+//            registers against the row's running reference m as it stands, the reference raised (and the x
+//            shifted in place) only when a logit exceeds it by more than 8 log2 units, exp2 on the
+//            special-function unit (a polynomial share on the FMA pipe measured slower: the packed FMA
+//            instructions issue at half rate), P as bf16 over the first 64 columns of the tile's own logit
+//            buffer. While tile 0's warpgroup works, the tensor pipe runs tile 1's products, and vice versa.
 // Tensor memory: S0 | S1 | O0 | O1, 128 columns each (all 512). The MMAs of one thread execute in issue order,
 // so "O_t(j) before S_t(j+1)" (P_t lives in S_t's columns) needs no barrier, and a commit that follows S_t(j)
 // also covers O_t(j-1): a row thread that holds S_t(j) may rescale O_t at once. Every wait is bounded; a
@@ -26,6 +28,8 @@
 #include "pd_kernels.cuh"
 #include "pd_ptx.cuh"
 #include "pd_tcgen05.cuh"
+
+#include <type_traits>
 
 namespace pd {
 
@@ -46,15 +50,32 @@ constexpr int kTileBytes = 2 * kHalfBytes;     // 32 KB
 constexpr int kStages = 2;
 constexpr int kTmemCols = 512;
 constexpr int kColS = 0, kColO = 256;          // S_t at kColS + 128 t, O_t at kColO + 128 t
-// Exponentials per group of 8 logits that run on the FMA pipe as a polynomial instead of the special-function
-// unit (0..8). The two units work side by side inside one warp, which shortens the softmax of a block.
-#ifndef PD_PREFILL_POLY_PER_8
-#define PD_PREFILL_POLY_PER_8 2
-#endif
-constexpr int kPolyPer8 = PD_PREFILL_POLY_PER_8;
-
 constexpr int kPParts = 2;                     // P and the O product of a block go in two parts of 64 tokens
 constexpr int kPartKeys = kBlock / kPParts;
+
+// Cycle stamps of CTA (0,0,0) for a timeline of the hand-overs; compiled in only by a profiling build.
+#if defined(PD_ENABLE_TUNING) && defined(PD_PF_LIFE)
+// -DPD_PF_LIFE instead records the life of the first CTAs of the grid, one record of 8 words per CTA:
+// [entry, setup done, first logits, loop end, exit] in ns of the global timer, then block count << 32 | SM id
+__device__ __forceinline__ unsigned long long smid() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(r));
+    return r;
+}
+#define PD_STAMP(region, per_block, j, k)
+#define PD_LIFE(k, v)                                                                                            \
+    if (p.trace != nullptr && life_id * 8 + 8 <= p.trace_ctas * 16) p.trace[life_id * 8 + (k)] = (v);
+#elif defined(PD_ENABLE_TUNING)
+#define PD_LIFE(k, v)
+constexpr int kLogFirst = 8, kLogBlocks = 16;
+#define PD_STAMP(region, per_block, j, k)                                                                       \
+    if (p.trace != nullptr && (blockIdx.x | blockIdx.y | blockIdx.z) == 0 && (j) >= kLogFirst &&                  \
+        (j) < kLogFirst + kLogBlocks)                                                                            \
+        p.trace[1024 * (region) + ((region) >= 3 ? ((threadIdx.x >> 5) & 3) * 64 : 0) + ((j) - kLogFirst) * (per_block) + (k)] = static_cast<unsigned long long>(clock64());
+#else
+#define PD_STAMP(region, per_block, j, k)
+#define PD_LIFE(k, v)
+#endif
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
@@ -87,27 +108,6 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         : "memory");
 }
 
-// 2^x for a pair of arguments on the FMA pipe: x = n + f with n = round(x), f in [-1/2, 1/2]; 2^f by a
-// degree-4 polynomial (relative error 2.6e-6, of the order of ex2.approx), 2^n by adding n to the exponent
-// field. Arguments are clamped at -125 so the exponent field stays positive (the result is then ~1e-38).
-__device__ __forceinline__ float2 exp2_poly2(float2 x) {
-    const float kMagic = 12582912.f;  // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
-    x.x = fmaxf(x.x, -125.f);
-    x.y = fmaxf(x.y, -125.f);
-    const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
-    const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
-    const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
-    float2 p = __ffma2_rn(f, make_float2(0.009570102207362652f, 0.009570102207362652f),
-                          make_float2(0.05591785907745361f, 0.05591785907745361f));
-    p = __ffma2_rn(p, f, make_float2(0.240247443318367f, 0.240247443318367f));
-    p = __ffma2_rn(p, f, make_float2(0.6931217908859253f, 0.6931217908859253f));
-    p = __ffma2_rn(p, f, make_float2(0.9999992847442627f, 0.9999992847442627f));
-    float2 r;
-    r.x = __uint_as_float(__float_as_uint(p.x) + (__float_as_uint(t.x) << 23));
-    r.y = __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(t.y) << 23));
-    return r;
-}
-
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                          const PrefillParams p) {
@@ -120,6 +120,11 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
 
     grid_dependency_wait();
     launch_dependents();
+#if defined(PD_ENABLE_TUNING) && defined(PD_PF_LIFE)
+    const int life_id = tid == 0 ? static_cast<int>(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z)) : 1 << 30;
+    PD_LIFE(0, global_timer_ns())
+    PD_LIFE(5, 0)
+#endif
     const int b = p.order != nullptr ? p.order[blockIdx.z] : static_cast<int>(blockIdx.z);  // heaviest sequences first
     const int q0 = p.q_indptr[b], q_len = p.q_indptr[b + 1] - q0;
     // CTAs are scheduled in index order: start a sequence's last tokens (the longest contexts) first
@@ -151,14 +156,13 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     // part (with one barrier and two phases per block a waiter that looks late finds the parity it waits for two
     // phases on and never wakes)
     const uint32_t bar_p = smem_u32(bars + 10);
-    // [2] the last O_t product has completed
+    // [2] the last O_t product has completed; [2] the first part's O_t product of the current block has completed
     const uint32_t bar_o = smem_u32(bars + 14);
 
     if (tid == 0) {
         for (int i = 0; i < 10; ++i) mbar_init(smem_u32(bars + i), 1);
         for (int i = 0; i < 4; ++i) mbar_init(bar_p + i * 8, kRows / 32);
-        mbar_init(bar_o, 1);
-        mbar_init(bar_o + 8, 1);
+        for (int i = 0; i < 4; ++i) mbar_init(bar_o + i * 8, 1);
         mbar_init_fence();
         prefetch_tensormap(&tm_k);
         prefetch_tensormap(&tm_v);
@@ -188,6 +192,8 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tm = tmem_slot;
+    PD_LIFE(1, global_timer_ns())
+    PD_LIFE(5, (static_cast<unsigned long long>(nb) << 32) | smid())
     bool ok = true;
 
     if (warp == kTiles * 4) {
@@ -216,6 +222,8 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                 if (part == kPParts - 1) {
                     if (t == kTiles - 1) umma_commit(bar_vfree + (j % kStages) * 8);
                     if (j == nb - 1) umma_commit(bar_o + t * 8);
+                } else {
+                    umma_commit(bar_o + (2 + t) * 8);  // lets a row thread rescale O_t between the two parts (rare)
                 }
             };
             ok = mbar_wait(bar_k, 0);
@@ -225,29 +233,41 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                 issue_s(1, 0);
             }
             for (int j = 0; j < nb && ok; ++j) {
+                PD_STAMP(0, 12, j, 0)
                 ok = mbar_wait(bar_p, j & 1) && mbar_wait(bar_v + (j % kStages) * 8, (j >> 1) & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
+                PD_STAMP(0, 12, j, 1)
                 issue_o(0, j, 0);
+                PD_STAMP(0, 12, j, 2)
                 ok = mbar_wait(bar_p + 8, j & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
+                PD_STAMP(0, 12, j, 3)
                 issue_o(0, j, 1);
+                PD_STAMP(0, 12, j, 4)
                 if (j + 1 < nb) {
                     ok = mbar_wait(bar_k + ((j + 1) % kStages) * 8, ((j + 1) >> 1) & 1);
                     if (!ok) break;
                     tc_fence_after_sync();
+                    PD_STAMP(0, 12, j, 5)
                     issue_s(0, j + 1);
+                    PD_STAMP(0, 12, j, 6)
                 }
                 ok = mbar_wait(bar_p + 16, j & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
+                PD_STAMP(0, 12, j, 7)
                 issue_o(1, j, 0);
+                PD_STAMP(0, 12, j, 8)
                 ok = mbar_wait(bar_p + 24, j & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
+                PD_STAMP(0, 12, j, 9)
                 issue_o(1, j, 1);
+                PD_STAMP(0, 12, j, 10)
                 if (j + 1 < nb) issue_s(1, j + 1);
+                PD_STAMP(0, 12, j, 11)
             }
             if (!ok) latch(p.status, kDevTimeout, b, blockIdx.x);
         }
@@ -307,55 +327,14 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         float m_run = -INFINITY, l_run = 0.f;
         const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
         for (int j = 0; j < nb && ok; ++j) {
+            if (row == 0) { PD_STAMP(1 + t, 6, j, 0) }
             ok = mbar_wait(bar_s + t * 8, j & 1);
             tc_fence_after_sync();
-            uint32_t s[kBlock];
-#pragma unroll
-            for (int c = 0; c < kBlock / 32; ++c) tmem_ld32(s_buf + c * 32, *reinterpret_cast<uint32_t(*)[32]>(s + c * 32));
-            tmem_wait_ld();
             if (!ok) break;
-
-            // ---- the row maximum on the raw logits (sm_scale * log2(e) > 0 is folded into the exponent's FMA)
+            if (row == 0) { PD_STAMP(1 + t, 6, j, 1) }
+            if (j == 0) { PD_LIFE(2, global_timer_ns()) }
             const int t0 = j * kBlock;
-            float mx;
-            if (t0 + kBlock - 1 > my_pos) {  // the block reaches past this row's position: mask by select
-                mx = -INFINITY;
-#pragma unroll
-                for (int c = 0; c < kBlock; ++c) {
-                    if (t0 + c > my_pos) s[c] = 0xff800000u;  // -inf
-                    mx = fmaxf(mx, __uint_as_float(s[c]));
-                }
-            } else {  // independent chains instead of one 128-long dependency
-                float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
-#pragma unroll
-                for (int c = 0; c < kBlock; c += 8) {
-                    m0 = max3(m0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
-                    m1 = max3(m1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
-                    m2 = max3(m2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
-                    m3 = max3(m3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
-                }
-                mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-            }
-            mx *= p.scale_log2;
-            float alpha = 1.f;
-            if (mx > m_run + kSlack) {
-                const float m_new = fmaxf(m_run, mx);
-                alpha = fast_exp2(m_run - m_new);
-                m_run = m_new;
-            }
-            // rare: a running max moved by more than the slack, so O_t must be rescaled. The commit that announced
-            // S_t(j) also covers O_t(j-1), and O_t(j) is not issued before this warp has arrived on bar_p.
-            if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll 1
-                for (int c = 0; c < kD / 16; ++c) {
-                    uint32_t o[16];
-                    tmem_ld16(o_buf + c * 16, o);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                    tmem_st16(o_buf + c * 16, o);
-                }
-            }
+            const bool masked = t0 + kBlock - 1 > my_pos;  // the block reaches past this row's position
             // V rows past the context inside the last page may hold NaN; 0 * NaN is NaN, so tile 0's warpgroup
             // clears them (both tiles' products of this block are issued after its first arrival below)
             const int valid_rows = L - t0;
@@ -369,42 +348,113 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                 }
                 fence_proxy_async();
             }
-            // ---- exponentials: x = s * scale - m; a share of them by the polynomial on the FMA pipe. P overwrites
-            // the first 64 columns of the logits (all held in registers by now), one part of the block at a time,
-            // so that the first part's product runs while the second part is computed.
-            const float2 nm2 = make_float2(-m_run, -m_run);
-            float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+            // ---- one part of 64 tokens at a time, in two passes over registers. Pass 1: x = s * scale - m against
+            // the running reference m of the row AS IT STANDS, in place, and the largest x. Only if that exceeds the
+            // slack (rare; the first part of the first block always, its reference is a placeholder) is the
+            // reference raised by it: what the row has accumulated is rescaled and the x are shifted in their
+            // registers, nothing is recomputed. Pass 2: exponentials, row sum, P stored 32 tokens at a time so the
+            // stores overlap the arithmetic. Blocks no row of the warp sees masked (all but the last one or two)
+            // run a copy without the mask selects.
+            float blk_sum = 0.f;
+            auto do_part = [&](auto masked_c, int part) {
+                constexpr bool kMasked = decltype(masked_c)::value;
+                const bool first = j == 0 && part == 0;
+                uint32_t sreg[kPartKeys];
 #pragma unroll
-            for (int part = 0; part < kPParts; ++part) {
+                for (int c = 0; c < kPartKeys / 32; ++c)
+                    tmem_ld32(s_buf + part * kPartKeys + c * 32, *reinterpret_cast<uint32_t(*)[32]>(sreg + c * 32));
+                tmem_wait_ld();
+                if (row == 0 && part == 0) { PD_STAMP(1 + t, 6, j, 2) }
+                if (kMasked) {  // mask by select: masked logits become -inf, their exponentials exact zeros
+                    const int visible = my_pos - (t0 + part * kPartKeys) + 1;  // logits of this part the row may see
 #pragma unroll
-                for (int c0 = part * kPartKeys; c0 < (part + 1) * kPartKeys; c0 += 32) {
+                    for (int c = 0; c < kPartKeys; ++c)
+                        if (c >= visible) sreg[c] = 0xff800000u;
+                }
+                if (first) m_run = 0.f;  // placeholder; the branch below replaces it by the part's maximum
+                float x[kPartKeys];
+                {
+                    const float2 nm2 = make_float2(-m_run, -m_run);
+                    float xm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                    for (int c = 0; c < kPartKeys; c += 4) {
+                        const float2 u = __ffma2_rn(make_float2(__uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1])), sc2, nm2);
+                        const float2 v = __ffma2_rn(make_float2(__uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3])), sc2, nm2);
+                        x[c] = u.x, x[c + 1] = u.y, x[c + 2] = v.x, x[c + 3] = v.y;
+                        xm[(c >> 2) & 1] = max3(xm[(c >> 2) & 1], u.x, u.y);
+                        xm[2 + ((c >> 2) & 1)] = max3(xm[2 + ((c >> 2) & 1)], v.x, v.y);
+                    }
+                    const float xmax = fmaxf(fmaxf(xm[0], xm[1]), fmaxf(xm[2], xm[3]));
+                    if (first || __any_sync(0xffffffffu, xmax > kSlack)) {
+                        float shift = 0.f, alpha = 1.f;
+                        if (first || xmax > kSlack) {  // position 0 is visible to every row, so the first maximum is finite
+                            shift = xmax;
+                            alpha = fast_exp2(-xmax);
+                            m_run += xmax;
+                        }
+                        if (!first) {
+                            if (part > 0) {  // the first part's product of this block must be over before O_t is touched
+                                ok = ok && mbar_wait(bar_o + (2 + t) * 8, j & 1);
+                                tc_fence_after_sync();
+                            }
+                            // the commit that announced S_t(j) also covers O_t(j-1)
+#pragma unroll 1
+                            for (int c = 0; c < kD / 16; ++c) {
+                                uint32_t o[16];
+                                tmem_ld16(o_buf + c * 16, o);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                                tmem_st16(o_buf + c * 16, o);
+                            }
+                            tmem_wait_st();
+                            l_run *= alpha;
+                            blk_sum *= alpha;
+                        }
+                        const float2 ns2 = make_float2(-shift, -shift);
+#pragma unroll
+                        for (int c = 0; c < kPartKeys; c += 2) {
+                            const float2 u = __fadd2_rn(make_float2(x[c], x[c + 1]), ns2);
+                            x[c] = u.x, x[c + 1] = u.y;
+                        }
+                    }
+                }
+                float2 a0 = make_float2(0.f, 0.f), a1 = make_float2(0.f, 0.f);
+#pragma unroll
+                for (int c0 = 0; c0 < kPartKeys; c0 += 32) {
                     uint32_t pk[16];
 #pragma unroll
                     for (int c = c0; c < c0 + 32; c += 8) {
                         float2 e[4];
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[c + 2 * u]), __uint_as_float(s[c + 2 * u + 1])), sc2, nm2);
-                            // pairs 0 .. kPolyPer8/2 - 1 of every eight go to the FMA pipe; an odd share alternates
-                            const bool poly = 2 * u + 1 < kPolyPer8 || (2 * u < kPolyPer8 && ((c >> 3) & 1));
-                            e[u] = poly ? exp2_poly2(x) : make_float2(fast_exp2(x.x), fast_exp2(x.y));
-                        }
-                        acc0 = __fadd2_rn(acc0, __fadd2_rn(e[0], e[1]));
-                        acc1 = __fadd2_rn(acc1, __fadd2_rn(e[2], e[3]));
+                        for (int u = 0; u < 4; ++u) e[u] = make_float2(fast_exp2(x[c + 2 * u]), fast_exp2(x[c + 2 * u + 1]));
+                        a0 = __fadd2_rn(a0, __fadd2_rn(e[0], e[1]));
+                        a1 = __fadd2_rn(a1, __fadd2_rn(e[2], e[3]));
 #pragma unroll
                         for (int u = 0; u < 4; ++u) pk[((c - c0) >> 1) + u] = pack_bf16x2(e[u].x, e[u].y);
                     }
-                    tmem_st16(s_buf + (c0 >> 1), pk);
+                    // P over the first 64 columns of the tile's logit buffer (columns this thread has already consumed)
+                    tmem_st16(s_buf + ((part * kPartKeys + c0) >> 1), pk);
                 }
+                blk_sum += (a0.x + a0.y) + (a1.x + a1.y);
                 tmem_wait_st();
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_p + (t * 2 + part) * 8);
+                if (row == 0) { PD_STAMP(1 + t, 6, j, 3 + part) }
+            };
+            if (__any_sync(0xffffffffu, masked)) {
+                do_part(std::true_type{}, 0);
+                do_part(std::true_type{}, 1);
+            } else {
+                do_part(std::false_type{}, 0);
+                do_part(std::false_type{}, 1);
             }
-            l_run = l_run * alpha + ((acc0.x + acc0.y) + (acc1.x + acc1.y));
+            l_run += blk_sum;
         }
 
         // ---- epilogue: O_t / l -> bf16 rows
+        PD_LIFE(3, global_timer_ns())
         if (ok) ok = mbar_wait(bar_o + t * 8, 0);
         tc_fence_after_sync();
         const float inv = 1.f / l_run;
@@ -433,11 +483,12 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tm, kTmemCols);
+    PD_LIFE(4, global_timer_ns())
 }
 
 }  // namespace
 
-size_t prefill_d128_smem_bytes() { return static_cast<size_t>(kTiles) * kQTileBytes + 2 * kStages * kTileBytes + 1024 + 16 * 8 + 64; }
+size_t prefill_d128_smem_bytes() { return static_cast<size_t>(kTiles) * kQTileBytes + 2 * kStages * kTileBytes + 1024 + 18 * 8 + 64; }
 
 cudaError_t prepare_prefill_attn_d128() {
     return cudaFuncSetAttribute(prefill_attn_d128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
