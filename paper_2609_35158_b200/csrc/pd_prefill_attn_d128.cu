@@ -232,28 +232,28 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                 issue_s(0, 0);
                 issue_s(1, 0);
             }
+            // Nothing queues behind the tensor pipe: a cycle this thread spends between two products is a cycle the
+            // pipe idles (a satisfied mbarrier wait costs it ~90). So the waits that are satisfied long before they
+            // are needed (the V tile of this block, the K tile of the next) are taken just ahead of a wait on P,
+            // where the thread would be standing anyway.
             for (int j = 0; j < nb && ok; ++j) {
                 PD_STAMP(0, 12, j, 0)
-                ok = mbar_wait(bar_p, j & 1) && mbar_wait(bar_v + (j % kStages) * 8, (j >> 1) & 1);
+                ok = mbar_wait(bar_v + (j % kStages) * 8, (j >> 1) & 1) && mbar_wait(bar_p, j & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
                 PD_STAMP(0, 12, j, 1)
                 issue_o(0, j, 0);
                 PD_STAMP(0, 12, j, 2)
-                ok = mbar_wait(bar_p + 8, j & 1);
+                if (j + 1 < nb) ok = mbar_wait(bar_k + ((j + 1) % kStages) * 8, ((j + 1) >> 1) & 1);
+                ok = ok && mbar_wait(bar_p + 8, j & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
                 PD_STAMP(0, 12, j, 3)
                 issue_o(0, j, 1);
                 PD_STAMP(0, 12, j, 4)
-                if (j + 1 < nb) {
-                    ok = mbar_wait(bar_k + ((j + 1) % kStages) * 8, ((j + 1) >> 1) & 1);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    PD_STAMP(0, 12, j, 5)
-                    issue_s(0, j + 1);
-                    PD_STAMP(0, 12, j, 6)
-                }
+                PD_STAMP(0, 12, j, 5)
+                if (j + 1 < nb) issue_s(0, j + 1);
+                PD_STAMP(0, 12, j, 6)
                 ok = mbar_wait(bar_p + 16, j & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
@@ -356,15 +356,14 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
             // stores overlap the arithmetic. Blocks no row of the warp sees masked (all but the last one or two)
             // run a copy without the mask selects.
             float blk_sum = 0.f;
-            auto do_part = [&](auto masked_c, int part) {
-                constexpr bool kMasked = decltype(masked_c)::value;
-                const bool first = j == 0 && part == 0;
-                uint32_t sreg[kPartKeys];
+            auto load_part = [&](int part, uint32_t (&sreg)[kPartKeys]) {
 #pragma unroll
                 for (int c = 0; c < kPartKeys / 32; ++c)
                     tmem_ld32(s_buf + part * kPartKeys + c * 32, *reinterpret_cast<uint32_t(*)[32]>(sreg + c * 32));
-                tmem_wait_ld();
-                if (row == 0 && part == 0) { PD_STAMP(1 + t, 6, j, 2) }
+            };
+            auto pass1 = [&](auto masked_c, int part, uint32_t (&sreg)[kPartKeys], float (&x)[kPartKeys]) {
+                constexpr bool kMasked = decltype(masked_c)::value;
+                const bool first = j == 0 && part == 0;
                 if (kMasked) {  // mask by select: masked logits become -inf, their exponentials exact zeros
                     const int visible = my_pos - (t0 + part * kPartKeys) + 1;  // logits of this part the row may see
 #pragma unroll
@@ -372,7 +371,6 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                         if (c >= visible) sreg[c] = 0xff800000u;
                 }
                 if (first) m_run = 0.f;  // placeholder; the branch below replaces it by the part's maximum
-                float x[kPartKeys];
                 {
                     const float2 nm2 = make_float2(-m_run, -m_run);
                     float xm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -419,6 +417,8 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                         }
                     }
                 }
+            };
+            auto pass2 = [&](int part, float (&x)[kPartKeys]) {
                 float2 a0 = make_float2(0.f, 0.f), a1 = make_float2(0.f, 0.f);
 #pragma unroll
                 for (int c0 = 0; c0 < kPartKeys; c0 += 32) {
@@ -443,13 +443,22 @@ prefill_attn_d128_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                 if (lane == 0) mbar_arrive(bar_p + (t * 2 + part) * 8);
                 if (row == 0) { PD_STAMP(1 + t, 6, j, 3 + part) }
             };
-            if (__any_sync(0xffffffffu, masked)) {
-                do_part(std::true_type{}, 0);
-                do_part(std::true_type{}, 1);
-            } else {
-                do_part(std::false_type{}, 0);
-                do_part(std::false_type{}, 1);
-            }
+            // the second part's logits are fetched while the first part's exponentials run
+            auto do_block = [&](auto masked_c) {
+                uint32_t sa[kPartKeys], sb[kPartKeys];
+                float x[kPartKeys];
+                load_part(0, sa);
+                tmem_wait_ld();
+                if (row == 0) { PD_STAMP(1 + t, 6, j, 2) }
+                pass1(masked_c, 0, sa, x);
+                load_part(1, sb);
+                pass2(0, x);
+                tmem_wait_ld();
+                pass1(masked_c, 1, sb, x);
+                pass2(1, x);
+            };
+            if (__any_sync(0xffffffffu, masked)) do_block(std::true_type{});
+            else do_block(std::false_type{});
             l_run += blk_sum;
         }
 
