@@ -398,9 +398,10 @@ int pd_decode_attn_fp8(pd_ctx *ctx, const void *q, const void *k8, const void *v
                        int32_t batch, float sm_scale, int32_t split_pages, void *stream);
 
 /*
- * pd_decode_step for FP8 pools: pd_kv_append_fp8 (advancing) followed by pd_decode_attn_fp8 in two launches,
- * with the append inside the split kernel; pools, scale records, lengths, output and LSE are bit-identical to
- * the two-call path. ctx_lens holds the lengths BEFORE the append on entry. Errors as pd_decode_step.
+ * pd_decode_step for FP8 pools: pd_kv_append_fp8 (advancing) followed by pd_decode_attn_fp8, enqueued by one
+ * call (append, split and merge kernels; a split kernel that also quantised the new token measured slower and
+ * is not built). Arguments are validated before anything is enqueued; results are those of the two calls.
+ * ctx_lens holds the lengths BEFORE the append on entry. Errors as pd_kv_append_fp8 and pd_decode_attn_fp8.
  */
 int pd_decode_step_fp8(pd_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *k8, void *v8,
                        float *kv_scales, const int32_t *page_table, int32_t *ctx_lens, void *out, float *lse,

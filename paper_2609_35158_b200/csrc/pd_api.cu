@@ -560,17 +560,25 @@ int pd_kv_append_fp8(pd_ctx *ctx, const void *k_new, const void *v_new, void *k8
 
 namespace {
 
-int decode_attn_fp8_impl(pd_ctx *ctx, const void *q, const void *k_new, const void *v_new, const void *k8, const void *v8,
-                         const float *kv_scales, const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse,
-                         int32_t batch, float sm_scale, int32_t split_pages, void *stream) {
-    const bool fused = k_new != nullptr;
+constexpr int32_t kFp8StaticFairMax = 1024;  // pages per worker up to which the FP8 split kernel takes one equal range per worker
+
+int fp8_attn_check_args(pd_ctx *ctx, const void *q, const void *k8, const void *v8, const float *kv_scales,
+                        const int32_t *page_table, const int32_t *ctx_lens, const void *out, int32_t batch, float sm_scale,
+                        int32_t split_pages) {
     if (int rc = check_batch(ctx, batch)) return rc;
     if (ctx->cfg.head_dim != 128) return fail(ctx, PD_ERR_UNSUPPORTED, "FP8 attention: head_dim must be 128");
     if (!aligned16(q) || !aligned16(k8) || !aligned16(v8) || !aligned16(kv_scales) || !aligned16(out) ||
-        page_table == nullptr || ctx_lens == nullptr || (fused && (!aligned16(k_new) || !aligned16(v_new))))
+        page_table == nullptr || ctx_lens == nullptr)
         return fail(ctx, PD_ERR_INVALID_ARG, "FP8 attention: null or misaligned pointer");
     if (!(sm_scale > 0.f) || !(sm_scale < 3.0e38f)) return fail(ctx, PD_ERR_INVALID_ARG, "sm_scale must be finite and positive");
     if (split_pages < 0) return fail(ctx, PD_ERR_INVALID_ARG, "split_pages must be >= 0");
+    return PD_OK;
+}
+
+int decode_attn_fp8_impl(pd_ctx *ctx, const void *q, const void *k8, const void *v8, const float *kv_scales,
+                         const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse, int32_t batch,
+                         float sm_scale, int32_t split_pages, void *stream) {
+    if (int rc = fp8_attn_check_args(ctx, q, k8, v8, kv_scales, page_table, ctx_lens, out, batch, sm_scale, split_pages)) return rc;
     if (batch == 0) return PD_OK;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
@@ -590,15 +598,6 @@ int decode_attn_fp8_impl(pd_ctx *ctx, const void *q, const void *k_new, const vo
     pd::AttnParams p{};
     p.q = static_cast<const __nv_bfloat16 *>(q);
     p.kv_scales = kv_scales;
-    if (fused) {
-        p.k_new = static_cast<const __nv_bfloat16 *>(k_new);
-        p.v_new = static_cast<const __nv_bfloat16 *>(v_new);
-        p.k8_w = static_cast<uint8_t *>(const_cast<void *>(k8));
-        p.v8_w = static_cast<uint8_t *>(const_cast<void *>(v8));
-        p.scales_w = const_cast<float *>(kv_scales);
-        p.ctx_lens_w = const_cast<int32_t *>(ctx_lens);
-        p.fused = 1;
-    }
     p.page_table = page_table;
     p.ctx_lens = ctx_lens;
     p.out = static_cast<__nv_bfloat16 *>(out);
@@ -620,9 +619,14 @@ int decode_attn_fp8_impl(pd_ctx *ctx, const void *q, const void *k_new, const vo
     p.min_pages_auto = ctx->min_pages_auto;
     p.halving_levels = ctx->halving_levels;
     p.tail_pages = ctx->tail_pages;
+    // Measured on configs[1..4] (call of split + merge, us): equal ranges 129 / 181 / 416 / 2168 against 138 / 196 /
+    // 443 / 2139 for the halving plan, the opposite of the bf16 kernel (263 / 390 / 858 / 4075 against 236 / 345 /
+    // 766 / 3623), whose workers differ in speed with their SM's distance to the memory they read.
+    p.static_fair_max = kFp8StaticFairMax;
     const bool hooked = ctx->ev_before != nullptr;
     p.pdl = hooked ? 0 : ctx->pdl;
     p.merge_rows = ctx->merge_rows;
+    p.trace = ctx->trace;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (hooked) cudaEventRecord(ctx->ev_before, s);
     cudaError_t err = pd::launch_decode_attn_fp8(ctx->tm_k8, ctx->tm_v8, p, ctx->num_ctas, s);
@@ -645,8 +649,7 @@ extern "C" {
 int pd_decode_attn_fp8(pd_ctx *ctx, const void *q, const void *k8, const void *v8, const float *kv_scales,
                        const int32_t *page_table, const int32_t *ctx_lens, void *out, float *lse, int32_t batch,
                        float sm_scale, int32_t split_pages, void *stream) {
-    return decode_attn_fp8_impl(ctx, q, nullptr, nullptr, k8, v8, kv_scales, page_table, ctx_lens, out, lse, batch, sm_scale,
-                                split_pages, stream);
+    return decode_attn_fp8_impl(ctx, q, k8, v8, kv_scales, page_table, ctx_lens, out, lse, batch, sm_scale, split_pages, stream);
 }
 
 int pd_decode_step_fp8(pd_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *k8, void *v8,
@@ -654,8 +657,11 @@ int pd_decode_step_fp8(pd_ctx *ctx, const void *q, const void *k_new, const void
                        int32_t batch, float sm_scale, int32_t split_pages, void *stream) {
     if (ctx == nullptr) return PD_ERR_INVALID_ARG;
     if (k_new == nullptr || v_new == nullptr) return fail(ctx, PD_ERR_INVALID_ARG, "pd_decode_step_fp8: null k_new / v_new");
-    return decode_attn_fp8_impl(ctx, q, k_new, v_new, k8, v8, kv_scales, page_table, ctx_lens, out, lse, batch, sm_scale,
-                                split_pages, stream);
+    // Two launches (three with the merge). A split kernel that also quantised and patched the new token measured
+    // slower than this on every configuration (137 against 127 us on configs[3]), so there is none.
+    if (int rc = fp8_attn_check_args(ctx, q, k8, v8, kv_scales, page_table, ctx_lens, out, batch, sm_scale, split_pages)) return rc;
+    if (int rc = pd_kv_append_fp8(ctx, k_new, v_new, k8, v8, kv_scales, page_table, ctx_lens, batch, 0u, stream)) return rc;
+    return decode_attn_fp8_impl(ctx, q, k8, v8, kv_scales, page_table, ctx_lens, out, lse, batch, sm_scale, split_pages, stream);
 }
 
 int pd_kv_append_tokens(pd_ctx *ctx, const void *k_new, const void *v_new, const int32_t *q_indptr, void *k_pages,

@@ -17,8 +17,9 @@
 //     k_scale times sm_scale log2(e) multiplies the fp32 logits;
 //   * for O^T += V^T P^T, ldmatrix.trans delivers (token 2t, token 2t+1) x (d, d+1) in one register; one
 //     byte permute regroups it into the two fp16 pairs the A operand wants. P is fp16 (11 significant
-//     bits, no high/low split needed). The page's product goes to a temporary accumulator that is added
-//     to O with v_scale in fp32: folding v_scale into the fp16 P would flush small probabilities.
+//     bits, no high/low split needed). v_scale is folded into P relative to the largest scale of the segment
+//     so far (O is kept in that unit and rescaled when a larger scale arrives), so the page's product
+//     accumulates straight into O: no temporary accumulator, no per-element multiply.
 // head_dim 128 and |q| below the fp16 range (65504) are required.
 #include "pd_decode_plan.cuh"
 #include "pd_kernels.cuh"
@@ -41,18 +42,7 @@ __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) {
     return *reinterpret_cast<const uint32_t *>(&h);
 }
 
-__device__ __forceinline__ uint32_t quantize4(const float (&x)[4], float scale) {
-    // IEEE division (the build uses fast-math, so spell it out), round to nearest even, saturate: as kv_append_fp8_kernel
-    const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(x[0], scale), __fdiv_rn(x[1], scale)), __NV_SATFINITE, __NV_E4M3);
-    const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(x[2], scale), __fdiv_rn(x[3], scale)), __NV_SATFINITE, __NV_E4M3);
-    return lo | (hi << 16);
-}
-
-// FUSED: ctx_lens holds the lengths before a one-token append; the worker that reads a pair's last page
-// quantises the new token's rows exactly as kv_append_fp8_kernel does (a token that opens a page sets the
-// page's scales), writes them to the pools and patches them into the tile it is about to use; the last
-// worker to finish advances the lengths.
-template <int WARPS, int STAGES, bool FUSED>
+template <int WARPS, int STAGES>
 __global__ void __launch_bounds__(WARPS * 32, 1)
 decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                              const AttnParams p) {
@@ -70,11 +60,16 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
     uint64_t *bars = reinterpret_cast<uint64_t *>(scale_slots + WARPS * STAGES);
     Plan *plan_s = reinterpret_cast<Plan *>(bars + WARPS * STAGES * 2);
     int32_t *stage_range = reinterpret_cast<int32_t *>(plan_s + 1);
-    int32_t *stage_pid = stage_range + WARPS * STAGES;  // physical page in a stage, -1 if its id was out of range
-    int32_t *warp_sums = stage_pid + WARPS * STAGES;
+    int32_t *warp_sums = stage_range + WARPS * STAGES;
     int32_t *cum = warp_sums + 32;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+#ifdef PD_ENABLE_TUNING
+    // profiling build only (the kernel has no register to spare): per worker two words, the low 32 bits of
+    // {entry, first data} and {last data, exit} in ns
+    const unsigned long long t_entry = p.trace != nullptr ? global_timer_ns() : 0ull;
+    unsigned long long t_first = 0ull, t_last = 0ull;
+#endif
 
     launch_dependents();
     if (lane == 0) {
@@ -116,7 +111,6 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
     const uint32_t scale0 = smem_u32(scale_slots + warp * STAGES);
     const float4 *my_scales = scale_slots + warp * STAGES;
     int32_t *my_stage_range = stage_range + warp * STAGES;
-    int32_t *my_stage_pid = stage_pid + warp * STAGES;
     const uint64_t policy = l2_policy_evict_first();
     const int quad_row = lane >> 2;       // g: token row of the accumulators; head whose Q this lane holds as B operand
     const int quad_t = lane & 3;          // t
@@ -174,7 +168,6 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
             const uint32_t bk = bar0 + p_stage * 16, bv = bk + 8;
             if (lane == 0) {
                 my_stage_range[p_stage] = p_rid;
-                if (FUSED) my_stage_pid[p_stage] = pid_ok ? pid : -1;
                 mbar_arrive_expect_tx(bk, TILE_BYTES + 16);
                 mbar_arrive_expect_tx(bv, TILE_BYTES);
             }
@@ -203,13 +196,18 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
     cons.b = 0; cons.kvh = 0; cons.page = 0; cons.np = 1;
     int c_rid = -1, c_left = 0;
     uint32_t stage = 0, parity = 0;
-    bool alive = true, seg_open = false, seg_append = false;
+    bool alive = true, seg_open = false;
     int seg_page0 = 0, L = 0;
     // Q^T as the fp16 B operand: for chunk c, head quad_row, d = 16 c + 4 t + {0, 1} and + {2, 3}
     uint32_t qb[CHUNKS][2];
     // O^T: for chunk c, rows d = 16 c + 2 g (regs 0, 1) and 16 c + 2 g + 1 (regs 2, 3), columns heads quad_col, quad_col + 1
     float O[CHUNKS][4];
     float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
+    // O is kept in units of v_ref, the largest |v_scale| the segment has met: a page's probabilities go to the
+    // tensor core as p * v_scale / v_ref (fp32 product, at most p, then fp16), so its product accumulates
+    // straight into O. What fp16 drops of a page whose scale is far below v_ref is below 2^-25 of v_ref per
+    // code unit, i.e. nothing against the pages that set v_ref.
+    float v_ref = 0.f;
 
     while (inflight > 0) {
         if (c_left == 0) {
@@ -221,9 +219,7 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
         if (!seg_open) {
             seg_open = true;
             seg_page0 = cons.page;
-            const int L_raw = __ldg(p.ctx_lens + cons.b) + (FUSED ? 1 : 0);
-            L = clamp_len(L_raw, p.MP);
-            seg_append = FUSED && L == L_raw && L > 0;  // never patch a row of a length that was clamped
+            L = clamp_len(__ldg(p.ctx_lens + cons.b), p.MP);
             const __nv_bfloat16 *qrow = p.q + (static_cast<size_t>(cons.b) * p.Hq + cons.kvh * G + quad_row) * D;
 #pragma unroll
             for (int c = 0; c < CHUNKS; ++c) {
@@ -240,6 +236,7 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
             for (int c = 0; c < CHUNKS; ++c) { O[c][0] = 0.f; O[c][1] = 0.f; O[c][2] = 0.f; O[c][3] = 0.f; }
             m_a = -INFINITY; m_b = -INFINITY;
             l_a = 0.f; l_b = 0.f;
+            v_ref = 0.f;
         }
 
         const uint32_t kbase = ring + stage * STAGE_BYTES;
@@ -247,56 +244,14 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
         const uint32_t bk = bar0 + stage * 16, bv = bk + 8;
         const int valid = L - cons.page * kPageSize;
 
-        // fused append: this lane's four values of the new K row and of the new V row (d = 4 lane .. 4 lane + 3)
-        const bool appending = FUSED && seg_append && cons.page == cons.np - 1;
-        const int new_slot = (L - 1) & (kPageSize - 1);
-        float kx[4] = {0.f, 0.f, 0.f, 0.f}, vx[4] = {0.f, 0.f, 0.f, 0.f};
-        if (appending) {
-            const size_t row = (static_cast<size_t>(cons.b) * p.Hkv + cons.kvh) * D + lane * 4;
-            const uint2 kw = __ldg(reinterpret_cast<const uint2 *>(p.k_new + row));
-            const uint2 vw = __ldg(reinterpret_cast<const uint2 *>(p.v_new + row));
-            const float2 k01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&kw.x));
-            const float2 k23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&kw.y));
-            const float2 v01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&vw.x));
-            const float2 v23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&vw.y));
-            kx[0] = k01.x; kx[1] = k01.y; kx[2] = k23.x; kx[3] = k23.y;
-            vx[0] = v01.x; vx[1] = v01.y; vx[2] = v23.x; vx[3] = v23.y;
-        }
         if (!__all_sync(0xffffffffu, mbar_wait(bk, parity))) { alive = false; break; }
-        float4 sc = my_scales[stage];  // {k_scale, v_scale, -, -} of this page
-        uint32_t new_v8 = 0u;
-        if (appending) {
-            if (new_slot == 0) {  // the token opens the page: it sets both scales, with a factor two of headroom
-                float ak = 0.f, av = 0.f;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float a = fabsf(kx[i]), b2 = fabsf(vx[i]);
-                    if (a > ak) ak = a;  // NaN never wins
-                    if (b2 > av) av = b2;
-                }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    ak = fmaxf(ak, __shfl_xor_sync(0xffffffffu, ak, o));
-                    av = fmaxf(av, __shfl_xor_sync(0xffffffffu, av, o));
-                }
-                sc.x = ak > 0.f ? __fdiv_rn(ak * 2.f, 448.f) : 1.f;
-                sc.y = av > 0.f ? __fdiv_rn(av * 2.f, 448.f) : 1.f;
-            }
-            const uint32_t new_k8 = quantize4(kx, sc.x);
-            new_v8 = quantize4(vx, sc.y);
-            const int pid = my_stage_pid[stage];
-            if (pid >= 0) {  // the append itself
-                const size_t tile = static_cast<size_t>(pid) * p.Hkv + cons.kvh;
-                const size_t at = (tile * kPageSize + new_slot) * D + lane * 4;
-                *reinterpret_cast<uint32_t *>(p.k8_w + at) = new_k8;
-                *reinterpret_cast<uint32_t *>(p.v8_w + at) = new_v8;
-                if (new_slot == 0 && lane == 0) *reinterpret_cast<float4 *>(p.scales_w + tile * 4) = make_float4(sc.x, sc.y, 0.f, 0.f);
-            }
-            // the tile in shared memory still holds whatever the pool had in that slot: patch the K row now
-            const uint32_t a = kbase + new_slot * 128 + ((((lane >> 2) ^ (new_slot & 7)) << 4)) + (lane & 3) * 4;
-            asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(new_k8) : "memory");
-            __syncwarp();
+#ifdef PD_ENABLE_TUNING
+        if (p.trace != nullptr) {
+            t_last = global_timer_ns();
+            if (t_first == 0ull) t_first = t_last;
         }
+#endif
+        const float4 sc = my_scales[stage];  // {k_scale, v_scale, -, -} of this page
 
         // S^T = K8 Q^T: one ldmatrix.x4 feeds two MMAs (two 16-byte chunks of d)
         float Se[4] = {0.f, 0.f, 0.f, 0.f}, So[4] = {0.f, 0.f, 0.f, 0.f};
@@ -339,24 +294,26 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
         const float p2 = fast_exp2(s2 - m_a), p3 = fast_exp2(s3 - m_b);
         l_a += p0 + p2;
         l_b += p1 + p3;
+        if (fabsf(sc.y) > v_ref) {  // the page's scale, so the whole warp branches together; rare after the first pages
+            const float r = v_ref / fabsf(sc.y);  // 0 at the first page, where O is 0 anyway
+#pragma unroll
+            for (int c = 0; c < CHUNKS; ++c) { O[c][0] *= r; O[c][1] *= r; O[c][2] *= r; O[c][3] *= r; }
+            v_ref = fabsf(sc.y);
+        }
+        const float vr = v_ref > 0.f ? sc.y / v_ref : 0.f;
         // P^T as the fp16 B operand: (token x head) fragments transposed to (head x token)
-        const __half2 h01 = __floats2half2_rn(p0, p1), h23 = __floats2half2_rn(p2, p3);
+        const __half2 h01 = __floats2half2_rn(p0 * vr, p1 * vr), h23 = __floats2half2_rn(p2 * vr, p3 * vr);
         const uint32_t pb0 = movmatrix_trans(*reinterpret_cast<const uint32_t *>(&h01));
         const uint32_t pb1 = movmatrix_trans(*reinterpret_cast<const uint32_t *>(&h23));
 
         if (!__all_sync(0xffffffffu, mbar_wait(bv, parity))) { alive = false; break; }
-        if (appending) {
-            const uint32_t a = vbase + new_slot * 128 + ((((lane >> 2) ^ (new_slot & 7)) << 4)) + (lane & 3) * 4;
-            asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(new_v8) : "memory");
-            __syncwarp();
-        }
         if (valid < kPageSize) {
             // V rows past the context may hold NaN codes; 0 * NaN is NaN, so clear them first
             for (int row = valid; row < kPageSize; ++row)
                 if (lane < 8) st_shared_zero16(vbase + row * 128 + lane * 16);
             __syncwarp();
         }
-        // O^T += v_scale * V8^T P^T, two chunks of d per ldmatrix
+        // O^T += V8^T (P v_scale / v_ref)^T, two chunks of d per ldmatrix
 #pragma unroll
         for (int j = 0; j < CHUNKS / 2; ++j) {
             uint32_t r0, r1, r2, r3;  // (chunk 2 j | 2 j + 1) x (tokens 2t, 2t+1 | 2t+8, 2t+9), d = 2 g, 2 g + 1 of the chunk
@@ -366,19 +323,13 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
             r1 = __byte_perm(r1, 0u, 0x3120);
             r2 = __byte_perm(r2, 0u, 0x3120);
             r3 = __byte_perm(r3, 0u, 0x3120);
-            float T0[4] = {0.f, 0.f, 0.f, 0.f}, T1[4] = {0.f, 0.f, 0.f, 0.f};
-            mma_f16_16816(T0, e4m3x2_lo_to_f16x2(r0), e4m3x2_hi_to_f16x2(r0), e4m3x2_lo_to_f16x2(r2), e4m3x2_hi_to_f16x2(r2),
+            mma_f16_16816(O[2 * j], e4m3x2_lo_to_f16x2(r0), e4m3x2_hi_to_f16x2(r0), e4m3x2_lo_to_f16x2(r2), e4m3x2_hi_to_f16x2(r2),
                           pb0, pb1);
-            mma_f16_16816(T1, e4m3x2_lo_to_f16x2(r1), e4m3x2_hi_to_f16x2(r1), e4m3x2_lo_to_f16x2(r3), e4m3x2_hi_to_f16x2(r3),
+            mma_f16_16816(O[2 * j + 1], e4m3x2_lo_to_f16x2(r1), e4m3x2_hi_to_f16x2(r1), e4m3x2_lo_to_f16x2(r3), e4m3x2_hi_to_f16x2(r3),
                           pb0, pb1);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                O[2 * j][i] = fmaf(sc.y, T0[i], O[2 * j][i]);
-                O[2 * j + 1][i] = fmaf(sc.y, T1[i], O[2 * j + 1][i]);
-            }
         }
         __syncwarp();
-        if (valid < kPageSize || appending) fence_proxy_async();  // generic-proxy stores before the next TMA write
+        if (valid < kPageSize) fence_proxy_async();  // generic-proxy stores before the next TMA write
         --inflight;
         issue_next();
         if (++stage == STAGES) { stage = 0; parity ^= 1u; }
@@ -394,7 +345,7 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
             const size_t row0 = static_cast<size_t>(cons.b) * p.Hq + cons.kvh * G + quad_col;
             const bool has_a = quad_col < G, has_b = quad_col + 1 < G;
             if (seg_page0 == 0 && pair_end) {
-                const float inv_a = 1.f / l_a, inv_b = 1.f / l_b;
+                const float inv_a = v_ref / l_a, inv_b = v_ref / l_b;
                 __nv_bfloat16 *oa = p.out + row0 * D + 2 * quad_row, *ob = oa + D;
 #pragma unroll
                 for (int c = 0; c < CHUNKS; ++c) {
@@ -412,8 +363,8 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
                 float *oa = p.part_o + (slot * G + quad_col) * D + 2 * quad_row, *ob = oa + D;
 #pragma unroll
                 for (int c = 0; c < CHUNKS; ++c) {
-                    if (has_a) *reinterpret_cast<float2 *>(oa + 16 * c) = make_float2(O[c][0], O[c][2]);
-                    if (has_b) *reinterpret_cast<float2 *>(ob + 16 * c) = make_float2(O[c][1], O[c][3]);
+                    if (has_a) *reinterpret_cast<float2 *>(oa + 16 * c) = make_float2(O[c][0] * v_ref, O[c][2] * v_ref);
+                    if (has_b) *reinterpret_cast<float2 *>(ob + 16 * c) = make_float2(O[c][1] * v_ref, O[c][3] * v_ref);
                 }
                 if (quad_row == 0) {
                     if (has_a) p.part_ml[slot * G + quad_col] = make_float2(m_a, l_a);
@@ -425,22 +376,18 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
         advance(cons, cum, p.B, p.Hkv);
     }
 
-    bool last_worker = false;
     if (lane == 0) {
         if (!alive) latch_status(p.status, kDevTimeout, -1, worker);
+#ifdef PD_ENABLE_TUNING
+        if (p.trace != nullptr) {  // the buffer holds four words per worker of the 8-warp bf16 kernel: two per worker here
+            const unsigned long long t_exit = global_timer_ns();
+            p.trace[2 * worker] = (t_entry & 0xffffffffull) | (t_first << 32);
+            p.trace[2 * worker + 1] = (t_last & 0xffffffffull) | (t_exit << 32);
+        }
+#endif
         if (atomicAdd(p.status + kSchedDone, 1) == n_workers - 1) {  // the last worker re-arms the claim counter
             p.status[kSchedNext] = 0;
             p.status[kSchedDone] = 0;
-            last_worker = true;
-        }
-    }
-    // fused append: the last worker to finish (every CTA has long read the old lengths) advances them
-    if (FUSED && __shfl_sync(0xffffffffu, static_cast<int>(last_worker), 0)) {
-        for (int i = lane; i < p.B; i += 32) {
-            const int Lold = p.ctx_lens_w[i];
-            if (Lold < 0 || Lold + 1 > p.MP * kPageSize) continue;  // latched as a bad length by the scan
-            const int pid = __ldg(p.page_table + static_cast<size_t>(i) * p.MP + Lold / kPageSize);
-            if (pid >= 0 && pid < p.num_pages) p.ctx_lens_w[i] = Lold + 1;
         }
     }
 }
@@ -448,7 +395,7 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
 template <int WARPS, int STAGES>
 constexpr size_t fp8_smem_bytes() {
     return static_cast<size_t>(WARPS) * STAGES * (2 * kPageSize * kD8) + 1024 + WARPS * STAGES * 16 + WARPS * STAGES * 2 * 8 +
-           sizeof(Plan) + 2 * WARPS * STAGES * 4 + 32 * 4 + (kMaxBatch + 1) * 4;
+           sizeof(Plan) + WARPS * STAGES * 4 + 32 * 4 + (kMaxBatch + 1) * 4;
 }
 
 
@@ -552,9 +499,9 @@ namespace {
 // dependent chains (convert, MMA, softmax) left the issue slots idle: measured 4.4 TB/s with 8 warps x 6
 // stages, 5.5 with 12 x 4, 6.3 with 16 x 3 (128 registers, no spills), which is the shape that is built.
 constexpr int kFp8Warps = 16, kFp8Stages = 3;
-template <bool FUSED, typename F>
+template <typename F>
 cudaError_t with_fp8_kernel(F &&f) {
-    return f(decode_attn_split_fp8_kernel<kFp8Warps, kFp8Stages, FUSED>, fp8_smem_bytes<kFp8Warps, kFp8Stages>(), kFp8Warps);
+    return f(decode_attn_split_fp8_kernel<kFp8Warps, kFp8Stages>, fp8_smem_bytes<kFp8Warps, kFp8Stages>(), kFp8Warps);
 }
 }  // namespace
 
@@ -562,8 +509,7 @@ cudaError_t prepare_decode_attn_fp8() {
     auto set = [](auto *k, size_t bytes, int) {
         return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
     };
-    const cudaError_t e = with_fp8_kernel<false>(set);
-    return e != cudaSuccess ? e : with_fp8_kernel<true>(set);
+    return with_fp8_kernel(set);
 }
 
 cudaError_t launch_decode_attn_fp8(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, int num_ctas,
@@ -571,7 +517,7 @@ cudaError_t launch_decode_attn_fp8(const CUtensorMap &tm_k, const CUtensorMap &t
     auto go = [&](auto *k, size_t bytes, int warps) {
         return launch_pdl(k, dim3(num_ctas), dim3(warps * 32), bytes, stream, p.pdl != 0, tm_k, tm_v, p);
     };
-    return p.fused != 0 ? with_fp8_kernel<true>(go) : with_fp8_kernel<false>(go);
+    return with_fp8_kernel(go);
 }
 
 cudaError_t launch_kv_quantize_pages(const QuantizeParams &p, cudaStream_t stream) {

@@ -92,9 +92,12 @@ __host__ __device__ inline void make_plan(Plan &pl, long long total, int n_worke
         nl = 1;
     } else {
         long long fair = (total + n_workers - 1) / n_workers;
+        // a kernel whose workers all run at the same speed (the FP8 one: bound by its own instruction stream, not by
+        // the memory system) gains nothing from claiming small ranges late and pays for every extra range
+        const int levels = fair <= p.static_fair_max ? 0 : p.halving_levels;
         const int tail = static_cast<int>(max(static_cast<long long>(p.min_pages_auto),
                                               min(static_cast<long long>(p.tail_pages), fair)));
-        for (int l = 0; l < p.halving_levels && nl < kMaxLevels - 1; ++l) {
+        for (int l = 0; l < levels && nl < kMaxLevels - 1; ++l) {
             const long long rem = total - pos;
             const long long size = (rem + 2ll * n_workers - 1) / (2ll * n_workers);
             if (size < 2ll * tail || first + 2 * n_workers > p.max_ranges) break;
@@ -105,7 +108,7 @@ __host__ __device__ inline void make_plan(Plan &pl, long long total, int n_worke
         }
         const long long rem = total - pos;
         if (rem > 0 || nl == 0) {
-            long long size = p.halving_levels > 0 ? tail : max(fair, static_cast<long long>(p.min_pages_auto));
+            long long size = levels > 0 ? tail : max(fair, static_cast<long long>(p.min_pages_auto));
             const long long room = max(1, p.max_ranges - first);
             if ((rem + size - 1) / size > room) size = (rem + room - 1) / room;
             if (size < 1) size = 1;

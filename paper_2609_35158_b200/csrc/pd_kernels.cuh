@@ -45,6 +45,7 @@ struct AttnParams {
     int32_t max_ranges;         // partial slots available beyond one per (sequence, KV head)
     int32_t min_pages_auto;     // lower bound on pages per range in automatic mode
     int32_t halving_levels;     // automatic plan: number of levels whose ranges halve the remaining fair share
+    int32_t static_fair_max;    // automatic plan: with a fair share of at most this many pages per worker, one equal range each (0 = never)
     int32_t tail_pages;         // automatic plan: pages per range of the last level
     int32_t pdl;                // launch with programmatic stream serialization
     // fused one-token append (all null / 0 for plain attention): ctx_lens holds the lengths BEFORE the

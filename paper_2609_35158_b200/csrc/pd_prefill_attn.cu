@@ -363,8 +363,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                     }
                 }
             }
-#pragma unroll
             if constexpr (kD != 64)
+#pragma unroll
                 for (int c = 0; c < kBlock / 64; ++c) tmem_st32(buf + c * 32, *reinterpret_cast<uint32_t(*)[32]>(pk + c * 32));
             tmem_wait_st();
             // V rows past the context inside the last page may hold NaN; 0 * NaN is NaN, so clear them
