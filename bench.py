@@ -744,8 +744,8 @@ def run_fit_b(args):
 # ------------------------------------------------------------------------------------------ FP8 pages
 
 def run_decode_fp8(args):
-    """The decode step over FP8 (e4m3) KV pages: pd_decode_step_fp8 (or, with --step separate, pd_kv_append_fp8 +
-    pd_decode_attn_fp8), device-resident inputs.
+    """The decode step over FP8 (e4m3) KV pages: pd_kv_append_fp8 + pd_decode_attn_fp8 (with --step fused the one call
+    pd_decode_step_fp8, which enqueues the same three kernels), device-resident inputs.
     Bytes per cached token: one byte per K and V value plus the 16-byte scale record of each (page, KV head)."""
     import torch
 
@@ -1076,8 +1076,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer loop (small ncu captures)")
     ap.add_argument("--step", default=None, choices=["separate", "fused"],
-                    help="pd_kv_append + pd_decode_attn (3 launches) or pd_decode_step (2 launches); default: fused for "
-                         "--op decode, separate for --op decode_fp8 (there the fused kernel measured slower)")
+                    help="pd_kv_append + pd_decode_attn (two calls, 3 launches) or pd_decode_step (one call; 2 launches for "
+                         "bf16, the same 3 for FP8, which has no fused kernel); default: fused for --op decode, "
+                         "separate for --op decode_fp8")
     ap.add_argument("--op", default="decode", choices=["decode", "decode_fp8", "kv_transfer", "prefill", "fit_b", "pool_toggle", "read_ceiling"],
                     help="decode = the headline decode step; kv_transfer = page gather + scatter; "
                          "prefill = one append-prefill turn; fit_b = decode step time over batch size, fitted to A + b * B; "
