@@ -757,7 +757,6 @@ def run_decode_fp8(args):
     dev = "cuda:0"
     cfg_id = args.config
     w = wl.WORKLOADS[cfg_id]
-    assert w.head_dim == 128, "FP8 attention is built for head_dim 128"
     K, W = args.steps, args.warmup
     lens0 = wl.context_lengths(cfg_id)
     B = w.batch

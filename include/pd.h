@@ -366,7 +366,7 @@ int pd_fit_decode_cost(const double *concurrency, const double *step_seconds, in
  *   k8, v8     [num_pages][num_kv_heads][16][head_dim] bytes, OCP FP8 E4M3 (bias 7, no infinities,
  *              0x7f / 0xff = NaN, largest finite value 448), device, 16-byte aligned
  *   kv_scales  [num_pages][num_kv_heads][4] fp32 = {k_scale, v_scale, 0, 0}, device, 16-byte aligned
- * and K_t = k_scale * e4m3(byte), V_t = v_scale * e4m3(byte). head_dim must be 128 for attention.
+ * and K_t = k_scale * e4m3(byte), V_t = v_scale * e4m3(byte). head_dim 64 or 128.
  */
 
 /*

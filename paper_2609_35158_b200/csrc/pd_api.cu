@@ -130,10 +130,11 @@ int encode_pool_map_fp8(pd_ctx *ctx, const void *pool, CUtensorMap *out) {
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c.head_dim),
                                 static_cast<cuuint64_t>(c.num_pages) * c.num_kv_heads * c.page_size};
     const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c.head_dim)};
-    const cuuint32_t box[2] = {128, static_cast<cuuint32_t>(c.page_size)};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(c.head_dim), static_cast<cuuint32_t>(c.page_size)};  // one row = head_dim bytes
     const cuuint32_t elem_strides[2] = {1, 1};
     const CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(pool), dims, strides, box,
-                                   elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                   c.head_dim == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         std::snprintf(ctx->last_error, sizeof ctx->last_error, "cuTensorMapEncodeTiled failed (%d)", static_cast<int>(r));
@@ -566,7 +567,6 @@ int fp8_attn_check_args(pd_ctx *ctx, const void *q, const void *k8, const void *
                         const int32_t *page_table, const int32_t *ctx_lens, const void *out, int32_t batch, float sm_scale,
                         int32_t split_pages) {
     if (int rc = check_batch(ctx, batch)) return rc;
-    if (ctx->cfg.head_dim != 128) return fail(ctx, PD_ERR_UNSUPPORTED, "FP8 attention: head_dim must be 128");
     if (!aligned16(q) || !aligned16(k8) || !aligned16(v8) || !aligned16(kv_scales) || !aligned16(out) ||
         page_table == nullptr || ctx_lens == nullptr)
         return fail(ctx, PD_ERR_INVALID_ARG, "FP8 attention: null or misaligned pointer");
@@ -583,7 +583,7 @@ int decode_attn_fp8_impl(pd_ctx *ctx, const void *q, const void *k8, const void 
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return fail(ctx, PD_ERR_CUDA, "cudaSetDevice");
     if (!ctx->fp8_ready) {
-        const cudaError_t e = pd::prepare_decode_attn_fp8();
+        const cudaError_t e = pd::prepare_decode_attn_fp8(ctx->cfg.head_dim);
         if (e != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "fp8 decode kernel attribute", e);
         ctx->fp8_ready = true;
     }
@@ -629,7 +629,7 @@ int decode_attn_fp8_impl(pd_ctx *ctx, const void *q, const void *k8, const void 
     p.trace = ctx->trace;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (hooked) cudaEventRecord(ctx->ev_before, s);
-    cudaError_t err = pd::launch_decode_attn_fp8(ctx->tm_k8, ctx->tm_v8, p, ctx->num_ctas, s);
+    cudaError_t err = pd::launch_decode_attn_fp8(ctx->cfg.head_dim, ctx->tm_k8, ctx->tm_v8, p, ctx->num_ctas, s);
     if (err != cudaSuccess) return fail(ctx, PD_ERR_CUDA, "decode_attn_split_fp8 launch", err);
     if (hooked) {
         cudaEventRecord(ctx->ev_after, s);

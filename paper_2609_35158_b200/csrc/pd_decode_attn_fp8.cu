@@ -3,14 +3,14 @@
 //
 // The decode cost this library exists for is "extra KV-cache HBM reads" per concurrent sequence (Eq. 1):
 // storing the cache in one byte per value halves those bytes. The paper has no such variant; the format
-// is this repository's: K8 / V8 pools [num_pages][num_kv_heads][16][128] of OCP E4M3 bytes and a scale
+// is this repository's: K8 / V8 pools [num_pages][num_kv_heads][16][head_dim] of OCP E4M3 bytes and a scale
 // record {k_scale, v_scale, 0, 0} (fp32) per (page, KV head); K_t = k_scale * e4m3(byte), likewise V.
 //
 // The kernel is the bf16 split kernel's skeleton (same plan of ranges, same warp-private TMA rings, same
 // partial format, same merge kernel) with a different inner product:
-//   * a tile is one 16 x 128 B TMA box (128-byte swizzle); the page's scale record rides along as a
-//     16-byte bulk copy on the K barrier; sixteen worker warps with three stages each keep as many bytes
-//     in flight per SM as the bf16 kernel does;
+//   * a tile is one 16 x head_dim byte TMA box (128-byte swizzle at head_dim 128, 64-byte at 64); the page's
+//     scale record rides along as a 16-byte bulk copy on the K barrier; sixteen worker warps with three
+//     stages each (six at head_dim 64) keep as many bytes in flight per SM as the bf16 kernel does;
 //   * ldmatrix on the byte tile (viewed as b16) hands every lane four consecutive d of a token; two
 //     cvt.rn.f16x2.e4m3x2 make them fp16 pairs, exactly, and Q is converted to fp16 once per segment with
 //     the matching d order, so S^T = K8 Q^T runs on mma.sync fp16 (tokens as M, as in the bf16 kernel);
@@ -20,7 +20,7 @@
 //     bits, no high/low split needed). v_scale is folded into P relative to the largest scale of the segment
 //     so far (O is kept in that unit and rescaled when a larger scale arrives), so the page's product
 //     accumulates straight into O: no temporary accumulator, no per-element multiply.
-// head_dim 128 and |q| below the fp16 range (65504) are required.
+// head_dim 64 or 128; |q| below the fp16 range (65504) is required.
 #include "pd_decode_plan.cuh"
 #include "pd_kernels.cuh"
 #include "pd_ptx.cuh"
@@ -34,7 +34,6 @@ namespace pd {
 
 namespace {
 
-constexpr int kD8 = 128;
 
 __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) {
     const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162 *>(&w);
@@ -42,13 +41,21 @@ __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) {
     return *reinterpret_cast<const uint32_t *>(&h);
 }
 
-template <int WARPS, int STAGES>
+// The 16-byte chunk of a tile row as the TMA swizzle stores it: rows of 128 B under the 128-byte swizzle (chunk
+// index xor the row's low three bits), rows of 64 B under the 64-byte swizzle (xor bits 1-2 of the row); r8 is
+// the row modulo 8. Either way the eight rows of an ldmatrix phase land in eight different 16-byte bank groups.
+template <int D>
+__device__ __forceinline__ int swizzled_chunk(int chunk, int r8) {
+    return D == 128 ? (chunk ^ r8) : (chunk ^ ((r8 >> 1) & 3));
+}
+
+template <int D, int WARPS, int STAGES>
 __global__ void __launch_bounds__(WARPS * 32, 1)
 decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                              const AttnParams p) {
-    constexpr int D = kD8;
+    static_assert(D == 64 || D == 128, "head_dim 64 or 128");
     constexpr int THREADS = WARPS * 32;
-    constexpr int TILE_BYTES = kPageSize * D;    // one TMA box: 16 rows x 128 B
+    constexpr int TILE_BYTES = kPageSize * D;    // one TMA box: 16 rows x D bytes
     constexpr int STAGE_BYTES = 2 * TILE_BYTES;  // K tile then V tile
     constexpr int CHUNKS = D / 16;               // 16-byte chunks per row = MMAs per product
 
@@ -117,9 +124,9 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
     const int quad_col = quad_t * 2;      // accumulator columns: heads quad_col and quad_col + 1
     const int G = p.G;
     const int mat = lane >> 3, r8 = lane & 7;
-    const uint32_t k_row_off = (((mat & 1) * 8 + r8) * 128);   // K tile: matrices 0/1 = tokens 0-7 / 8-15, 2/3 = next chunk
+    const uint32_t k_row_off = (((mat & 1) * 8 + r8) * D);   // K tile: matrices 0/1 = tokens 0-7 / 8-15, 2/3 = next chunk
     const int k_sel = mat >> 1;
-    const uint32_t v_row_off = (((mat >> 1) * 8 + r8) * 128);  // V tile read transposed: matrices 0/1 = chunk, chunk + 1 of tokens 0-7
+    const uint32_t v_row_off = (((mat >> 1) * 8 + r8) * D);  // V tile read transposed: matrices 0/1 = chunk, chunk + 1 of tokens 0-7
     const int v_sel = mat & 1;
 
     PageIdCache pt;
@@ -258,7 +265,7 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
 #pragma unroll
         for (int kk = 0; kk < CHUNKS / 2; ++kk) {
             uint32_t r0, r1, r2, r3;  // (tokens g | g + 8) x (chunk 2 kk | 2 kk + 1), four consecutive d each
-            ldmatrix_x4(r0, r1, r2, r3, kbase + k_row_off + (((kk * 2 + k_sel) ^ r8) << 4));
+            ldmatrix_x4(r0, r1, r2, r3, kbase + k_row_off + (swizzled_chunk<D>(kk * 2 + k_sel, r8) << 4));
             mma_f16_16816(Se, e4m3x2_lo_to_f16x2(r0), e4m3x2_lo_to_f16x2(r1), e4m3x2_hi_to_f16x2(r0), e4m3x2_hi_to_f16x2(r1),
                           qb[2 * kk][0], qb[2 * kk][1]);
             mma_f16_16816(So, e4m3x2_lo_to_f16x2(r2), e4m3x2_lo_to_f16x2(r3), e4m3x2_hi_to_f16x2(r2), e4m3x2_hi_to_f16x2(r3),
@@ -310,14 +317,14 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
         if (valid < kPageSize) {
             // V rows past the context may hold NaN codes; 0 * NaN is NaN, so clear them first
             for (int row = valid; row < kPageSize; ++row)
-                if (lane < 8) st_shared_zero16(vbase + row * 128 + lane * 16);
+                if (lane < D / 16) st_shared_zero16(vbase + row * D + lane * 16);
             __syncwarp();
         }
         // O^T += V8^T (P v_scale / v_ref)^T, two chunks of d per ldmatrix
 #pragma unroll
         for (int j = 0; j < CHUNKS / 2; ++j) {
             uint32_t r0, r1, r2, r3;  // (chunk 2 j | 2 j + 1) x (tokens 2t, 2t+1 | 2t+8, 2t+9), d = 2 g, 2 g + 1 of the chunk
-            ldmatrix_x4_trans(r0, r1, r2, r3, vbase + v_row_off + (((j * 2 + v_sel) ^ r8) << 4));
+            ldmatrix_x4_trans(r0, r1, r2, r3, vbase + v_row_off + (swizzled_chunk<D>(j * 2 + v_sel, r8) << 4));
             // bytes (tok a: d, d+1 | tok a+1: d, d+1) -> (d: tok a, a+1 | d+1: tok a, a+1)
             r0 = __byte_perm(r0, 0u, 0x3120);
             r1 = __byte_perm(r1, 0u, 0x3120);
@@ -392,9 +399,9 @@ decode_attn_split_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __g
     }
 }
 
-template <int WARPS, int STAGES>
+template <int D, int WARPS, int STAGES>
 constexpr size_t fp8_smem_bytes() {
-    return static_cast<size_t>(WARPS) * STAGES * (2 * kPageSize * kD8) + 1024 + WARPS * STAGES * 16 + WARPS * STAGES * 2 * 8 +
+    return static_cast<size_t>(WARPS) * STAGES * (2 * kPageSize * D) + 1024 + WARPS * STAGES * 16 + WARPS * STAGES * 2 * 8 +
            sizeof(Plan) + WARPS * STAGES * 4 + 32 * 4 + (kMaxBatch + 1) * 4;
 }
 
@@ -499,25 +506,29 @@ namespace {
 // dependent chains (convert, MMA, softmax) left the issue slots idle: measured 4.4 TB/s with 8 warps x 6
 // stages, 5.5 with 12 x 4, 6.3 with 16 x 3 (128 registers, no spills), which is the shape that is built.
 constexpr int kFp8Warps = 16, kFp8Stages = 3;
+// head_dim 64: tiles of 1 KB, so twice the stages keep the same bytes in flight
+constexpr int kFp8Stages64 = 6;
 template <typename F>
-cudaError_t with_fp8_kernel(F &&f) {
-    return f(decode_attn_split_fp8_kernel<kFp8Warps, kFp8Stages>, fp8_smem_bytes<kFp8Warps, kFp8Stages>(), kFp8Warps);
+cudaError_t with_fp8_kernel(int head_dim, F &&f) {
+    if (head_dim == 64)
+        return f(decode_attn_split_fp8_kernel<64, kFp8Warps, kFp8Stages64>, fp8_smem_bytes<64, kFp8Warps, kFp8Stages64>(), kFp8Warps);
+    return f(decode_attn_split_fp8_kernel<128, kFp8Warps, kFp8Stages>, fp8_smem_bytes<128, kFp8Warps, kFp8Stages>(), kFp8Warps);
 }
 }  // namespace
 
-cudaError_t prepare_decode_attn_fp8() {
+cudaError_t prepare_decode_attn_fp8(int head_dim) {
     auto set = [](auto *k, size_t bytes, int) {
         return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
     };
-    return with_fp8_kernel(set);
+    return with_fp8_kernel(head_dim, set);
 }
 
-cudaError_t launch_decode_attn_fp8(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, int num_ctas,
-                                   cudaStream_t stream) {
+cudaError_t launch_decode_attn_fp8(int head_dim, const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p,
+                                   int num_ctas, cudaStream_t stream) {
     auto go = [&](auto *k, size_t bytes, int warps) {
         return launch_pdl(k, dim3(num_ctas), dim3(warps * 32), bytes, stream, p.pdl != 0, tm_k, tm_v, p);
     };
-    return with_fp8_kernel(go);
+    return with_fp8_kernel(head_dim, go);
 }
 
 cudaError_t launch_kv_quantize_pages(const QuantizeParams &p, cudaStream_t stream) {

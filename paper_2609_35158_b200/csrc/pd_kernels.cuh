@@ -179,9 +179,9 @@ cudaError_t launch_decode_attn(const AttnVariant &v, const CUtensorMap &tm_k, co
                                const AttnParams &p, int num_ctas, size_t smem_bytes, cudaStream_t stream);
 cudaError_t launch_lse_merge(int head_dim, const AttnParams &p, cudaStream_t stream);
 // FP8 pages (head_dim 128): the split kernel writes the same partials and plan, so launch_lse_merge follows it
-cudaError_t prepare_decode_attn_fp8();
-cudaError_t launch_decode_attn_fp8(const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, int num_ctas,
-                                   cudaStream_t stream);  // p.fused selects the variant that appends the new token itself
+cudaError_t prepare_decode_attn_fp8(int head_dim);
+cudaError_t launch_decode_attn_fp8(int head_dim, const CUtensorMap &tm_k, const CUtensorMap &tm_v, const AttnParams &p, int num_ctas,
+                                   cudaStream_t stream);
 cudaError_t launch_kv_quantize_pages(const QuantizeParams &p, cudaStream_t stream);
 cudaError_t launch_kv_append_fp8(const AppendFp8Params &p, cudaStream_t stream);
 cudaError_t prepare_prefill_attn(int head_dim);  // opt-in shared memory, once

@@ -65,12 +65,12 @@ def test_quantize_pages_bit_exact(Hkv, d):
 GEOMS = [(32, 8), (32, 4), (8, 8), (4, 2), (16, 2)]
 
 
+@pytest.mark.parametrize("d", [128, 64])
 @pytest.mark.parametrize("Hq,Hkv", GEOMS)
 @pytest.mark.parametrize("split_pages", [0, 1, 3, 100000])
-def test_fp8_attention_small_ragged_poisoned(Hq, Hkv, split_pages):
+def test_fp8_attention_small_ragged_poisoned(Hq, Hkv, split_pages, d):
     import paper_2609_35158_b200 as pd
 
-    d = 128
     lens = np.array([1, 15, 16, 17, 31, 33, 64, 300, 1000, 0, 2500], dtype=np.int32)
     cache = wl.build_paged_cache(lens, Hkv, d, seed=81, device=DEV, poison=True)
     cache.v_pages.mul_(0.02)  # small values: a v_scale folded into fp16 probabilities would flush them
@@ -94,7 +94,7 @@ def test_fp8_attention_small_ragged_poisoned(Hq, Hkv, split_pages):
     # outputs here are ~0.02 in magnitude: compare relative to the output scale
     live = lens > 0
     assert_parity((out[torch.from_numpy(live).to(DEV)].float() * 50).to(torch.bfloat16), ref[live] * 50,
-                  f"{Hq}/{Hkv} split {split_pages}", scale_abs_by_magnitude=True)
+                  f"{Hq}/{Hkv} d={d} split {split_pages}", scale_abs_by_magnitude=True)
     got_lse = lse.cpu().numpy()
     assert np.all(np.isneginf(got_lse[~live])) and np.all(out[torch.from_numpy(~live).to(DEV)].float().cpu().numpy() == 0)
     np.testing.assert_allclose(got_lse[live], ref_lse[live], rtol=3e-5, atol=3e-5)
@@ -179,16 +179,44 @@ def test_fp8_append_errors_are_reported_and_skipped():
         assert len(touched) and bool((touched[:, 0] == int(cache.page_table_host[1, 0])).all()) and bool((touched[:, 2] == 5).all())
 
 
-def test_fp8_attention_needs_head_dim_128():
+def test_fp8_head_dim_64_on_the_small_config_geometry():
+    """configs[0]'s geometry (16/2 heads, head_dim 64) through append + attention and through the one-call step:
+    codes, scale records and lengths bit-exact against the oracle's append, attention against the FP8 oracle."""
     import paper_2609_35158_b200 as pd
 
-    with Ctx(8, 2, 64, 1, 1, 4) as ctx:
-        x = torch.zeros(4096, dtype=torch.uint8, device=DEV)
-        q = torch.zeros((1, 8, 64), dtype=torch.bfloat16, device=DEV)
-        i = torch.zeros(4, dtype=torch.int32, device=DEV)
-        with pytest.raises(pd.PdError) as e:
-            pd.pd_decode_attn_fp8(ctx.h, q, x, x, x.view(torch.float32), i, i, q)
-        assert e.value.code == pd.PD_ERR_UNSUPPORTED
+    w = wl.WORKLOADS[0]
+    assert w.head_dim == 64
+    Hq, Hkv, d = w.num_q_heads, w.num_kv_heads, w.head_dim
+    lens0 = wl.context_lengths(0).astype(np.int32)
+    B, steps = len(lens0), 18  # crosses a page boundary for every sequence
+    cache = wl.build_paged_cache(lens0, Hkv, d, seed=95, device=DEV, reserve_tokens=steps)  # codes of empty slots are poisoned below
+    NP, MP = cache.k_pages.shape[0], cache.page_table.shape[1]
+    k8, v8, sc, _ = quantized_on_host(cache, lens0)
+    k8d, v8d, scd = to_dev(k8, v8, sc)
+    lens = lens0.copy()
+    scale = d ** -0.5
+    with Ctx(Hq, Hkv, d, B, MP, NP) as ctx:
+        for i in range(steps):
+            q = wl.random_bf16((B, Hq, d), 960 + i, DEV)
+            kn = wl.random_bf16((B, Hkv, d), 970 + i, DEV)
+            vn = wl.random_bf16((B, Hkv, d), 980 + i, DEV)
+            out = torch.full((B, Hq, d), float("nan"), dtype=torch.bfloat16, device=DEV)
+            lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device=DEV)
+            if i % 2:
+                pd.pd_decode_step_fp8(ctx.h, q, kn, vn, k8d, v8d, scd, cache.page_table, cache.ctx_lens, out, lse, sm_scale=scale)
+            else:
+                pd.pd_kv_append_fp8(ctx.h, kn, vn, k8d, v8d, scd, cache.page_table, cache.ctx_lens)
+                pd.pd_decode_attn_fp8(ctx.h, q, k8d, v8d, scd, cache.page_table, cache.ctx_lens, out, lse, sm_scale=scale)
+            torch.cuda.synchronize()
+            assert pd.pd_device_status(ctx.h)[0] == 0
+            oracle.fp8_kv_append(oracle.bf16_bits(kn), oracle.bf16_bits(vn), k8, v8, sc, cache.page_table_host, lens)
+            assert np.array_equal(cache.ctx_lens.cpu().numpy(), lens)
+            if i in (0, 1, steps - 2, steps - 1):
+                assert np.array_equal(k8d.cpu().numpy(), k8) and np.array_equal(v8d.cpu().numpy(), v8)
+                assert np.array_equal(scd.cpu().numpy().view(np.uint32), sc.view(np.uint32))
+                ref, ref_lse = oracle.fp8_decode_attn(oracle.bf16_bits(q), k8, v8, sc, cache.page_table_host, lens, scale)
+                assert_parity(out, ref, f"head_dim 64 step {i}", scale_abs_by_magnitude=True)
+                np.testing.assert_allclose(lse.cpu().numpy(), ref_lse, rtol=3e-5, atol=3e-5)
 
 
 @pytest.mark.parametrize("config", [1, 3])
@@ -246,7 +274,7 @@ def test_fp8_random_case(seed):
     import paper_2609_35158_b200 as pd
 
     rng = np.random.default_rng(4000 + seed)
-    d = 128
+    d = 128 if seed % 3 else 64
     g = int(rng.choice([1, 2, 4, 8]))
     Hkv = int(rng.choice([1, 2, 4, 8]))
     Hq = g * Hkv
