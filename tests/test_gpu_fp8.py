@@ -219,6 +219,36 @@ def test_fp8_head_dim_64_on_the_small_config_geometry():
                 np.testing.assert_allclose(lse.cpu().numpy(), ref_lse, rtol=3e-5, atol=3e-5)
 
 
+def test_fp8_automatic_plan_is_one_equal_range_per_worker_on_small_totals():
+    """With a fair share of at most 1024 pages per worker the automatic plan of the FP8 kernel is one equal range
+    per worker: the same ranges, hence the same bits, as split_pages = fair share."""
+    import paper_2609_35158_b200 as pd
+
+    Hq, Hkv, d = 32, 8, 128
+    rng = np.random.default_rng(77)
+    lens = rng.integers(3000, 9000, size=24).astype(np.int32)
+    cache = wl.build_paged_cache(lens, Hkv, d, seed=97, device=DEV)
+    k8, v8, sc, _ = quantized_on_host(cache, lens, poison_codes=False)
+    k8d, v8d, scd = to_dev(k8, v8, sc)
+    q = wl.random_bf16((len(lens), Hq, d), 98, DEV)
+    outs, plans = [], []
+    with Ctx(Hq, Hkv, d, len(lens), cache.page_table.shape[1], cache.k_pages.shape[0]) as ctx:
+        pd.pd_decode_attn_fp8(ctx.h, q, k8d, v8d, scd, cache.page_table, cache.ctx_lens, torch.empty_like(q), sm_scale=0.088)
+        torch.cuda.synchronize()
+        auto = pd.pd_last_plan(ctx.h)
+        fair = -(-auto["total_units"] // auto["num_workers"])
+        assert fair <= 1024 and auto["num_ranges"] <= auto["num_workers"] and auto["pages_per_range"] == fair
+        for split in (0, fair):
+            out = torch.full_like(q, float("nan"))
+            pd.pd_decode_attn_fp8(ctx.h, q, k8d, v8d, scd, cache.page_table, cache.ctx_lens, out, sm_scale=0.088, split_pages=split)
+            torch.cuda.synchronize()
+            assert pd.pd_device_status(ctx.h)[0] == 0
+            outs.append(out)
+            plans.append(pd.pd_last_plan(ctx.h))
+    assert plans[0]["num_ranges"] == plans[1]["num_ranges"]
+    assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
+
+
 @pytest.mark.parametrize("config", [1, 3])
 def test_fp8_full_size_config_all_rows(config):
     """Configs 1 and 3 at full size in the automatic split mode: every (sequence, query head) row against the

@@ -70,6 +70,35 @@ def test_prefill_first_token_and_rising_logits():
         assert torch.equal(out[300, h], first)
 
 
+@pytest.mark.parametrize("jump_at", [640, 700, 710, 767])
+def test_prefill_logit_jump_far_beyond_the_slack(jump_at):
+    """Logits that jump by ~200 log2 units inside a block (at its first column, inside its first part, inside its
+    second part, at its last column): the running reference must be raised before any exponential of the part is
+    taken, or the probabilities overflow."""
+    Hq, Hkv, d = 8, 2, 128
+    L = 1100
+    lens = np.array([L], dtype=np.int32)
+    q_lens = np.array([400], dtype=np.int32)  # queries at positions 700..1099: some see the jump, some do not
+    cache = wl.build_paged_cache(lens, Hkv, d, seed=120, device=DEV, poison=True)
+    ip = np.array([0, 400], dtype=np.int32)
+    q = torch.zeros((400, Hq, d), dtype=torch.bfloat16, device=DEV)
+    q[:, :, 0] = 16.0
+    q[:, :, 1:] = (0.05 * wl.random_bf16((400, Hq, d - 1), 121, DEV).float()).to(torch.bfloat16)
+    a = np.where(np.arange(L) >= jump_at, 100.0, 0.0).astype(np.float32)  # 16 * 100 / sqrt(128) = 141 nats
+    pages = torch.from_numpy(cache.page_table_host[0, np.arange(L) // 16].astype(np.int64)).to(DEV)
+    slots = torch.from_numpy(np.arange(L) % 16).to(DEV)
+    for h in range(Hkv):
+        cache.k_pages[pages, h, slots, 0] = torch.from_numpy(a).to(DEV).to(torch.bfloat16)
+    scale = 1.0 / math.sqrt(d)
+    with ctx_for(cache, Hq) as ctx:
+        out, lse = run_prefill(ctx, cache, q, torch.from_numpy(ip).to(DEV), cache.ctx_lens, scale, 400)
+    ref, ref_lse = oracle.prefill_attn(oracle.bf16_bits(q), ip, oracle.bf16_bits(cache.k_pages),
+                                       oracle.bf16_bits(cache.v_pages), cache.page_table_host, lens, scale)
+    assert np.isfinite(out.float().cpu().numpy()).all()
+    assert_parity(out, ref, f"jump at {jump_at}", scale_abs_by_magnitude=True)
+    np.testing.assert_allclose(lse.cpu().numpy(), ref_lse, rtol=3e-5, atol=3e-5)
+
+
 def test_multi_token_append_bit_exact_then_prefill():
     Hq, Hkv, d = 32, 8, 128
     lens0 = np.array([30, 0, 16, 500, 7], dtype=np.int32)
