@@ -57,8 +57,6 @@ struct AttnParams {
     int32_t fused;
     // FP8 pages (null for bf16 pools): {k_scale, v_scale, 0, 0} fp32 per (page, KV head)
     const float *kv_scales;
-    uint8_t *k8_w, *v8_w;       // fused append into FP8 pools: the pools and the scale records, writable
-    float *scales_w;
     int32_t merge_rows;         // rows per CTA of the merge kernel, 0 = chosen from the row count
     // Host-visible result (null / 0 otherwise): the merge kernel delivers every final row to out_host, the
     // device alias of a pinned host buffer [B][Hq][D] (rows the split kernel wrote to `out` are forwarded), and
