@@ -285,7 +285,9 @@ int pd_last_plan(pd_ctx *ctx, void *stream, int64_t *total_units, int32_t *pages
  * pd_plan_ranges: the plan for `total_units` units and `n_workers` worker warps under the given
  * parameters (split_pages as in pd_decode_attn; max_ranges, min_pages, halving_levels, tail_pages as a
  * context holds them: 16 * workers, 4, 6, 16 by default). *n_ranges receives the number of ranges;
- * range r covers units [starts[r], starts[r] + lens[r]). capacity = 0 only counts.
+ * range r covers units [starts[r], starts[r] + lens[r]). capacity = 0 only counts. The FP8 entry points
+ * plan with halving_levels = 0 (one equal range per worker, 16 worker warps per SM) while the fair share
+ * ceil(total_units / n_workers) is at most 1024 pages, and as above beyond that.
  * pd_plan_walk: the triples of `count` consecutive units from `first_unit`, given the exclusive prefix
  * sums of pages per sequence (cum_pages, batch + 1 entries): how a worker finds the start of a range and
  * steps through it.

@@ -78,3 +78,18 @@ def test_plan_rejects_bad_parameters():
         assert e.value.code == pd.PD_ERR_INVALID_ARG
     with pytest.raises(pd.PdError):
         pd.pd_plan_ranges(10, 8, halving_levels=99)
+
+
+def test_equal_ranges_plan_of_the_fp8_entry_points():
+    """halving_levels = 0 is the plan the FP8 kernels take while the fair share is at most 1024 pages: one range
+    of ceil(total / workers) units per worker, at most `workers` ranges, tiling the unit list exactly. The figures
+    are configs[3]'s (192 496 units, 148 SMs x 16 worker warps): 2 348 ranges of 82 units, the last one 42."""
+    import paper_2609_35158_b200 as pd
+
+    total, workers = 192496, 148 * 16
+    starts, lens = pd.pd_plan_ranges(total, workers, 0, 16 * workers, 4, 0, 16)
+    fair = -(-total // workers)
+    assert fair == 82 and len(lens) == 2348 <= workers
+    assert all(n == fair for n in lens[:-1]) and lens[-1] == total - fair * (len(lens) - 1) == 42
+    assert starts[0] == 0 and all(starts[i + 1] == starts[i] + lens[i] for i in range(len(lens) - 1))
+    assert starts[-1] + lens[-1] == total
