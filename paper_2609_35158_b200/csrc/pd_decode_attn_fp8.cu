@@ -506,12 +506,14 @@ namespace {
 // dependent chains (convert, MMA, softmax) left the issue slots idle: measured 4.4 TB/s with 8 warps x 6
 // stages, 5.5 with 12 x 4, 6.3 with 16 x 3 (128 registers, no spills), which is the shape that is built.
 constexpr int kFp8Warps = 16, kFp8Stages = 3;
-// head_dim 64: tiles of 1 KB, so twice the stages keep the same bytes in flight
-constexpr int kFp8Stages64 = 6;
+// head_dim 64: tiles of 1 KB and 96 registers per thread, so more warps (the kernel is bound by its instruction
+// stream there) and more stages per warp
+// (measured on a configs[1]-shaped batch at d = 64: 16 x 6 4066 GB/s, 20 x 5 4425, 24 x 4 4366 with spills, 12 x 8 3413)
+constexpr int kFp8Warps64 = 20, kFp8Stages64 = 5;
 template <typename F>
 cudaError_t with_fp8_kernel(int head_dim, F &&f) {
     if (head_dim == 64)
-        return f(decode_attn_split_fp8_kernel<64, kFp8Warps, kFp8Stages64>, fp8_smem_bytes<64, kFp8Warps, kFp8Stages64>(), kFp8Warps);
+        return f(decode_attn_split_fp8_kernel<64, kFp8Warps64, kFp8Stages64>, fp8_smem_bytes<64, kFp8Warps64, kFp8Stages64>(), kFp8Warps64);
     return f(decode_attn_split_fp8_kernel<128, kFp8Warps, kFp8Stages>, fp8_smem_bytes<128, kFp8Warps, kFp8Stages>(), kFp8Warps);
 }
 }  // namespace
