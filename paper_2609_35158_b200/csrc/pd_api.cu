@@ -201,8 +201,8 @@ int pd_create(const pd_config *cfg, pd_ctx **out) {
     // kernel shape: one CTA per SM, each warp an independent worker with its own stage ring
     pd::AttnVariant v{};
     v.head_dim = cfg->head_dim;
-    v.warps = tune_int("PD_TUNE_WARPS", 8);
-    v.stages = tune_int("PD_TUNE_STAGES", cfg->head_dim == 128 ? 3 : 6);
+    v.warps = tune_int("PD_TUNE_WARPS", cfg->head_dim == 128 ? 8 : 16);
+    v.stages = tune_int("PD_TUNE_STAGES", 3);
     v.hilo = tune_int("PD_TUNE_HILO", 1);
     ctx->variant = v;
     ctx->num_ctas = ctx->num_sms * tune_int("PD_TUNE_CTAS_PER_SM", 1);
