@@ -388,12 +388,46 @@ def run_cuda(args):
     result = measure_decode(head_cfg, args, rank, world, local_rank)
     if others:
         result["per_config"] = per
+        if world == 1 and not args.no_next_rows:
+            result["next_rows"] = measure_next_rows(args)
     if rank == 0:
         print(json.dumps(result), flush=True)
     if world > 1:
         import torch.distributed as dist
 
         dist.destroy_process_group()
+
+
+def measure_next_rows(args):
+    """Short runs of the other operations of the library (what `--op prefill`, `--op decode_fp8`, `--op kv_transfer`
+    print at length), so that the default line also carries a measurement of each; a failure is reported, not raised."""
+    import contextlib
+    import copy
+    import io
+
+    import torch
+
+    rows = {}
+    torch.cuda.empty_cache()  # the headline workload's pools are gone by now; give their memory back first
+    jobs = (("prefill", run_prefill, {"steps": 10, "warmup": 3}),
+            ("decode_fp8 configs[1]", run_decode_fp8, {"steps": 50, "warmup": 10, "config": 1, "step": "separate"}),
+            ("decode_fp8 configs[3]", run_decode_fp8, {"steps": 50, "warmup": 10, "config": 3, "step": "separate"}),
+            ("kv_transfer", run_transfer, {"steps": 20, "warmup": 5}))
+    for name, fn, overrides in jobs:
+        a = copy.copy(args)
+        for k, v in overrides.items():
+            setattr(a, k, v)
+        buf = io.StringIO()
+        try:
+            with contextlib.redirect_stdout(buf):
+                fn(a)
+            line = json.loads([ln for ln in buf.getvalue().splitlines() if ln.startswith("{")][-1])
+            rows[name] = {k: line[k] for k in ("metric", "value", "unit", "steps", "ms_per_step", "roofline", "clocks")
+                          if k in line}
+        except Exception as e:
+            rows[name] = {"error": repr(e)[:300]}
+        torch.cuda.empty_cache()
+    return rows
 
 
 def time_oracle_once(w, cache, q, lens, max_seconds_hint: float = 30.0):
@@ -1074,6 +1108,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference", "stub"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer loop (small ncu captures)")
+    ap.add_argument("--no-next-rows", action="store_true",
+                    help="default run only: skip the short prefill / FP8 decode / KV transfer measurements under next_rows")
     ap.add_argument("--step", default=None, choices=["separate", "fused"],
                     help="pd_kv_append + pd_decode_attn (two calls, 3 launches) or pd_decode_step (one call; 2 launches for "
                          "bf16, the same 3 for FP8, which has no fused kernel); default: fused for --op decode, "
