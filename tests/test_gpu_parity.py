@@ -367,6 +367,37 @@ def test_full_size_configs_all_rows(config):
     print(f"config {config}: max_abs {max_abs:.2e} rel_l2 {rel:.2e} plan {plan}")
 
 
+def test_head_dim_64_with_every_worker_busy():
+    """configs[1]'s batch and context lengths at head_dim 64 (16 worker warps per CTA there): the automatic plan
+    gives every worker ranges of its own and claims more from the counter; every row checked, for the attention
+    call and for the fused step (bit-identical to append + attention)."""
+    Hq, Hkv, d = 32, 8, 64
+    lens = wl.context_lengths(1)
+    B = len(lens)
+    cache = wl.build_paged_cache(lens, Hkv, d, seed=61, device=DEV, reserve_tokens=2)
+    q = wl.random_bf16((B, Hq, d), 161, DEV)
+    scale = d ** -0.5
+    with ctx_for(cache, Hq) as ctx:
+        out, lse = run_attn(ctx, cache, q, cache.ctx_lens, scale)
+        plan = ctx.pd.pd_last_plan(ctx.h)
+        assert plan["num_workers"] == 16 * (plan["num_workers"] // 16) and plan["num_ranges"] > plan["num_workers"]
+        ref, ref_lse = oracle_on_cache(q, cache, lens, scale)
+        assert_parity(out, ref, "head_dim 64, configs[1] lengths")
+        np.testing.assert_allclose(lse.cpu().numpy(), ref_lse, rtol=2e-5, atol=2e-5)
+        # one step both ways on copies of the cache
+        kn = wl.random_bf16((B, Hkv, d), 162, DEV)
+        vn = wl.random_bf16((B, Hkv, d), 163, DEV)
+        k2, v2, l2 = cache.k_pages.clone(), cache.v_pages.clone(), cache.ctx_lens.clone()
+        out_a, out_b = torch.empty_like(q), torch.empty_like(q)
+        ctx.pd.pd_kv_append(ctx.h, kn, vn, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens)
+        ctx.pd.pd_decode_attn(ctx.h, q, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, out_a, sm_scale=scale)
+        ctx.pd.pd_decode_step(ctx.h, q, kn, vn, k2, v2, cache.page_table, l2, out_b, sm_scale=scale)
+        torch.cuda.synchronize()
+        assert ctx.pd.pd_device_status(ctx.h)[0] == 0
+    assert torch.equal(out_a.view(torch.int16), out_b.view(torch.int16))
+    assert torch.equal(cache.k_pages.view(torch.int16), k2.view(torch.int16)) and torch.equal(cache.ctx_lens, l2)
+
+
 def _compact_host_mirror(cache, lens, seq_ids, extra_pages):
     """Host copy of the pages the given sequences own, renumbered 0, 1, 2, ... with `extra_pages` fresh
     (NaN-filled) pages of room behind each sequence, and the table that goes with it."""
