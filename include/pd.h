@@ -131,6 +131,10 @@ int pd_decode_attn(pd_ctx *ctx, const void *q, const void *k_pages, const void *
  * its pools and length stay as they were (its output is then unspecified).
  * Shapes as pd_kv_append and pd_decode_attn; out rows of the step are
  * attention over ctx_lens[b] + 1 tokens.
+ * The call only enqueues kernels on `stream` (no allocation, no synchronisation;
+ * the tensor maps of a pool pointer are encoded on the host the first time it is
+ * seen), so a run of steps can be captured in a CUDA graph after one eager call
+ * and replayed: the lengths advance on the device with every replay.
  */
 int pd_decode_step(pd_ctx *ctx, const void *q, const void *k_new, const void *v_new, void *k_pages,
                    void *v_pages, const int32_t *page_table, int32_t *ctx_lens, void *out, float *lse,

@@ -174,3 +174,45 @@ def test_argument_errors():
             pd.pd_decode_step(ctx.h, q, kn, kn, cache.k_pages, cache.v_pages, cache.page_table, None, out)
         assert e.value.code == pd.PD_ERR_INVALID_ARG
         assert cache.ctx_lens.cpu().tolist() == [5]
+
+
+def test_decode_step_captured_in_a_cuda_graph_replays_bit_identically():
+    """pd_decode_step only enqueues kernels on the given stream (no allocation, no synchronisation, lengths advanced
+    on the device), so a run of steps can be captured once and replayed: pools, lengths and outputs after 24
+    replayed steps equal those of 24 eager steps bit for bit."""
+    import paper_2609_35158_b200 as pd
+
+    w = wl.WORKLOADS[0]
+    lens = wl.context_lengths(0)
+    B, steps, per_graph = w.batch, 24, 6
+    q = wl.random_bf16((B, w.num_q_heads, w.head_dim), 301, DEV)
+    kn = wl.random_bf16((B, w.num_kv_heads, w.head_dim), 302, DEV)
+    vn = wl.random_bf16((B, w.num_kv_heads, w.head_dim), 303, DEV)
+    results = []
+    for use_graph in (False, True):
+        cache = wl.build_paged_cache(lens, w.num_kv_heads, w.head_dim, seed=300, device=DEV, reserve_tokens=steps + 8)
+        out = torch.full_like(q, float("nan"))
+        with ctx_for(cache, w.num_q_heads) as ctx:
+            def step():
+                pd.pd_decode_step(ctx.h, q, kn, vn, cache.k_pages, cache.v_pages, cache.page_table, cache.ctx_lens, out,
+                                  sm_scale=w.sm_scale)
+            step()  # the first call encodes the tensor maps of these pools
+            torch.cuda.synchronize()
+            if use_graph:
+                graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+                with torch.cuda.stream(side), torch.cuda.graph(graph, stream=side):
+                    for _ in range(per_graph):
+                        step()
+                torch.cuda.synchronize()
+                for _ in range(steps // per_graph):
+                    graph.replay()
+            else:
+                for _ in range(steps):
+                    step()
+            torch.cuda.synchronize()
+            assert pd.pd_device_status(ctx.h)[0] == 0
+        results.append((out.clone(), cache.ctx_lens.clone(), cache.k_pages.clone(), cache.v_pages.clone()))
+    (o0, l0, k0, v0), (o1, l1, k1, v1) = results
+    assert torch.equal(l0, l1) and int(l0[0]) == int(lens[0]) + steps + 1
+    assert torch.equal(o0.view(torch.int16), o1.view(torch.int16))
+    assert torch.equal(k0.view(torch.int16), k1.view(torch.int16)) and torch.equal(v0.view(torch.int16), v1.view(torch.int16))
